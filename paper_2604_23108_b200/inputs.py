@@ -1,0 +1,99 @@
+"""Seeded synthetic inputs for the MoHGE layer.
+
+This module only draws random tensors; it holds none of the method's
+arithmetic and imports neither the CUDA binding nor the test oracle, so both
+sides can be fed from it.
+
+Recipe (all on the CPU with one torch.Generator, so the values do not depend
+on the device): draw order x, w_router, dy, w13[g] for g ascending, w2[g] for
+g ascending.  x and dy ~ N(0, 1); every weight ~ N(0, 0.02).  Values are
+drawn in float32 and cast to the layer dtype.  The skewed workload adds a
+Zipf(s = 1.2) log-bias to the group logits (rank = g + 1) and to the expert
+logits (rank = i + 1 inside each group), scaled by `zipf_beta`.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import torch
+
+__all__ = ["Workload", "WORKLOADS", "make_inputs", "zipf_logit_bias"]
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    dtype: str                 # "bf16" | "f32"
+    T: int
+    d_model: int
+    n_groups: int
+    experts_per_group: int
+    group_width: tuple
+    k_groups: int
+    k_experts: int
+    zipf_beta: float = 0.0     # 0: no logit bias
+    seed: int = 0
+
+    @property
+    def n_experts(self) -> int:
+        return self.n_groups * self.experts_per_group
+
+    @property
+    def n_logits(self) -> int:
+        return self.n_groups + self.n_experts
+
+
+# The five benchmark workloads (K_g is not fixed by the benchmark statement;
+# the paper's ratio K_g/N_g = 3/8 rounds to these values for N_g <= 4).
+WORKLOADS = {
+    "cfg1_tiny_f32": Workload("cfg1_tiny_f32", "f32", 256, 128, 2, 4, (256, 128), 1, 2),
+    "cfg2_bf16": Workload("cfg2_bf16", "bf16", 8192, 1024, 3, 8, (1408, 704, 352), 2, 4),
+    "cfg3_bf16_aux": Workload("cfg3_bf16_aux", "bf16", 16384, 2048, 4, 16,
+                              (1536, 1024, 768, 384), 2, 6),
+    "cfg4_bf16_skew": Workload("cfg4_bf16_skew", "bf16", 16384, 2048, 4, 16,
+                               (1536, 1024, 768, 384), 2, 6, zipf_beta=1.0),
+    "cfg5_bf16_large": Workload("cfg5_bf16_large", "bf16", 65536, 4096, 4, 32,
+                                (2048, 1536, 1024, 512), 2, 8),
+}
+
+
+def zipf_logit_bias(wl: Workload, s: float = 1.2) -> Optional[torch.Tensor]:
+    """beta * log(rank^-s / Z) for group ranks and in-group expert ranks."""
+    if wl.zipf_beta == 0.0:
+        return None
+    def logp(n):
+        z = sum(r ** -s for r in range(1, n + 1))
+        return [math.log(r ** -s / z) for r in range(1, n + 1)]
+    gb = logp(wl.n_groups)
+    eb = logp(wl.experts_per_group)
+    vals = gb + eb * wl.n_groups
+    return torch.tensor(vals, dtype=torch.float32) * wl.zipf_beta
+
+
+def _torch_dtype(name: str):
+    return {"bf16": torch.bfloat16, "f32": torch.float32}[name]
+
+
+def make_inputs(wl: Workload, seed: Optional[int] = None, T: Optional[int] = None,
+                weights: bool = True):
+    """Returns a dict of CPU tensors in the layer dtype:
+    x [T,d], w_router [N_g+N_e, d], w13[g] [N, 2W_g, d], w2[g] [N, d, W_g],
+    dy [T,d], logit_bias [N_g+N_e] float32 or None."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(wl.seed if seed is None else seed)
+    dt = _torch_dtype(wl.dtype)
+    T = wl.T if T is None else T
+    d = wl.d_model
+
+    def normal(shape, std):
+        return (torch.randn(shape, generator=gen, dtype=torch.float32) * std).to(dt)
+
+    out = {"x": normal((T, d), 1.0), "w_router": normal((wl.n_logits, d), 0.02),
+           "dy": normal((T, d), 1.0)}
+    if weights:
+        out["w13"] = [normal((wl.experts_per_group, 2 * w, d), 0.02) for w in wl.group_width]
+        out["w2"] = [normal((wl.experts_per_group, d, w), 0.02) for w in wl.group_width]
+    out["logit_bias"] = zipf_logit_bias(wl)
+    return out
