@@ -1,0 +1,213 @@
+/*
+ * mohge.h -- C ABI of the B200 (sm_100a) MoHGE expert layer: forward and backward of the
+ * "Mixture of Heterogeneous Grouped Experts" layer on one GPU.
+ *
+ * Notation follows the paper (Sec. 3.1, 3.2):
+ *   T     tokens in the batch                    d     model width (d_model)
+ *   N_g   expert groups                          N     experts per group,  N_e = N_g * N
+ *   K_g   groups selected per token              K_e   experts selected per token
+ *   W_g   hidden width of every expert of group g (widths differ between groups, Sec. 3.1)
+ *   NL    = N_g + N_e router outputs per token   R     = T * K_e routed token copies ("rows")
+ * Flat expert id e = g * N + i.  Router weight rows: 0..N_g-1 are the group centroids e_g of
+ * Eq. 2, rows N_g.. are the expert embeddings e_{g,i} of Eq. 3, group-major.
+ *
+ * Conventions
+ *   - Every function returns 0 (MOHGE_OK) or a negative mohge_status; mohge_last_error() gives
+ *     the text for the calling thread.  Nothing throws, aborts or traps.
+ *   - Unless a parameter is marked HOST, every pointer is a DEVICE pointer owned by the caller,
+ *     16-byte aligned, row-major and contiguous with the row pitch stated.  The library
+ *     allocates no caller-visible memory, frees nothing, and never synchronises the device:
+ *     work is enqueued on `stream` (a cudaStream_t passed as void*) and the call returns.
+ *   - Arguments are validated before anything is launched; an invalid call launches nothing.
+ *   - `ws` is a caller-provided workspace of mohge_workspace_bytes() bytes.  It holds the
+ *     device status word, tile lists and partial sums.  Calls that share a workspace must be
+ *     ordered on one stream.
+ *   - "dtype" below means the layer dtype of the config: bfloat16 (tensor-core path, FP32
+ *     accumulation) or float32 (plain FP32 FMA path).  Router scores, gate weights, statistics
+ *     and weight gradients are always float32.
+ *   - Physical row numbering: expert segments of the permuted buffers start at multiples of
+ *     `row_align` rows (1 or 128).  `offsets`/`row_of`/`src_of` use the dense numbering
+ *     [0, R); `aligned_offsets`/`prow_of` use the physical one.  Permuted buffers have
+ *     mohge_perm_rows() rows.  Padding rows are kept at zero by the library.
+ *   - Per-group weights: w13[g] is [N, 2*W_g, d] (rows 0..W_g-1 gate projection, W_g..2W_g-1 up
+ *     projection), w2[g] is [N, d, W_g] (down projection); expert E_{g,i}(x) =
+ *     W_down( silu(W_gate x) * (W_up x) ), no bias (the paper only says "FFN with hidden
+ *     dimension W_g", Sec. 3.1; gated-SiLU follows its DeepSeek-V2 baseline, App. A.2).
+ *     The `w13`, `w2`, `dw13`, `dw2` arguments are HOST arrays of N_g device pointers.
+ */
+#ifndef MOHGE_H_
+#define MOHGE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOHGE_MAX_GROUPS 8
+#define MOHGE_MAX_EXPERTS_PER_GROUP 32
+#define MOHGE_MAX_K_EXPERTS 32
+
+enum mohge_dtype { MOHGE_BF16 = 0, MOHGE_F32 = 1 };
+
+enum mohge_status {
+  MOHGE_OK = 0,
+  MOHGE_ERR_INVALID_ARG = -1,
+  MOHGE_ERR_UNSUPPORTED = -2,
+  MOHGE_ERR_WORKSPACE = -3,
+  MOHGE_ERR_CUDA = -4,
+  MOHGE_ERR_TIMEOUT = -5,        /* a device-side bounded wait gave up (status word) */
+  MOHGE_ERR_DEVICE_CHECK = -6    /* a device-side index check failed (status word) */
+};
+
+typedef struct mohge_config {
+  int32_t d_model;                           /* d; multiple of 8 */
+  int32_t n_groups;                          /* N_g <= MOHGE_MAX_GROUPS */
+  int32_t experts_per_group;                 /* N   <= MOHGE_MAX_EXPERTS_PER_GROUP */
+  int32_t k_groups;                          /* K_g, 1..N_g */
+  int32_t k_experts;                         /* K_e, 1..min(K_g*N, MOHGE_MAX_K_EXPERTS) */
+  int32_t group_width[MOHGE_MAX_GROUPS];     /* W_g, any order, each a multiple of 8 */
+  int32_t dtype;                             /* mohge_dtype */
+  float alpha_g;                             /* balance factor of L_G (Eq. 7); paper: 1e-4 */
+  float alpha_e;                             /* balance factor of L_E (Eq. 11); paper: 2.5e-3 */
+  float eps;                                 /* epsilon of Eq. 14 */
+  int32_t f_norm_by_T;                       /* 1: f^G, f^E carry 1/T; 0: Eq. 8 / Eq. 12 literally */
+  int32_t fe_mode;                           /* 0: Eq. 12 literally (top-K_e of ES'); 1: routing mask */
+  int32_t row_align;                         /* 1 or 128; the BF16 path needs 128 */
+} mohge_config;
+
+/* Text of the last error raised on the calling thread ("" if none). HOST. */
+const char* mohge_last_error(void);
+
+/* Bytes of workspace needed for T tokens (0 on invalid config). */
+int64_t mohge_workspace_bytes(const mohge_config* cfg, int64_t T);
+
+/* Number of rows every permuted buffer must have: R + N_e*(row_align-1) rounded up to
+ * row_align (an upper bound of aligned_offsets[N_e]). */
+int64_t mohge_perm_rows(const mohge_config* cfg, int64_t T);
+
+/* Clears the device status word.  Call once after allocating the workspace. */
+int32_t mohge_workspace_init(const mohge_config* cfg, int64_t T, void* ws, void* stream);
+
+/* Copies the device status word to *host_out (HOST) and synchronises `stream`; the only
+ * device-to-host transfer in the library, off the hot path.  0 = no device-side error;
+ * otherwise (code << 24) | detail with code 1 = bounded wait expired, 2 = index check. */
+int32_t mohge_get_device_status(const void* ws, int32_t* host_out, void* stream);
+
+/*
+ * Two-level router, Sec. 3.2, Eq. 2-6.
+ *   logits[t, :] = x_t . W_r^T (+ logit_bias)            arguments of Eq. 2 and Eq. 3
+ *   GS = sigmoid(group logits), top-K_g groups            Eq. 2
+ *   ES' = softmax inside each selected group, else 0      Eq. 3
+ *   ES'' = ES' * GS                                       Eq. 4
+ *   top-K_e of ES'' over all experts                      Eq. 5
+ *   gate = ES''_selected / sum ES''_selected              Eq. 6
+ * "top-K" picks exactly K entries, ties go to the lowest index; slot k of group_idx /
+ * expert_idx holds the k-th largest.  The selection arithmetic is a fixed float32 sequence
+ * (documented in router.cu) so that indices are reproducible bit for bit from the logits.
+ *   x          [T, d] dtype                 w_router  [NL, d] dtype
+ *   logit_bias [NL] float32 or NULL         logits_in [T, NL] float32 or NULL
+ *     (when logits_in is given, x / w_router / logit_bias are not read)
+ *   logits_out [T, NL] float32; required when logits_in is NULL, else may be NULL
+ *   group_idx  [T, K_g] int32    expert_idx [T, K_e] int32    gate_w [T, K_e] float32
+ *   gs_saved   [T, N_g] float32 (GS)        esp_saved [T, N_e] float32 (ES')
+ */
+int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const void* w_router,
+                    const float* logit_bias, const float* logits_in, float* logits_out,
+                    int32_t* group_idx, int32_t* expert_idx, float* gate_w, float* gs_saved,
+                    float* esp_saved, void* ws, void* stream);
+
+/*
+ * Statistics behind the Group-Wise loss (Sec. 3.3, Eq. 7-10) and the Intra-Group Experts loss
+ * (Sec. 3.4.2, Eq. 11-14), and the two loss values.
+ *   group_count[g]         tokens whose top-K_g holds g                    (indicator of Eq. 8)
+ *   group_psum[g]          sum_t GS_{g,t} / sum_j GS_{j,t}                 (Eq. 9-10 before 1/T)
+ *   expert_count_routed[e] tokens routed to e (Eq. 5)
+ *   expert_count_lit[e]    tokens with ES'_{e,t} in top-K_e(ES'_t)         (indicator of Eq. 12)
+ *   expert_psum[e]         sum_t ES'_{e,t} / (sum_{j in g} ES'_{j,t} + eps) (Eq. 13-14 before 1/T)
+ *   loss_out[0] = L_G (Eq. 7), loss_out[1] = L_E (Eq. 11); f carries 1/T when f_norm_by_T,
+ *   L_E uses expert_count_lit (fe_mode 0) or expert_count_routed (fe_mode 1).
+ * Counts are int32 and exact; sums are accumulated in a fixed order (deterministic).
+ */
+int32_t mohge_aux_stats(const mohge_config* cfg, int64_t T, const float* gs_saved,
+                        const float* esp_saved, const int32_t* group_idx,
+                        const int32_t* expert_idx, int32_t* group_count, float* group_psum,
+                        int32_t* expert_count_routed, int32_t* expert_count_lit,
+                        float* expert_psum, float* loss_out, void* ws, void* stream);
+
+/*
+ * Token permutation.  Not a paper equation: the stable counting sort by (expert, token) that
+ * grouped execution of Eq. 15's sum needs.  Integer outputs are deterministic and bit-exact.
+ *   counts [N_e], offsets [N_e+1] (exclusive prefix sum), aligned_offsets [N_e+1],
+ *   row_of [T, K_e], prow_of [T, K_e], src_of [R] (src_of[row_of[t,k]] = t*K_e + k),
+ *   x_perm [mohge_perm_rows, d] dtype: x_perm[prow_of[t,k], :] = x[t, :], padding rows zero.
+ */
+int32_t mohge_dispatch(const mohge_config* cfg, int64_t T, const void* x,
+                       const int32_t* expert_idx, int32_t* counts, int32_t* offsets,
+                       int32_t* aligned_offsets, int32_t* row_of, int32_t* prow_of,
+                       int32_t* src_of, void* x_perm, void* ws, void* stream);
+
+/*
+ * Experts, forward (Sec. 3.1; FFN form see above).  For every physical row r of expert (g,i):
+ *   A = x_perm[r] . W_gate^T, U = x_perm[r] . W_up^T, H = silu(A) * U, y_perm[r] = H . W_down^T
+ *   au_saved [rows, 2*W_max] dtype: A in columns [0, W_g), U in [W_g, 2 W_g) (row pitch 2*W_max)
+ *   h_saved  [rows, W_max] dtype (row pitch W_max)        y_perm [rows, d] dtype
+ */
+int32_t mohge_expert_fwd(const mohge_config* cfg, int64_t T, const void* x_perm,
+                         const int32_t* counts, const int32_t* aligned_offsets,
+                         const void* const* w13, const void* const* w2, void* au_saved,
+                         void* h_saved, void* y_perm, void* ws, void* stream);
+
+/*
+ * Weighted combine: y[t, :] = sum_k gate_w[t,k] * y_perm[prow_of[t,k], :]   (Eq. 15 with the
+ * gate of Eq. 6), FP32 accumulation.   y [T, d] dtype.
+ */
+int32_t mohge_combine(const mohge_config* cfg, int64_t T, const void* y_perm,
+                      const int32_t* prow_of, const float* gate_w, void* y, void* stream);
+
+/*
+ * Backward of the combine:  dgate_w[t,k] = <dy[t], y_perm[prow_of[t,k]]>,
+ * dy_perm[prow_of[t,k], :] = gate_w[t,k] * dy[t, :]; padding rows of dy_perm are zeroed.
+ */
+int32_t mohge_combine_bwd(const mohge_config* cfg, int64_t T, const void* dy, const void* y_perm,
+                          const int32_t* prow_of, const float* gate_w, const int32_t* counts,
+                          const int32_t* aligned_offsets, void* dy_perm, float* dgate_w,
+                          void* stream);
+
+/*
+ * Experts, backward.  dH = dy_perm . W_down;  dW_down = dy_perm^T . H;
+ * dA = dH * U * s(A) * (1 + A (1 - s(A))), dU = dH * silu(A);  dx_perm = [dA, dU] . W13;
+ * dW13 = [dA, dU]^T . x_perm.
+ *   dau [rows, 2*W_max] dtype (output, same layout as au_saved)   dx_perm [rows, d] dtype
+ *   dw13[g] [N, 2 W_g, d] float32, dw2[g] [N, d, W_g] float32; accumulate != 0 adds into them.
+ */
+int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm,
+                         const void* x_perm, const void* au_saved, const void* h_saved,
+                         const int32_t* counts, const int32_t* aligned_offsets,
+                         const void* const* w13, const void* const* w2, void* dau, void* dx_perm,
+                         float* const* dw13, float* const* dw2, int32_t accumulate, void* ws,
+                         void* stream);
+
+/* Backward of the permutation: dx[t, :] = sum_k dx_perm[prow_of[t,k], :].  dx [T, d] dtype. */
+int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,
+                           const int32_t* prow_of, void* dx, void* stream);
+
+/*
+ * Router backward: dgate_w through Eq. 6, 4, 3, 2 (top-k choices carry no gradient) to the
+ * logits, then dw_router = dlogits^T . x and dx += dlogits . W_r.  When group_count and
+ * expert_count are non-NULL the gradients of L_G and L_E (Eq. 7-14, with f^G, f^E constant)
+ * are added; expert_count must be the count selected by fe_mode.
+ *   dlogits [T, NL] float32 (output)    dx [T, d] dtype (accumulated into)
+ *   dw_router [NL, d] float32 (overwritten)
+ */
+int32_t mohge_route_bwd(const mohge_config* cfg, int64_t T, const void* x, const void* w_router,
+                        const float* dgate_w, const float* gs_saved, const float* esp_saved,
+                        const int32_t* group_idx, const int32_t* expert_idx,
+                        const int32_t* group_count, const int32_t* expert_count, float* dlogits,
+                        void* dx, float* dw_router, void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOHGE_H_ */

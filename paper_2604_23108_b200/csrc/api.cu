@@ -1,0 +1,391 @@
+// extern "C" entry points of include/mohge.h: argument validation, workspace carving and the
+// launch sequence of every step.  No allocation, no synchronisation (except the status read).
+
+#include <stdarg.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace mohge {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+int32_t cuda_fail(cudaError_t e, const char* what) {
+  set_error("CUDA error %d (%s) at %s", (int)e, cudaGetErrorString(e), what);
+  return MOHGE_ERR_CUDA;
+}
+
+int32_t make_dims(const mohge_config* c, int64_t T, Dims* D) {
+  MOHGE_CHECK_ARG(c != nullptr, "config is NULL");
+  MOHGE_CHECK_ARG(T >= 0 && T <= (1 << 24), "T = %lld out of range [0, 2^24]", (long long)T);
+  MOHGE_CHECK_ARG(c->n_groups >= 1 && c->n_groups <= MOHGE_MAX_GROUPS, "n_groups = %d not in 1..%d",
+                  c->n_groups, MOHGE_MAX_GROUPS);
+  MOHGE_CHECK_ARG(c->experts_per_group >= 1 && c->experts_per_group <= MOHGE_MAX_EXPERTS_PER_GROUP,
+                  "experts_per_group = %d not in 1..%d", c->experts_per_group,
+                  MOHGE_MAX_EXPERTS_PER_GROUP);
+  MOHGE_CHECK_ARG(c->k_groups >= 1 && c->k_groups <= c->n_groups, "k_groups = %d not in 1..n_groups",
+                  c->k_groups);
+  MOHGE_CHECK_ARG(c->k_experts >= 1 && c->k_experts <= MOHGE_MAX_K_EXPERTS &&
+                      c->k_experts <= c->k_groups * c->experts_per_group,
+                  "k_experts = %d must be in 1..min(%d, k_groups*experts_per_group): Eq. 5 can only "
+                  "pick experts of selected groups",
+                  c->k_experts, MOHGE_MAX_K_EXPERTS);
+  MOHGE_CHECK_ARG(c->dtype == MOHGE_BF16 || c->dtype == MOHGE_F32, "unknown dtype %d", c->dtype);
+  MOHGE_CHECK_ARG(c->d_model >= 8 && c->d_model % 8 == 0, "d_model = %d must be a positive multiple of 8",
+                  c->d_model);
+  MOHGE_CHECK_ARG(c->row_align == 1 || c->row_align == 128, "row_align = %d must be 1 or 128",
+                  c->row_align);
+  MOHGE_CHECK_ARG(c->eps >= 0.0f, "eps must be >= 0");
+  D->d = c->d_model; D->Ng = c->n_groups; D->N = c->experts_per_group;
+  D->P = 1;
+  while (D->P < D->N) D->P *= 2;
+  D->Ne = D->Ng * D->N; D->NL = D->Ng + D->Ne; D->Kg = c->k_groups; D->Ke = c->k_experts;
+  D->Wmax = 0;
+  for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) {
+    D->W[g] = 0;
+    if (g < D->Ng) {
+      MOHGE_CHECK_ARG(c->group_width[g] >= 8 && c->group_width[g] % 8 == 0,
+                      "group_width[%d] = %d must be a positive multiple of 8", g, c->group_width[g]);
+      D->W[g] = c->group_width[g];
+      if (D->W[g] > D->Wmax) D->Wmax = D->W[g];
+    }
+  }
+  D->align = c->row_align;
+  D->T = T; D->R = T * D->Ke;
+  D->Rcap = (D->R + (int64_t)D->Ne * (D->align - 1) + D->align - 1) / D->align * D->align;
+  D->bf16 = c->dtype == MOHGE_BF16;
+  MOHGE_CHECK_ARG(D->Rcap < (1LL << 31) / 2, "too many routed rows (%lld)", (long long)D->Rcap);
+  return MOHGE_OK;
+}
+
+static int64_t up256(int64_t v) { return (v + 255) / 256 * 256; }
+
+WsLayout ws_layout(const Dims& D) {
+  WsLayout L;
+  L.chunks = ceil_div(D.T, kDispatchChunk);
+  L.status_off = 0;
+  L.stats_off = 256;
+  L.hist_off = L.stats_off + up256((int64_t)kStatsBlocks * D.NL * 8);
+  L.base_off = L.hist_off + up256((int64_t)(L.chunks + 1) * D.Ne * 4);
+  L.tiles_off = L.base_off + up256((int64_t)(L.chunks + 1) * D.Ne * 4);
+  // tile capacity: the smallest tile either path uses is 64 x 64
+  const int64_t mt = D.Rcap / 64 + D.Ne + 1;
+  const int64_t wide = (D.d > 2 * D.Wmax ? D.d : 2 * D.Wmax);
+  const int64_t row_tiled = mt * ((wide + 63) / 64);
+  const int64_t wgrad = (int64_t)D.Ne * ((2 * D.Wmax + 63) / 64) * ((D.d + 63) / 64);
+  L.tiles_cap = row_tiled > wgrad ? row_tiled : wgrad;
+  L.total = L.tiles_off + 256 + up256(L.tiles_cap * (int64_t)sizeof(Tile));
+  return L;
+}
+
+struct Ws {
+  int32_t* status;
+  double* stats;
+  int32_t* hist;
+  int32_t* base;
+  int32_t* tile_count;
+  Tile* tiles;
+  int64_t tiles_cap;
+};
+
+static Ws carve(const Dims& D, void* ws) {
+  const WsLayout L = ws_layout(D);
+  char* p = (char*)ws;
+  Ws w;
+  w.status = (int32_t*)(p + L.status_off);
+  w.stats = (double*)(p + L.stats_off);
+  w.hist = (int32_t*)(p + L.hist_off);
+  w.base = (int32_t*)(p + L.base_off);
+  w.tile_count = (int32_t*)(p + L.tiles_off);
+  w.tiles = (Tile*)(p + L.tiles_off + 256);
+  w.tiles_cap = L.tiles_cap;
+  return w;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+#define REQ_PTR(p) MOHGE_CHECK_ARG((p) != nullptr && aligned16(p), #p " must be a non-NULL 16-byte aligned device pointer")
+#define OPT_PTR(p) MOHGE_CHECK_ARG(aligned16(p), #p " must be 16-byte aligned")
+
+static bool force_simt() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("MOHGE_FORCE_SIMT");
+    v = (e && e[0] == '1') ? 1 : 0;
+  }
+  return v == 1;
+}
+
+static int32_t group_ptrs(const Dims& D, const void* const* w13, const void* const* w2,
+                          float* const* dw13, float* const* dw2, GroupPtrs* P) {
+  memset(P, 0, sizeof(*P));
+  for (int g = 0; g < D.Ng; ++g) {
+    if (w13) { REQ_PTR(w13[g]); P->w13[g] = w13[g]; }
+    if (w2) { REQ_PTR(w2[g]); P->w2[g] = w2[g]; }
+    if (dw13) { REQ_PTR(dw13[g]); P->dw13[g] = dw13[g]; }
+    if (dw2) { REQ_PTR(dw2[g]); P->dw2[g] = dw2[g]; }
+  }
+  return MOHGE_OK;
+}
+
+}  // namespace mohge
+
+using namespace mohge;
+
+extern "C" {
+
+const char* mohge_last_error(void) { return g_err; }
+
+int64_t mohge_workspace_bytes(const mohge_config* cfg, int64_t T) {
+  Dims D;
+  if (make_dims(cfg, T, &D) != MOHGE_OK) return 0;
+  return ws_layout(D).total;
+}
+
+int64_t mohge_perm_rows(const mohge_config* cfg, int64_t T) {
+  Dims D;
+  if (make_dims(cfg, T, &D) != MOHGE_OK) return 0;
+  return D.Rcap;
+}
+
+int32_t mohge_workspace_init(const mohge_config* cfg, int64_t T, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(ws);
+  MOHGE_CUDA(cudaMemsetAsync(ws, 0, 256, (cudaStream_t)stream));
+  return MOHGE_OK;
+}
+
+int32_t mohge_get_device_status(const void* ws, int32_t* host_out, void* stream) {
+  MOHGE_CHECK_ARG(ws != nullptr && host_out != nullptr, "ws and host_out must be non-NULL");
+  MOHGE_CUDA(cudaMemcpyAsync(host_out, ws, sizeof(int32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  MOHGE_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  return MOHGE_OK;
+}
+
+int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const void* w_router,
+                    const float* logit_bias, const float* logits_in, float* logits_out,
+                    int32_t* group_idx, int32_t* expert_idx, float* gate_w, float* gs_saved,
+                    float* esp_saved, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  REQ_PTR(group_idx); REQ_PTR(expert_idx); REQ_PTR(gate_w); REQ_PTR(gs_saved); REQ_PTR(esp_saved);
+  REQ_PTR(ws);
+  const float* logits = logits_in;
+  if (!logits_in) {
+    REQ_PTR(x); REQ_PTR(w_router); REQ_PTR(logits_out); OPT_PTR(logit_bias);
+    const int f32 = D.bf16 ? 0 : 1;
+    rc = launch_simt_plain((int)T, D.NL, D.d, x, f32, D.d, 1, w_router, f32, D.d, 1, logits_out, 1,
+                           D.NL, logit_bias, 0, st);
+    if (rc) return rc;
+    logits = logits_out;
+  } else {
+    OPT_PTR(logits_in);
+    if (logits_out && logits_out != logits_in && T > 0)
+      MOHGE_CUDA(cudaMemcpyAsync(logits_out, logits_in, sizeof(float) * T * D.NL,
+                                 cudaMemcpyDeviceToDevice, st));
+  }
+  return launch_router_select(D, logits, group_idx, expert_idx, gate_w, gs_saved, esp_saved, st);
+}
+
+int32_t mohge_aux_stats(const mohge_config* cfg, int64_t T, const float* gs_saved,
+                        const float* esp_saved, const int32_t* group_idx,
+                        const int32_t* expert_idx, int32_t* group_count, float* group_psum,
+                        int32_t* expert_count_routed, int32_t* expert_count_lit,
+                        float* expert_psum, float* loss_out, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(gs_saved); REQ_PTR(esp_saved); REQ_PTR(group_idx); REQ_PTR(expert_idx);
+  REQ_PTR(group_count); REQ_PTR(group_psum); REQ_PTR(expert_count_routed);
+  REQ_PTR(expert_count_lit); REQ_PTR(expert_psum); REQ_PTR(loss_out); REQ_PTR(ws);
+  const Ws w = carve(D, ws);
+  return launch_aux_stats(D, *cfg, gs_saved, esp_saved, group_idx, expert_idx, group_count,
+                          group_psum, expert_count_routed, expert_count_lit, expert_psum, loss_out,
+                          w.stats, (cudaStream_t)stream);
+}
+
+int32_t mohge_dispatch(const mohge_config* cfg, int64_t T, const void* x,
+                       const int32_t* expert_idx, int32_t* counts, int32_t* offsets,
+                       int32_t* aligned_offsets, int32_t* row_of, int32_t* prow_of,
+                       int32_t* src_of, void* x_perm, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(x); REQ_PTR(expert_idx); REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR(aligned_offsets);
+  REQ_PTR(row_of); REQ_PTR(prow_of); REQ_PTR(src_of); REQ_PTR(x_perm); REQ_PTR(ws);
+  const Ws w = carve(D, ws);
+  return launch_dispatch(D, x, expert_idx, counts, offsets, aligned_offsets, row_of, prow_of, src_of,
+                         x_perm, w.hist, w.base, w.status, (cudaStream_t)stream);
+}
+
+int32_t mohge_expert_fwd(const mohge_config* cfg, int64_t T, const void* x_perm,
+                         const int32_t* counts, const int32_t* aligned_offsets,
+                         const void* const* w13, const void* const* w2, void* au_saved,
+                         void* h_saved, void* y_perm, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(x_perm); REQ_PTR(counts); REQ_PTR(aligned_offsets); REQ_PTR(au_saved); REQ_PTR(h_saved);
+  REQ_PTR(y_perm); REQ_PTR(ws);
+  MOHGE_CHECK_ARG(w13 && w2, "w13 and w2 must be host arrays of n_groups device pointers");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, nullptr, nullptr, &P);
+  if (rc) return rc;
+  const Ws w = carve(D, ws);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (D.bf16 && !force_simt()) {
+    MOHGE_CHECK_ARG(D.align == 128, "the BF16 tensor-core path needs row_align = 128");
+    rc = launch_tc_grouped(D, ROLE_FWD1, P, x_perm, nullptr, au_saved, h_saved, counts,
+                           aligned_offsets, 0, w.tile_count, w.tiles, w.tiles_cap, w.status, st);
+    if (rc) return rc;
+    return launch_tc_grouped(D, ROLE_FWD2, P, h_saved, nullptr, y_perm, nullptr, counts,
+                             aligned_offsets, 0, w.tile_count, w.tiles, w.tiles_cap, w.status, st);
+  }
+  rc = launch_build_tiles(D, ROLE_FWD1, 64, 64, counts, aligned_offsets, w.tile_count, w.tiles,
+                          w.tiles_cap, w.status, st);
+  if (rc) return rc;
+  rc = launch_simt_grouped(D, ROLE_FWD1, P, x_perm, nullptr, au_saved, aligned_offsets, 0,
+                           w.tile_count, w.tiles, st);
+  if (rc) return rc;
+  rc = launch_swiglu_fwd(D, aligned_offsets, au_saved, h_saved, st);
+  if (rc) return rc;
+  rc = launch_build_tiles(D, ROLE_FWD2, 64, 64, counts, aligned_offsets, w.tile_count, w.tiles,
+                          w.tiles_cap, w.status, st);
+  if (rc) return rc;
+  return launch_simt_grouped(D, ROLE_FWD2, P, h_saved, nullptr, y_perm, aligned_offsets, 0,
+                             w.tile_count, w.tiles, st);
+}
+
+int32_t mohge_combine(const mohge_config* cfg, int64_t T, const void* y_perm,
+                      const int32_t* prow_of, const float* gate_w, void* y, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(y);
+  return launch_combine(D, y_perm, prow_of, gate_w, y, (cudaStream_t)stream);
+}
+
+int32_t mohge_combine_bwd(const mohge_config* cfg, int64_t T, const void* dy, const void* y_perm,
+                          const int32_t* prow_of, const float* gate_w, const int32_t* counts,
+                          const int32_t* aligned_offsets, void* dy_perm, float* dgate_w,
+                          void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(dy); REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(counts);
+  REQ_PTR(aligned_offsets); REQ_PTR(dy_perm); REQ_PTR(dgate_w);
+  return launch_combine_bwd(D, dy, y_perm, prow_of, gate_w, counts, aligned_offsets, dy_perm,
+                            dgate_w, (cudaStream_t)stream);
+}
+
+int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm,
+                         const void* x_perm, const void* au_saved, const void* h_saved,
+                         const int32_t* counts, const int32_t* aligned_offsets,
+                         const void* const* w13, const void* const* w2, void* dau, void* dx_perm,
+                         float* const* dw13, float* const* dw2, int32_t accumulate, void* ws,
+                         void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(dy_perm); REQ_PTR(x_perm); REQ_PTR(au_saved); REQ_PTR(h_saved); REQ_PTR(counts);
+  REQ_PTR(aligned_offsets); REQ_PTR(dau); REQ_PTR(dx_perm); REQ_PTR(ws);
+  MOHGE_CHECK_ARG(w13 && w2 && dw13 && dw2, "w13, w2, dw13, dw2 must be host arrays of n_groups device pointers");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, dw13, dw2, &P);
+  if (rc) return rc;
+  const Ws w = carve(D, ws);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!accumulate) {
+    rc = launch_zero_empty_wgrad(D, P, counts, st);
+    if (rc) return rc;
+  }
+  if (D.bf16 && !force_simt()) {
+    MOHGE_CHECK_ARG(D.align == 128, "the BF16 tensor-core path needs row_align = 128");
+    const int roles[4] = {ROLE_DGRAD_DOWN, ROLE_WGRAD_DOWN, ROLE_DGRAD_13, ROLE_WGRAD_13};
+    for (int r = 0; r < 4; ++r) {
+      const void* A = nullptr; const void* B = nullptr; void* C = nullptr; void* C2 = nullptr;
+      switch (roles[r]) {
+        case ROLE_DGRAD_DOWN: A = dy_perm; B = au_saved; C = dau; break;
+        case ROLE_WGRAD_DOWN: A = dy_perm; B = h_saved; break;
+        case ROLE_DGRAD_13: A = dau; C = dx_perm; break;
+        default: A = dau; B = x_perm; break;
+      }
+      rc = launch_tc_grouped(D, roles[r], P, A, B, C, C2, counts, aligned_offsets, accumulate,
+                             w.tile_count, w.tiles, w.tiles_cap, w.status, st);
+      if (rc) return rc;
+    }
+    return MOHGE_OK;
+  }
+  struct Step { int role; const void* A; const void* B; void* C; };
+  const Step steps[4] = {{ROLE_DGRAD_DOWN, dy_perm, nullptr, dau},
+                         {ROLE_WGRAD_DOWN, dy_perm, h_saved, nullptr},
+                         {ROLE_DGRAD_13, dau, nullptr, dx_perm},
+                         {ROLE_WGRAD_13, dau, x_perm, nullptr}};
+  for (int s = 0; s < 4; ++s) {
+    rc = launch_build_tiles(D, steps[s].role, 64, 64, counts, aligned_offsets, w.tile_count,
+                            w.tiles, w.tiles_cap, w.status, st);
+    if (rc) return rc;
+    rc = launch_simt_grouped(D, steps[s].role, P, steps[s].A, steps[s].B, steps[s].C,
+                             aligned_offsets, accumulate, w.tile_count, w.tiles, st);
+    if (rc) return rc;
+    if (steps[s].role == ROLE_DGRAD_DOWN) {
+      rc = launch_swiglu_bwd(D, aligned_offsets, au_saved, dau, st);
+      if (rc) return rc;
+    }
+  }
+  return MOHGE_OK;
+}
+
+int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,
+                           const int32_t* prow_of, void* dx, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(dx_perm); REQ_PTR(prow_of); REQ_PTR(dx);
+  return launch_unpermute_sum(D, dx_perm, prow_of, dx, (cudaStream_t)stream);
+}
+
+int32_t mohge_route_bwd(const mohge_config* cfg, int64_t T, const void* x, const void* w_router,
+                        const float* dgate_w, const float* gs_saved, const float* esp_saved,
+                        const int32_t* group_idx, const int32_t* expert_idx,
+                        const int32_t* group_count, const int32_t* expert_count, float* dlogits,
+                        void* dx, float* dw_router, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(x); REQ_PTR(w_router); REQ_PTR(dgate_w); REQ_PTR(gs_saved); REQ_PTR(esp_saved);
+  REQ_PTR(group_idx); REQ_PTR(expert_idx); REQ_PTR(dlogits); REQ_PTR(dx); REQ_PTR(dw_router);
+  REQ_PTR(ws);
+  MOHGE_CHECK_ARG((group_count == nullptr) == (expert_count == nullptr),
+                  "group_count and expert_count must both be given or both be NULL");
+  cudaStream_t st = (cudaStream_t)stream;
+  rc = launch_router_bwd_elementwise(D, *cfg, dgate_w, nullptr, gs_saved, esp_saved, group_idx,
+                                     expert_idx, group_count, expert_count, dlogits, st);
+  if (rc) return rc;
+  const int f32 = D.bf16 ? 0 : 1;
+  if (T == 0) {
+    MOHGE_CUDA(cudaMemsetAsync(dw_router, 0, sizeof(float) * D.NL * D.d, st));
+    return MOHGE_OK;
+  }
+  // dw_router[NL, d] = dlogits^T . x
+  rc = launch_simt_plain(D.NL, D.d, (int)T, dlogits, 1, 1, D.NL, x, f32, 1, D.d, dw_router, 1, D.d,
+                         nullptr, 0, st);
+  if (rc) return rc;
+  // dx[T, d] += dlogits . W_r
+  return launch_simt_plain((int)T, D.d, D.NL, dlogits, 1, D.NL, 1, w_router, f32, 1, D.d, dx, f32,
+                           D.d, nullptr, 1, st);
+}
+
+}  // extern "C"

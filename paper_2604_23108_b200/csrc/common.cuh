@@ -1,0 +1,155 @@
+// Shared host/device declarations of the MoHGE library (internal; the public ABI is include/mohge.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "mohge.h"
+
+namespace mohge {
+
+// ---------------------------------------------------------------- errors
+void set_error(const char* fmt, ...);
+int32_t cuda_fail(cudaError_t e, const char* what);
+
+#define MOHGE_CHECK_ARG(cond, ...)          \
+  do {                                      \
+    if (!(cond)) {                          \
+      ::mohge::set_error(__VA_ARGS__);      \
+      return MOHGE_ERR_INVALID_ARG;         \
+    }                                       \
+  } while (0)
+
+#define MOHGE_CUDA(call)                                        \
+  do {                                                          \
+    cudaError_t e__ = (call);                                   \
+    if (e__ != cudaSuccess) return ::mohge::cuda_fail(e__, #call); \
+  } while (0)
+
+#define MOHGE_LAUNCH_CHECK(name)                                   \
+  do {                                                             \
+    cudaError_t e__ = cudaGetLastError();                          \
+    if (e__ != cudaSuccess) return ::mohge::cuda_fail(e__, name);  \
+  } while (0)
+
+// ---------------------------------------------------------------- derived sizes
+struct Dims {
+  int d, Ng, N, P, Ne, NL, Kg, Ke, Wmax, align;
+  int W[MOHGE_MAX_GROUPS];
+  int64_t T, R, Rcap;
+  bool bf16;
+};
+
+int32_t make_dims(const mohge_config* cfg, int64_t T, Dims* out);  // validates the config
+
+static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+// ---------------------------------------------------------------- workspace layout
+// [0, 256)            device status word (int32) and padding
+// stats partials      double [kStatsBlocks][NL]
+// dispatch histogram  int32 [chunks][Ne] (per-chunk counts) and the same size of chunk bases
+// tile list           int32 count (+pad to 16 B) followed by int4 entries
+constexpr int kStatsBlocks = 296;
+constexpr int kDispatchChunk = 256;  // tokens per dispatch block
+
+struct WsLayout {
+  int64_t status_off, stats_off, hist_off, base_off, tiles_off, total;
+  int64_t tiles_cap;
+  int chunks;
+};
+WsLayout ws_layout(const Dims& D);
+
+// One unit of GEMM work: expert e, output tile origin (m0, n0), and a role-specific extent.
+struct __align__(16) Tile {
+  int32_t e, m0, n0, ext;
+};
+
+struct GroupPtrs {
+  const void* w13[MOHGE_MAX_GROUPS];
+  const void* w2[MOHGE_MAX_GROUPS];
+  float* dw13[MOHGE_MAX_GROUPS];
+  float* dw2[MOHGE_MAX_GROUPS];
+};
+
+struct GroupShape {
+  int W[MOHGE_MAX_GROUPS];
+  int Ng, N, d, Wmax;
+};
+
+enum GemmRole {
+  ROLE_FWD1 = 0,        // AU[rows, 2W]   = Xp[rows, d]    . W13^T
+  ROLE_FWD2 = 1,        // Yp[rows, d]    = H[rows, W]     . W2^T
+  ROLE_DGRAD_DOWN = 2,  // dH[rows, W]    = dYp[rows, d]   . W2
+  ROLE_DGRAD_13 = 3,    // dXp[rows, d]   = dAU[rows, 2W]  . W13
+  ROLE_WGRAD_DOWN = 4,  // dW2[d, W]      = dYp^T . H      (contraction over the expert's rows)
+  ROLE_WGRAD_13 = 5,    // dW13[2W, d]    = dAU^T . Xp
+};
+
+// Parameters of the device-side tile scheduler (build_tiles_kernel).
+struct TilePlan {
+  int role, BM, Ng, N, Ne, d;
+  int BN[MOHGE_MAX_GROUPS];     // tile width per group
+  int Mext[MOHGE_MAX_GROUPS];   // wgrad only: rows of the output (d or 2W)
+  int Next[MOHGE_MAX_GROUPS];   // columns of the output
+  int Kcost[MOHGE_MAX_GROUPS];  // row-tiled roles: contraction length (cost of one tile)
+};
+TilePlan make_plan(const Dims& D, int role, int BM, const int* BN, bool fused_swiglu);
+int32_t launch_build_tiles_plan(const TilePlan& p, const int32_t* aligned, int32_t* tile_count,
+                                Tile* tiles, int64_t tiles_cap, int32_t* status, cudaStream_t st);
+GroupShape make_group_shape(const Dims& D);
+
+// ---------------------------------------------------------------- launchers (each enqueues on `st`)
+// router.cu
+int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_idx,
+                             int32_t* expert_idx, float* gate_w, float* gs, float* esp,
+                             cudaStream_t st);
+int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs, const float* esp,
+                         const int32_t* group_idx, const int32_t* expert_idx, int32_t* group_count,
+                         float* group_psum, int32_t* cnt_routed, int32_t* cnt_lit,
+                         float* expert_psum, float* loss_out, double* partials, cudaStream_t st);
+int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, const float* dgate,
+                                      const float* gate_unused, const float* gs, const float* esp,
+                                      const int32_t* group_idx, const int32_t* expert_idx,
+                                      const int32_t* group_count, const int32_t* expert_count,
+                                      float* dlogits, cudaStream_t st);
+
+// dispatch.cu
+int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx, int32_t* counts,
+                        int32_t* offsets, int32_t* aligned, int32_t* row_of, int32_t* prow_of,
+                        int32_t* src_of, void* x_perm, int32_t* hist, int32_t* base,
+                        int32_t* status, cudaStream_t st);
+int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of,
+                       const float* gate_w, void* y, cudaStream_t st);
+int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
+                           const int32_t* prow_of, const float* gate_w, const int32_t* counts,
+                           const int32_t* aligned, void* dy_perm, float* dgate_w, cudaStream_t st);
+int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* prow_of, void* dx,
+                             cudaStream_t st);
+
+// gemm_simt.cu
+int32_t launch_build_tiles(const Dims& D, int role, int BM, int BN, const int32_t* counts,
+                           const int32_t* aligned, int32_t* tile_count, Tile* tiles,
+                           int64_t tiles_cap, int32_t* status, cudaStream_t st);
+int32_t launch_simt_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
+                            const void* B, void* C, const int32_t* aligned, int accumulate,
+                            const int32_t* tile_count, const Tile* tiles, cudaStream_t st);
+int32_t launch_swiglu_fwd(const Dims& D, const int32_t* aligned, void* au, void* h,
+                          cudaStream_t st);
+int32_t launch_swiglu_bwd(const Dims& D, const int32_t* aligned, const void* au, void* dau,
+                          cudaStream_t st);
+int32_t launch_zero_empty_wgrad(const Dims& D, const GroupPtrs& P, const int32_t* counts,
+                                cudaStream_t st);
+// plain (single problem) GEMMs of the router:  C[M,N] (+)= A . B^T forms with generic strides
+int32_t launch_simt_plain(int M, int N, int K, const void* A, int a_f32, int64_t sAm, int64_t sAk,
+                          const void* B, int b_f32, int64_t sBn, int64_t sBk, void* C, int c_f32,
+                          int64_t sCm, const float* bias, int accumulate, cudaStream_t st);
+
+// gemm_tc.cu (tcgen05 path, BF16)
+int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
+                          const void* B, void* C, void* C2, const int32_t* counts,
+                          const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
+                          int64_t tiles_cap, int32_t* status, cudaStream_t st);
+
+}  // namespace mohge

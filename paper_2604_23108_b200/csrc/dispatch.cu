@@ -1,0 +1,390 @@
+// Token permutation (stable counting sort by expert, then token), row gather, weighted combine
+// and their backward kernels.  All HBM-bound: 16-byte vector accesses, one block per token row.
+//
+// Counting sort, deterministic and bit-exact:
+//   pass 1  every block takes kDispatchChunk consecutive tokens and counts, per expert, how
+//           many of them are routed to it (warp ballots, no atomics)
+//   pass 2  one block scans the per-chunk counts per expert (chunk bases), the totals (counts)
+//           and the exclusive prefix sums over experts (offsets, aligned_offsets)
+//   pass 3  every block recomputes its ballots; the rank of token t for expert e is
+//           chunk base + tokens of earlier warps + earlier lanes, i.e. ascending token order
+
+#include "common.cuh"
+
+namespace mohge {
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kChunkWarps = kDispatchChunk / 32;
+
+// bit e of the lane's 256-bit set <=> the lane's token is routed to expert e
+struct ExpertSet {
+  unsigned w[8];
+};
+
+__device__ __forceinline__ ExpertSet load_set(const int32_t* __restrict__ expert_idx, int t, int T,
+                                              int Ke, int Ne, int32_t* status) {
+  ExpertSet s;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s.w[i] = 0;
+  if (t < T) {
+    for (int k = 0; k < Ke; ++k) {
+      const int e = expert_idx[(size_t)t * Ke + k];
+      if (e < 0 || e >= Ne) {                // index check: record and skip
+        atomicCAS(status, 0, (2 << 24) | 1);
+        continue;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if ((e >> 5) == i) s.w[i] |= 1u << (e & 31);
+    }
+  }
+  return s;
+}
+
+// per-warp counts of every expert -> s_wcnt[warp][e]
+__device__ __forceinline__ void warp_counts(const ExpertSet& s, int Ne, int lane, int* wcnt) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    if (i * 32 < Ne) {
+#pragma unroll 8
+      for (int b = 0; b < 32; ++b) {
+        const unsigned bal = __ballot_sync(kFull, (s.w[i] >> b) & 1u);
+        if (lane == b) wcnt[i * 32 + b] = __popc(bal);
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kDispatchChunk)
+dispatch_hist_kernel(const int32_t* __restrict__ expert_idx, int T, int Ke, int Ne,
+                     int32_t* __restrict__ hist, int32_t* status) {
+  __shared__ int s_wcnt[kChunkWarps][256];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.x * kDispatchChunk + threadIdx.x;
+  const ExpertSet s = load_set(expert_idx, t, T, Ke, Ne, status);
+  warp_counts(s, Ne, lane, s_wcnt[warp]);
+  __syncthreads();
+  for (int e = threadIdx.x; e < Ne; e += blockDim.x) {
+    int c = 0;
+#pragma unroll
+    for (int w = 0; w < kChunkWarps; ++w) c += s_wcnt[w][e];
+    hist[(size_t)blockIdx.x * Ne + e] = c;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+dispatch_scan_kernel(int chunks, int Ne, int align, const int32_t* __restrict__ hist,
+                     int32_t* __restrict__ base, int32_t* __restrict__ counts,
+                     int32_t* __restrict__ offsets, int32_t* __restrict__ aligned) {
+  __shared__ int s_cnt[256];
+  const int e = threadIdx.x;
+  if (e < Ne) {
+    int run = 0;
+    for (int b = 0; b < chunks; ++b) {
+      base[(size_t)b * Ne + e] = run;
+      run += hist[(size_t)b * Ne + e];
+    }
+    counts[e] = run;
+    s_cnt[e] = run;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int o = 0, a = 0;
+    for (int i = 0; i < Ne; ++i) {
+      offsets[i] = o;
+      aligned[i] = a;
+      o += s_cnt[i];
+      a += (s_cnt[i] + align - 1) / align * align;
+    }
+    offsets[Ne] = o;
+    aligned[Ne] = a;
+  }
+}
+
+__global__ void __launch_bounds__(kDispatchChunk)
+dispatch_scatter_kernel(const int32_t* __restrict__ expert_idx, int T, int Ke, int Ne,
+                        const int32_t* __restrict__ base, const int32_t* __restrict__ offsets,
+                        const int32_t* __restrict__ aligned, int32_t* __restrict__ row_of,
+                        int32_t* __restrict__ prow_of, int32_t* __restrict__ src_of,
+                        int32_t* status) {
+  __shared__ int s_wcnt[kChunkWarps][256];
+  __shared__ int s_start[256];     // dense row of the chunk's first token for expert e
+  __shared__ int s_pstart[256];    // same in physical numbering
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.x * kDispatchChunk + threadIdx.x;
+  const ExpertSet s = load_set(expert_idx, t, T, Ke, Ne, status);
+  warp_counts(s, Ne, lane, s_wcnt[warp]);
+  __syncthreads();
+  for (int e = threadIdx.x; e < Ne; e += blockDim.x) {
+    int run = 0;                   // exclusive scan over the warps of the chunk
+#pragma unroll
+    for (int w = 0; w < kChunkWarps; ++w) {
+      const int c = s_wcnt[w][e];
+      s_wcnt[w][e] = run;
+      run += c;
+    }
+    const int b = base[(size_t)blockIdx.x * Ne + e];
+    s_start[e] = offsets[e] + b;
+    s_pstart[e] = aligned[e] + b;
+  }
+  __syncthreads();
+  const unsigned lt = (1u << lane) - 1u;
+  // Rank inside the warp: for slot k every lane holds one expert e; the lanes below it whose
+  // token is also routed to e (in any slot) come first.  The membership ballots are gathered
+  // once per distinct e of the warp; every lane takes part in every ballot (lanes past T hold
+  // empty sets and e = -1).
+  for (int k = 0; k < Ke; ++k) {
+    int e = t < T ? expert_idx[(size_t)t * Ke + k] : -1;
+    if (e >= Ne) e = -1;
+    unsigned todo = __ballot_sync(kFull, e >= 0);
+    unsigned bal = 0;
+    while (todo) {
+      const int leader = __ffs(todo) - 1;
+      const int el = __shfl_sync(kFull, e, leader);
+      unsigned member = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        if ((el >> 5) == i) member = (s.w[i] >> (el & 31)) & 1u;
+      const unsigned b2 = __ballot_sync(kFull, member);
+      const unsigned same = __ballot_sync(kFull, e == el);
+      if (e == el) bal = b2;
+      todo &= ~same;
+    }
+    if (e >= 0) {
+      const int rank = s_wcnt[warp][e] + __popc(bal & lt);
+      const int row = s_start[e] + rank;
+      row_of[(size_t)t * Ke + k] = row;
+      prow_of[(size_t)t * Ke + k] = s_pstart[e] + rank;
+      src_of[row] = t * Ke + k;
+    }
+  }
+}
+
+// ---------------------------------------------------------------- row movers
+struct alignas(16) Vec16 {
+  uint32_t v[4];
+};
+
+__device__ __forceinline__ void unpack(const Vec16& a, float (&f)[8], __nv_bfloat16) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(a.v[i] << 16);
+    f[2 * i + 1] = __uint_as_float(a.v[i] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ Vec16 pack(const float (&f)[8], __nv_bfloat16) {
+  Vec16 a;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    a.v[i] = *reinterpret_cast<const uint32_t*>(&h);
+  }
+  return a;
+}
+__device__ __forceinline__ void unpack(const Vec16& a, float (&f)[8], float) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) f[i] = __uint_as_float(a.v[i]);
+#pragma unroll
+  for (int i = 4; i < 8; ++i) f[i] = 0.0f;
+}
+__device__ __forceinline__ Vec16 pack(const float (&f)[8], float) {
+  Vec16 a;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) a.v[i] = __float_as_uint(f[i]);
+  return a;
+}
+
+// x_perm[prow_of[t,k], :] = x[t, :]   (row_vecs 16-byte vectors per row)
+__global__ void __launch_bounds__(256)
+permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ prow_of, int T, int Ke,
+                    int row_vecs, Vec16* __restrict__ x_perm) {
+  __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
+  for (int t = blockIdx.x; t < T; t += gridDim.x) {
+    __syncthreads();
+    if (threadIdx.x < Ke) s_row[threadIdx.x] = prow_of[(size_t)t * Ke + threadIdx.x];
+    __syncthreads();
+    for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
+      const Vec16 v = x[(size_t)t * row_vecs + c];
+      for (int k = 0; k < Ke; ++k) x_perm[(size_t)s_row[k] * row_vecs + c] = v;
+    }
+  }
+}
+
+// zero the padding rows [aligned[e] + counts[e], aligned[e+1]) of a permuted buffer
+__global__ void __launch_bounds__(256)
+zero_pad_rows_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ aligned,
+                     int row_vecs, Vec16* __restrict__ buf) {
+  const int e = blockIdx.x;
+  const int r0 = aligned[e] + counts[e], r1 = aligned[e + 1];
+  const Vec16 z = {{0, 0, 0, 0}};
+  const size_t n = (size_t)(r1 - r0) * row_vecs;
+  Vec16* p = buf + (size_t)r0 * row_vecs;
+  for (size_t i = (size_t)blockIdx.y * blockDim.x + threadIdx.x; i < n;
+       i += (size_t)gridDim.y * blockDim.x)
+    p[i] = z;
+}
+
+// y[t] = sum_k gate[t,k] * y_perm[prow[t,k]]   (gate == nullptr: plain sum)
+template <typename T>
+__global__ void __launch_bounds__(256)
+combine_kernel(const Vec16* __restrict__ y_perm, const int32_t* __restrict__ prow_of,
+               const float* __restrict__ gate_w, int Tn, int Ke, int row_vecs,
+               Vec16* __restrict__ y) {
+  __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
+  __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
+  for (int t = blockIdx.x; t < Tn; t += gridDim.x) {
+    __syncthreads();
+    if (threadIdx.x < Ke) {
+      s_row[threadIdx.x] = prow_of[(size_t)t * Ke + threadIdx.x];
+      s_g[threadIdx.x] = gate_w ? gate_w[(size_t)t * Ke + threadIdx.x] : 1.0f;
+    }
+    __syncthreads();
+    for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
+      float acc[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+#pragma unroll 4
+      for (int k = 0; k < Ke; ++k) {
+        const Vec16 v = y_perm[(size_t)s_row[k] * row_vecs + c];
+        float f[8];
+        unpack(v, f, T());
+        const float g = s_g[k];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = fmaf(g, f[i], acc[i]);
+      }
+      y[(size_t)t * row_vecs + c] = pack(acc, T());
+    }
+  }
+}
+
+// dgate[t,k] = <dy[t], y_perm[prow[t,k]]>,  dy_perm[prow[t,k]] = gate[t,k] * dy[t]
+template <typename T>
+__global__ void __launch_bounds__(256)
+combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_perm,
+                   const int32_t* __restrict__ prow_of, const float* __restrict__ gate_w, int Tn,
+                   int Ke, int row_vecs, Vec16* __restrict__ dy_perm, float* __restrict__ dgate_w) {
+  __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
+  __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
+  __shared__ float s_red[MOHGE_MAX_K_EXPERTS][8];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  for (int t = blockIdx.x; t < Tn; t += gridDim.x) {
+    __syncthreads();
+    if (threadIdx.x < Ke) {
+      s_row[threadIdx.x] = prow_of[(size_t)t * Ke + threadIdx.x];
+      s_g[threadIdx.x] = gate_w[(size_t)t * Ke + threadIdx.x];
+    }
+    __syncthreads();
+    for (int k = 0; k < Ke; ++k) {
+      float part = 0.0f;
+      const float g = s_g[k];
+      const size_t rbase = (size_t)s_row[k] * row_vecs;
+      for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
+        const Vec16 dv = dy[(size_t)t * row_vecs + c];
+        const Vec16 yv = y_perm[rbase + c];
+        float a[8], b[8], o[8];
+        unpack(dv, a, T());
+        unpack(yv, b, T());
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          part = fmaf(a[i], b[i], part);
+          o[i] = g * a[i];
+        }
+        dy_perm[rbase + c] = pack(o, T());
+      }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
+      if (lane == 0) s_red[k][warp] = part;
+    }
+    __syncthreads();
+    if (threadIdx.x < Ke) {
+      float v = 0.0f;
+      for (int w = 0; w < nwarps; ++w) v += s_red[threadIdx.x][w];
+      dgate_w[(size_t)t * Ke + threadIdx.x] = v;
+    }
+  }
+}
+
+int block_for(int row_vecs) {
+  int b = (row_vecs + 31) / 32 * 32;
+  if (b > 256) b = 256;
+  if (b < 32) b = 32;
+  return b;
+}
+
+}  // namespace
+
+int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx, int32_t* counts,
+                        int32_t* offsets, int32_t* aligned, int32_t* row_of, int32_t* prow_of,
+                        int32_t* src_of, void* x_perm, int32_t* hist, int32_t* base,
+                        int32_t* status, cudaStream_t st) {
+  const int chunks = ceil_div(D.T, kDispatchChunk);
+  const int T = (int)D.T;
+  if (chunks > 0) {
+    dispatch_hist_kernel<<<chunks, kDispatchChunk, 0, st>>>(expert_idx, T, D.Ke, D.Ne, hist, status);
+    MOHGE_LAUNCH_CHECK("dispatch_hist_kernel");
+  }
+  dispatch_scan_kernel<<<1, 256, 0, st>>>(chunks, D.Ne, D.align, hist, base, counts, offsets, aligned);
+  MOHGE_LAUNCH_CHECK("dispatch_scan_kernel");
+  if (chunks == 0) return MOHGE_OK;
+  dispatch_scatter_kernel<<<chunks, kDispatchChunk, 0, st>>>(expert_idx, T, D.Ke, D.Ne, base, offsets,
+                                                            aligned, row_of, prow_of, src_of, status);
+  MOHGE_LAUNCH_CHECK("dispatch_scatter_kernel");
+  const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
+  const int blocks = T < 148 * 16 ? T : 148 * 16;
+  permute_rows_kernel<<<blocks, block_for(row_vecs), 0, st>>>(
+      (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (Vec16*)x_perm);
+  MOHGE_LAUNCH_CHECK("permute_rows_kernel");
+  if (D.align > 1) {
+    zero_pad_rows_kernel<<<dim3(D.Ne, 4), 256, 0, st>>>(counts, aligned, row_vecs, (Vec16*)x_perm);
+    MOHGE_LAUNCH_CHECK("zero_pad_rows_kernel");
+  }
+  return MOHGE_OK;
+}
+
+int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of,
+                       const float* gate_w, void* y, cudaStream_t st) {
+  if (D.T == 0) return MOHGE_OK;
+  const int T = (int)D.T;
+  const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
+  const int blocks = T < 148 * 16 ? T : 148 * 16;
+  if (D.bf16)
+    combine_kernel<__nv_bfloat16><<<blocks, block_for(row_vecs), 0, st>>>(
+        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (Vec16*)y);
+  else
+    combine_kernel<float><<<blocks, block_for(row_vecs), 0, st>>>(
+        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (Vec16*)y);
+  MOHGE_LAUNCH_CHECK("combine_kernel");
+  return MOHGE_OK;
+}
+
+int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* prow_of, void* dx,
+                             cudaStream_t st) {
+  return launch_combine(D, dx_perm, prow_of, nullptr, dx, st);
+}
+
+int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
+                           const int32_t* prow_of, const float* gate_w, const int32_t* counts,
+                           const int32_t* aligned, void* dy_perm, float* dgate_w, cudaStream_t st) {
+  const int T = (int)D.T;
+  const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
+  if (T > 0) {
+    const int blocks = T < 148 * 16 ? T : 148 * 16;
+    if (D.bf16)
+      combine_bwd_kernel<__nv_bfloat16><<<blocks, block_for(row_vecs), 0, st>>>(
+          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs,
+          (Vec16*)dy_perm, dgate_w);
+    else
+      combine_bwd_kernel<float><<<blocks, block_for(row_vecs), 0, st>>>(
+          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs,
+          (Vec16*)dy_perm, dgate_w);
+    MOHGE_LAUNCH_CHECK("combine_bwd_kernel");
+  }
+  if (D.align > 1) {
+    zero_pad_rows_kernel<<<dim3(D.Ne, 4), 256, 0, st>>>(counts, aligned, row_vecs, (Vec16*)dy_perm);
+    MOHGE_LAUNCH_CHECK("zero_pad_rows_kernel");
+  }
+  return MOHGE_OK;
+}
+
+}  // namespace mohge

@@ -1,0 +1,475 @@
+// Two-level router (Sec. 3.2, Eq. 2-6), auxiliary-loss statistics (Eq. 7-14) and the
+// element-wise part of the router backward.  One warp per token.
+//
+// This translation unit is compiled with -fmad=false and every float operation that decides
+// an index is written with an explicit round-to-nearest intrinsic, because the selection is a
+// contract: given the float32 logits, the indices are reproducible bit for bit.
+//
+// Selection arithmetic (IEEE-754 binary32, round to nearest even, no fused multiply-add):
+//   groups   K_g rounds of arg-max over the raw group logits (sigmoid is monotone), ties to
+//            the lowest g
+//   exp_s(z) for z <= 0:  zc = max(z, -100); n = rint(zc * 0x1.715476p+0);
+//            r = zc - n * 0x1.62e4p-1;  r = r - n * 0x1.7f7d1cp-20;
+//            p = Horner (separate multiply, add) with 1/7!, 1/6!, ..., 1/2!, 1, 1 rounded to
+//            float32;  result p * 2^n;  z < -87 gives +0
+//   sig_s(z) e = exp_s(-|z|);  z >= 0 ? 1/(1+e) : e/(1+e)
+//   per selected group g: m = max_i l_i; p_i = exp_s(l_i - m); S = balanced binary tree sum
+//            of p (neighbours first, padded with +0 to a power of two); r = sig_s(l_g) / S;
+//            key_i = p_i * r; ES'_i = p_i / S.  Experts of unselected groups: key = -1.
+//   experts  K_e rounds of arg-max over (key descending, e ascending)
+//   gate_k = key_k / (left-to-right sum of the K_e selected keys)
+//
+// Slot layout inside a warp: group g owns P = next_pow2(N) consecutive slots, slot s = g*P + i
+// lives in lane s % 32, register s / 32; a group never straddles a register because P | 32.
+
+#include "common.cuh"
+
+namespace mohge {
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ float exp_s(float z) {
+  const float zc = fmaxf(z, -100.0f);
+  const float n = rintf(__fmul_rn(zc, 0x1.715476p+0f));
+  float r = __fsub_rn(zc, __fmul_rn(n, 0x1.62e4p-1f));
+  r = __fsub_rn(r, __fmul_rn(n, 0x1.7f7d1cp-20f));
+  float p = 0x1.a01a02p-13f;
+  p = __fadd_rn(__fmul_rn(p, r), 0x1.6c16c2p-10f);
+  p = __fadd_rn(__fmul_rn(p, r), 0x1.111112p-7f);
+  p = __fadd_rn(__fmul_rn(p, r), 0x1.555556p-5f);
+  p = __fadd_rn(__fmul_rn(p, r), 0x1.555556p-3f);
+  p = __fadd_rn(__fmul_rn(p, r), 0x1p-1f);
+  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
+  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
+  int ni = (int)n;
+  ni = ni < -126 ? -126 : (ni > 0 ? 0 : ni);
+  const float scale = __int_as_float((ni + 127) << 23);
+  const float out = __fmul_rn(p, scale);
+  return z < -87.0f ? 0.0f : out;
+}
+
+__device__ __forceinline__ float sig_s(float z) {
+  const float e = exp_s(-fabsf(z));
+  const float den = __fadd_rn(1.0f, e);
+  return z >= 0.0f ? __fdiv_rn(1.0f, den) : __fdiv_rn(e, den);
+}
+
+// K rounds of warp arg-max over (key descending, index ascending).  key[j] belongs to expert
+// eid[j] (ascending in j inside a lane).  Winner of round k is left in lane k (win_e, win_key).
+template <int J>
+__device__ __forceinline__ void warp_topk(float (&key)[J], const int (&eid)[J], int K, int lane,
+                                          int& win_e, float& win_key) {
+  win_e = -1;
+  win_key = 0.0f;
+  for (int k = 0; k < K; ++k) {
+    float bk = -4.0f;
+    int be = 0x7fffffff;
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      if (key[j] > bk) {
+        bk = key[j];
+        be = eid[j];
+      }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ok = __shfl_xor_sync(kFull, bk, off);
+      const int oe = __shfl_xor_sync(kFull, be, off);
+      if (ok > bk || (ok == bk && oe < be)) {
+        bk = ok;
+        be = oe;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < J; ++j)
+      if (eid[j] == be) key[j] = -3.0f;
+    if (lane == k) {
+      win_e = be;
+      win_key = bk;
+    }
+  }
+}
+
+struct RouterShape {
+  int T, Ng, N, P, logP, NL, Ne, Kg, Ke;
+};
+
+template <int J>
+__global__ void __launch_bounds__(256)
+router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* __restrict__ group_idx,
+                     int32_t* __restrict__ expert_idx, float* __restrict__ gate_w,
+                     float* __restrict__ gs_saved, float* __restrict__ esp_saved) {
+  const int lane = threadIdx.x & 31;
+  const int warps_total = (gridDim.x * blockDim.x) >> 5;
+  for (int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < s.T; t += warps_total) {
+    const float* L = logits + (size_t)t * s.NL;
+    // ---- Eq. 2: top-K_g groups by raw logit ----
+    float lg[MOHGE_MAX_GROUPS];
+#pragma unroll
+    for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) lg[g] = g < s.Ng ? L[g] : 0.0f;
+    unsigned gmask = 0;
+    for (int k = 0; k < s.Kg; ++k) {
+      int best = -1;
+      float bv = 0.0f;
+#pragma unroll
+      for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) {
+        if (g < s.Ng && !((gmask >> g) & 1u) && (best < 0 || lg[g] > bv)) {
+          best = g;
+          bv = lg[g];
+        }
+      }
+      gmask |= 1u << best;
+      if (lane == 0) group_idx[(size_t)t * s.Kg + k] = best;
+    }
+    if (lane < s.Ng) gs_saved[(size_t)t * s.Ng + lane] = sig_s(L[lane]);
+    // ---- Eq. 3, 4: keys of the lane's slots ----
+    float key[J];
+    int eid[J];
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int sl = lane + 32 * j;
+      const int g = sl >> s.logP;
+      const int i = sl & (s.P - 1);
+      const bool valid = g < s.Ng && i < s.N;
+      const int e = g * s.N + i;
+      const float l = valid ? L[s.Ng + e] : -INFINITY;
+      float m = l;
+      for (int mask = s.P >> 1; mask > 0; mask >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, mask));
+      const float p = valid ? exp_s(__fsub_rn(l, m)) : 0.0f;
+      float S = p;
+      for (int mask = 1; mask < s.P; mask <<= 1) S = __fadd_rn(S, __shfl_xor_sync(kFull, S, mask));
+      const bool sel = valid && ((gmask >> g) & 1u);
+      const float gl = valid ? L[g] : 0.0f;
+      float kv = valid ? -1.0f : -2.0f;
+      float ev = 0.0f;
+      if (sel) {
+        kv = __fmul_rn(p, __fdiv_rn(sig_s(gl), S));
+        ev = __fdiv_rn(p, S);
+      }
+      key[j] = kv;
+      eid[j] = valid ? e : (0x7ffffff0 + j);
+      if (valid) esp_saved[(size_t)t * s.Ne + e] = ev;
+    }
+    // ---- Eq. 5: top-K_e experts, Eq. 6: normalise ----
+    int we;
+    float wk;
+    warp_topk<J>(key, eid, s.Ke, lane, we, wk);
+    float sum = __shfl_sync(kFull, wk, 0);
+    for (int k = 1; k < s.Ke; ++k) sum = __fadd_rn(sum, __shfl_sync(kFull, wk, k));
+    if (lane < s.Ke) {
+      expert_idx[(size_t)t * s.Ke + lane] = we;
+      gate_w[(size_t)t * s.Ke + lane] = __fdiv_rn(wk, sum);
+    }
+  }
+}
+
+// ---------------------------------------------------------------- statistics (Eq. 7-14)
+constexpr int kStatsThreads = 256;
+constexpr int kStatsWarps = kStatsThreads / 32;
+
+template <int J>
+__global__ void __launch_bounds__(kStatsThreads)
+aux_stats_kernel(RouterShape s, float eps, const float* __restrict__ gs, const float* __restrict__ esp,
+                 const int32_t* __restrict__ group_idx, const int32_t* __restrict__ expert_idx,
+                 int32_t* __restrict__ group_count, int32_t* __restrict__ cnt_routed,
+                 int32_t* __restrict__ cnt_lit, double* __restrict__ partials) {
+  __shared__ int s_cg[MOHGE_MAX_GROUPS];
+  __shared__ int s_cr[256];
+  __shared__ int s_cl[256];
+  __shared__ double s_sum[kStatsWarps][256 + MOHGE_MAX_GROUPS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+    s_cr[i] = 0;
+    s_cl[i] = 0;
+    if (i < MOHGE_MAX_GROUPS) s_cg[i] = 0;
+  }
+  __syncthreads();
+  double accE[J];
+#pragma unroll
+  for (int j = 0; j < J; ++j) accE[j] = 0.0;
+  double accG = 0.0;
+  const int warps_total = gridDim.x * kStatsWarps;
+  for (int t = blockIdx.x * kStatsWarps + warp; t < s.T; t += warps_total) {
+    int myg = lane < s.Kg ? group_idx[(size_t)t * s.Kg + lane] : -1;
+    const unsigned gmask = __reduce_or_sync(kFull, myg >= 0 ? (1u << myg) : 0u);
+    if (myg >= 0) atomicAdd(&s_cg[myg], 1);
+    if (lane < s.Ke) atomicAdd(&s_cr[expert_idx[(size_t)t * s.Ke + lane]], 1);
+    // Eq. 10: s'_g = GS_g / sum_j GS_j
+    const float gv = lane < s.Ng ? gs[(size_t)t * s.Ng + lane] : 0.0f;
+    float gsum = gv;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) gsum += __shfl_xor_sync(kFull, gsum, off);
+    if (lane < s.Ng) accG += (double)(gv / gsum);
+    // Eq. 14 and the Eq. 12 indicator
+    float key[J];
+    int eid[J];
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int sl = lane + 32 * j;
+      const int g = sl >> s.logP;
+      const int i = sl & (s.P - 1);
+      const bool valid = g < s.Ng && i < s.N;
+      const int e = g * s.N + i;
+      const float ev = valid ? esp[(size_t)t * s.Ne + e] : 0.0f;
+      float grp = ev;
+      for (int mask = 1; mask < s.P; mask <<= 1) grp += __shfl_xor_sync(kFull, grp, mask);
+      if (valid) accE[j] += (double)(ev / (grp + eps));
+      const bool sel = valid && ((gmask >> g) & 1u);
+      key[j] = sel ? ev : (valid ? -1.0f : -2.0f);
+      eid[j] = valid ? e : (0x7ffffff0 + j);
+    }
+    int we;
+    float wk;
+    warp_topk<J>(key, eid, s.Ke, lane, we, wk);
+    if (lane < s.Ke) atomicAdd(&s_cl[we], 1);
+  }
+  // fixed-order reduction over the warps of the block, then one partial row per block
+#pragma unroll
+  for (int j = 0; j < J; ++j) {
+    const int sl = lane + 32 * j;
+    const int g = sl >> s.logP, i = sl & (s.P - 1);
+    if (g < s.Ng && i < s.N) s_sum[warp][g * s.N + i] = accE[j];
+  }
+  if (lane < s.Ng) s_sum[warp][256 + lane] = accG;
+  __syncthreads();
+  for (int c = threadIdx.x; c < s.Ne + s.Ng; c += blockDim.x) {
+    const int col = c < s.Ne ? c : 256 + (c - s.Ne);
+    double v = 0.0;
+    for (int w = 0; w < kStatsWarps; ++w) v += s_sum[w][col];
+    partials[(size_t)blockIdx.x * s.NL + c] = v;     // columns: experts first, then groups
+  }
+  for (int i = threadIdx.x; i < s.Ne; i += blockDim.x) {
+    if (s_cr[i]) atomicAdd(&cnt_routed[i], s_cr[i]);
+    if (s_cl[i]) atomicAdd(&cnt_lit[i], s_cl[i]);
+  }
+  if (threadIdx.x < s.Ng && s_cg[threadIdx.x]) atomicAdd(&group_count[threadIdx.x], s_cg[threadIdx.x]);
+}
+
+struct LossParams {
+  float alpha_g, alpha_e;
+  int f_norm_by_T, fe_mode;
+  float w_over_wmax[MOHGE_MAX_GROUPS];
+};
+
+__global__ void aux_finalize_kernel(RouterShape s, LossParams lp, int nblocks,
+                                    const double* __restrict__ partials,
+                                    const int32_t* __restrict__ group_count,
+                                    const int32_t* __restrict__ cnt_routed,
+                                    const int32_t* __restrict__ cnt_lit, float* __restrict__ group_psum,
+                                    float* __restrict__ expert_psum, float* __restrict__ loss_out) {
+  __shared__ double s_tot[256 + MOHGE_MAX_GROUPS];
+  for (int c = threadIdx.x; c < s.NL; c += blockDim.x) {
+    double v = 0.0;
+    for (int b = 0; b < nblocks; ++b) v += partials[(size_t)b * s.NL + c];
+    s_tot[c] = v;
+    if (c < s.Ne) expert_psum[c] = (float)v;
+    else group_psum[c - s.Ne] = (float)v;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const double T = (double)s.T;
+    const double fn = lp.f_norm_by_T ? 1.0 / T : 1.0;
+    double LG = 0.0, LE = 0.0;
+    for (int g = 0; g < s.Ng; ++g) {
+      const double f = (double)s.Ng / s.Kg * group_count[g] * fn;     // Eq. 8
+      LG += lp.w_over_wmax[g] * f * (s_tot[s.Ne + g] / T);             // Eq. 7, 9
+    }
+    const int32_t* ce = lp.fe_mode == 0 ? cnt_lit : cnt_routed;
+    for (int e = 0; e < s.Ne; ++e) {
+      const double f = (double)s.N / s.Ke * ce[e] * fn;                // Eq. 12
+      LE += f * (s_tot[e] / T);                                        // Eq. 11, 13
+    }
+    loss_out[0] = (float)(lp.alpha_g * LG);
+    loss_out[1] = (float)(lp.alpha_e * LE);
+  }
+}
+
+// ---------------------------------------------------------------- router backward (element-wise)
+struct BwdParams {
+  float alpha_g, alpha_e, eps;
+  int f_norm_by_T, with_aux;
+  float w_over_wmax[MOHGE_MAX_GROUPS];
+};
+
+constexpr int kBwdWarps = 8;
+
+template <int J>
+__global__ void __launch_bounds__(kBwdWarps * 32)
+router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
+                  const float* __restrict__ gs, const float* __restrict__ esp,
+                  const int32_t* __restrict__ group_idx, const int32_t* __restrict__ expert_idx,
+                  const int32_t* __restrict__ group_count, const int32_t* __restrict__ expert_count,
+                  float* __restrict__ dlogits) {
+  __shared__ float s_dkey[kBwdWarps][256];
+  __shared__ float s_dgs[kBwdWarps][MOHGE_MAX_GROUPS];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float invT = 1.0f / (float)s.T;
+  const float fn = bp.f_norm_by_T ? invT : 1.0f;
+  const int warps_total = gridDim.x * kBwdWarps;
+  for (int t = blockIdx.x * kBwdWarps + warp; t < s.T; t += warps_total) {
+    for (int i = lane; i < 256; i += 32) s_dkey[warp][i] = 0.0f;
+    const int myg = lane < s.Kg ? group_idx[(size_t)t * s.Kg + lane] : -1;
+    const unsigned gmask = __reduce_or_sync(kFull, myg >= 0 ? (1u << myg) : 0u);
+    // Eq. 6 backward: gate_k = key_k / sum key
+    int ek = -1;
+    float keyk = 0.0f, dgk = 0.0f;
+    if (lane < s.Ke) {
+      ek = expert_idx[(size_t)t * s.Ke + lane];
+      keyk = esp[(size_t)t * s.Ne + ek] * gs[(size_t)t * s.Ng + ek / s.N];
+      dgk = dgate[(size_t)t * s.Ke + lane];
+    }
+    float ssum = keyk;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) ssum += __shfl_xor_sync(kFull, ssum, off);
+    float dot = lane < s.Ke ? dgk * (keyk / ssum) : 0.0f;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(kFull, dot, off);
+    __syncwarp();
+    if (lane < s.Ke) s_dkey[warp][ek] = (dgk - dot) / ssum;
+    __syncwarp();
+    // Eq. 4, 3 backward on the lane's slots
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int sl = lane + 32 * j;
+      const int g = sl >> s.logP;
+      const int i = sl & (s.P - 1);
+      const bool valid = g < s.Ng && i < s.N;
+      const int e = g * s.N + i;
+      const float ev = valid ? esp[(size_t)t * s.Ne + e] : 0.0f;
+      const float gv = valid ? gs[(size_t)t * s.Ng + g] : 0.0f;
+      const float dpp = valid ? s_dkey[warp][e] : 0.0f;
+      float dgs = dpp * ev;                 // dGS_g = sum_i dES''_i ES'_i
+      float desp = dpp * gv;                // dES'_i = dES''_i GS_g
+      const bool sel = valid && ((gmask >> g) & 1u);
+      if (bp.with_aux) {
+        // L_E: S_e = ES'_e / D, D = sum_j ES'_j + eps (selected groups only; ES' is the constant 0 elsewhere)
+        const float fe = valid ? (float)s.N / s.Ke * (float)expert_count[e] * fn : 0.0f;
+        float grp = ev, fes = fe * ev;
+        for (int mask = 1; mask < s.P; mask <<= 1) {
+          grp += __shfl_xor_sync(kFull, grp, mask);
+          fes += __shfl_xor_sync(kFull, fes, mask);
+        }
+        const float Dn = grp + bp.eps;
+        if (sel) desp += bp.alpha_e * invT * (fe / Dn - fes / (Dn * Dn));
+      }
+      float inner = ev * desp;
+      for (int mask = 1; mask < s.P; mask <<= 1) {
+        inner += __shfl_xor_sync(kFull, inner, mask);
+        dgs += __shfl_xor_sync(kFull, dgs, mask);
+      }
+      if (valid) dlogits[(size_t)t * s.NL + s.Ng + e] = ev * (desp - inner);
+      if (valid && i == 0) s_dgs[warp][g] = dgs;
+    }
+    __syncwarp();
+    // Eq. 2 backward (+ L_G through Eq. 10)
+    const float gv = lane < s.Ng ? gs[(size_t)t * s.Ng + lane] : 0.0f;
+    float dG = lane < s.Ng ? s_dgs[warp][lane] : 0.0f;
+    if (bp.with_aux) {
+      const float cg = lane < s.Ng ? bp.w_over_wmax[lane] * ((float)s.Ng / s.Kg) *
+                                         (float)group_count[lane] * fn
+                                   : 0.0f;
+      float Ss = gv, cs = cg * gv;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        Ss += __shfl_xor_sync(kFull, Ss, off);
+        cs += __shfl_xor_sync(kFull, cs, off);
+      }
+      dG += bp.alpha_g * invT * (cg / Ss - cs / (Ss * Ss));
+    }
+    if (lane < s.Ng) dlogits[(size_t)t * s.NL + lane] = dG * gv * (1.0f - gv);
+    __syncwarp();
+  }
+}
+
+RouterShape make_shape(const Dims& D) {
+  RouterShape s;
+  s.T = (int)D.T; s.Ng = D.Ng; s.N = D.N; s.P = D.P; s.NL = D.NL; s.Ne = D.Ne; s.Kg = D.Kg; s.Ke = D.Ke;
+  s.logP = 0;
+  while ((1 << s.logP) < D.P) ++s.logP;
+  return s;
+}
+
+int slots_per_lane(const Dims& D) {
+  const int slots = D.Ng * D.P;
+  int J = 1;
+  while (J * 32 < slots) J *= 2;
+  return J;
+}
+
+}  // namespace
+
+#define MOHGE_DISPATCH_J(J_, ...)                      \
+  switch (J_) {                                        \
+    case 1: { constexpr int JJ = 1; __VA_ARGS__; } break; \
+    case 2: { constexpr int JJ = 2; __VA_ARGS__; } break; \
+    case 4: { constexpr int JJ = 4; __VA_ARGS__; } break; \
+    default: { constexpr int JJ = 8; __VA_ARGS__; } break; \
+  }
+
+int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_idx,
+                             int32_t* expert_idx, float* gate_w, float* gs, float* esp,
+                             cudaStream_t st) {
+  if (D.T == 0) return MOHGE_OK;
+  const RouterShape s = make_shape(D);
+  const int blocks = (int)((D.T + 7) / 8) < 148 * 8 ? (int)((D.T + 7) / 8) : 148 * 8;
+  MOHGE_DISPATCH_J(slots_per_lane(D), (router_select_kernel<JJ><<<blocks, 256, 0, st>>>(
+                                          s, logits, group_idx, expert_idx, gate_w, gs, esp)));
+  MOHGE_LAUNCH_CHECK("router_select_kernel");
+  return MOHGE_OK;
+}
+
+int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs, const float* esp,
+                         const int32_t* group_idx, const int32_t* expert_idx, int32_t* group_count,
+                         float* group_psum, int32_t* cnt_routed, int32_t* cnt_lit,
+                         float* expert_psum, float* loss_out, double* partials, cudaStream_t st) {
+  const RouterShape s = make_shape(D);
+  MOHGE_CUDA(cudaMemsetAsync(group_count, 0, sizeof(int32_t) * D.Ng, st));
+  MOHGE_CUDA(cudaMemsetAsync(cnt_routed, 0, sizeof(int32_t) * D.Ne, st));
+  MOHGE_CUDA(cudaMemsetAsync(cnt_lit, 0, sizeof(int32_t) * D.Ne, st));
+  int blocks = ceil_div(D.T, kStatsWarps);
+  if (blocks > kStatsBlocks) blocks = kStatsBlocks;
+  if (blocks > 0) {
+    MOHGE_DISPATCH_J(slots_per_lane(D),
+                     (aux_stats_kernel<JJ><<<blocks, kStatsThreads, 0, st>>>(
+                         s, cfg.eps, gs, esp, group_idx, expert_idx, group_count, cnt_routed,
+                         cnt_lit, partials)));
+    MOHGE_LAUNCH_CHECK("aux_stats_kernel");
+  }
+  LossParams lp;
+  lp.alpha_g = cfg.alpha_g; lp.alpha_e = cfg.alpha_e;
+  lp.f_norm_by_T = cfg.f_norm_by_T; lp.fe_mode = cfg.fe_mode;
+  for (int g = 0; g < MOHGE_MAX_GROUPS; ++g)
+    lp.w_over_wmax[g] = g < D.Ng ? (float)D.W[g] / (float)D.Wmax : 0.0f;
+  RouterShape s1 = s;
+  if (s1.T == 0) s1.T = 1;   // empty batch: sums are zero, avoid 0/0 in the loss
+  aux_finalize_kernel<<<1, 320, 0, st>>>(s1, lp, blocks, partials, group_count, cnt_routed, cnt_lit,
+                                         group_psum, expert_psum, loss_out);
+  MOHGE_LAUNCH_CHECK("aux_finalize_kernel");
+  return MOHGE_OK;
+}
+
+int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, const float* dgate,
+                                      const float*, const float* gs, const float* esp,
+                                      const int32_t* group_idx, const int32_t* expert_idx,
+                                      const int32_t* group_count, const int32_t* expert_count,
+                                      float* dlogits, cudaStream_t st) {
+  if (D.T == 0) return MOHGE_OK;
+  const RouterShape s = make_shape(D);
+  BwdParams bp;
+  bp.alpha_g = cfg.alpha_g; bp.alpha_e = cfg.alpha_e; bp.eps = cfg.eps;
+  bp.f_norm_by_T = cfg.f_norm_by_T;
+  bp.with_aux = (group_count != nullptr && expert_count != nullptr) ? 1 : 0;
+  for (int g = 0; g < MOHGE_MAX_GROUPS; ++g)
+    bp.w_over_wmax[g] = g < D.Ng ? (float)D.W[g] / (float)D.Wmax : 0.0f;
+  int blocks = ceil_div(D.T, kBwdWarps);
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  MOHGE_DISPATCH_J(slots_per_lane(D),
+                   (router_bwd_kernel<JJ><<<blocks, kBwdWarps * 32, 0, st>>>(
+                       s, bp, dgate, gs, esp, group_idx, expert_idx, group_count, expert_count,
+                       dlogits)));
+  MOHGE_LAUNCH_CHECK("router_bwd_kernel");
+  return MOHGE_OK;
+}
+
+}  // namespace mohge

@@ -1,0 +1,63 @@
+"""CPU-side checks of the C ABI: the library loads, exports every declared symbol, and rejects
+invalid arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2604_23108_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "mohge.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mohge_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2604_23108_b200.build import build
+    build()
+    lib = B.lib()
+    names = _declared_symbols()
+    assert "mohge_route" in names and "mohge_expert_bwd" in names and len(names) >= 13
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(B.exported_symbols())
+
+
+def test_sizes_and_validation_without_a_device():
+    cfg = B.Config(1024, 3, 8, 2, 4, [1408, 704, 352])
+    assert B.mohge_perm_rows(cfg, 8192) == 8192 * 4 + 24 * 127 + (128 - (8192 * 4 + 24 * 127) % 128) % 128
+    assert B.mohge_workspace_bytes(cfg, 8192) > 0
+    lib = B.lib()
+    bad = [
+        dict(k_experts=17),                 # K_e > K_g * N: Eq. 5 could not fill its slots
+        dict(k_groups=4),
+        dict(n_groups=9, group_width=[64] * 9),
+        dict(experts_per_group=33),
+        dict(d_model=1001),
+        dict(group_width=[1408, 700, 352]),
+        dict(row_align=64),
+    ]
+    for kw in bad:
+        args = dict(d_model=1024, n_groups=3, experts_per_group=8, k_groups=2, k_experts=4,
+                    group_width=[1408, 704, 352])
+        args.update(kw)
+        c = B.Config(**args).c() if len(args["group_width"]) <= 8 else None
+        if c is None:
+            c = B.Config(**dict(args, group_width=args["group_width"][:8])).c()
+            c.n_groups = 9
+        assert lib.mohge_workspace_bytes(C.byref(c), 128) == 0, kw
+        rc = lib.mohge_combine(C.byref(c), 128, None, None, None, None, None)
+        assert rc == -1, kw
+        assert len(lib.mohge_last_error()) > 0
+    # NULL and misaligned pointers are refused before any launch
+    good = cfg.c()
+    assert lib.mohge_combine(C.byref(good), 128, None, None, None, None, None) == -1
+    assert lib.mohge_combine(C.byref(good), 128, C.c_void_p(8), C.c_void_p(16), C.c_void_p(16),
+                             C.c_void_p(16), None) == -1
+    assert b"16-byte" in lib.mohge_last_error()
+    assert lib.mohge_route(C.byref(good), -5, *([None] * 12)) == -1

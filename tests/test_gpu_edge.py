@@ -1,0 +1,113 @@
+"""GPU edge cases: degenerate routing (all ties, every token to one expert, empty experts),
+single token, empty batch, K_g sweep, maximum slot count."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2604_23108_b200 import binding as B
+from paper_2604_23108_b200.inputs import Workload, make_inputs
+
+from _util import gpu_cfg, gpu_layer, max_rel, oracle_cfg, oracle_layer, to_np64, tol_for
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare(wl, inp, logits32):
+    fwd, bwd, _ = oracle_layer(wl, inp, logits32=logits32)
+    b, dev = gpu_layer(wl, inp, logits32=logits32)
+    tol = tol_for(wl.dtype)
+    assert (b.expert_idx.cpu().numpy() == fwd["expert_idx"]).all()
+    assert (b.group_idx.cpu().numpy() == fwd["group_idx"]).all()
+    dp = O.dispatch(fwd["expert_idx"], wl.n_experts, gpu_cfg(wl).row_align)
+    assert (b.counts.cpu().numpy() == dp["counts"]).all()
+    assert (b.prow_of.cpu().numpy() == dp["prow_of"]).all()
+    assert (b.src_of.cpu().numpy() == dp["src_of"]).all()
+    assert max_rel(to_np64(b.y), fwd["y"]) <= tol
+    assert max_rel(to_np64(b.dx), bwd["dx"]) <= tol
+    assert max_rel(to_np64(b.dw_router), bwd["dw_r"]) <= tol
+    for g in range(wl.n_groups):
+        assert max_rel(to_np64(b.dw13[g]), bwd["dw13"][g]) <= tol
+        assert max_rel(to_np64(b.dw2[g]), bwd["dw2"][g]) <= tol
+    return fwd, b
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_all_logits_equal_ties_go_to_lowest_index(dtype):
+    wl = Workload("ties", dtype, 300, 64, 3, 4, (64, 32, 48), 2, 6, seed=7)
+    inp = make_inputs(wl)
+    logits = np.zeros((wl.T, wl.n_logits), np.float32)
+    fwd, b = _compare(wl, inp, logits)
+    assert (fwd["expert_idx"] == np.arange(6)).all()          # experts 0..5, half of them empty after
+    assert (b.counts.cpu().numpy()[6:] == 0).all()
+    for g in (2,):                                            # empty experts: exactly zero gradients
+        assert float(b.dw13[g].abs().max()) == 0.0 and float(b.dw2[g].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_every_token_to_one_expert_set(dtype):
+    wl = Workload("funnel", dtype, 700, 64, 2, 8, (96, 40), 1, 2, seed=8)
+    inp = make_inputs(wl)
+    logits = np.zeros((wl.T, wl.n_logits), np.float32)
+    logits[:, 1] = 3.0                    # group 1 always wins
+    logits[:, 2 + 8 + 5] = 4.0            # its expert 5 first, expert 2 second
+    logits[:, 2 + 8 + 2] = 2.0
+    fwd, b = _compare(wl, inp, logits)
+    cnt = b.counts.cpu().numpy()
+    assert cnt[13] == wl.T and cnt[10] == wl.T and cnt.sum() == 2 * wl.T
+
+
+@pytest.mark.parametrize("dtype,T", [("f32", 1), ("bf16", 1), ("bf16", 129), ("f32", 257)])
+def test_tiny_batches(dtype, T):
+    wl = Workload("tiny", dtype, T, 64, 2, 4, (64, 32), 1, 2, seed=9)
+    inp = make_inputs(wl)
+    _, _, logits32 = oracle_layer(wl, inp)
+    _compare(wl, inp, logits32)
+
+
+@pytest.mark.parametrize("K_g", [1, 2, 3, 4])
+def test_group_budget_sweep(K_g):
+    wl = Workload("kg", "f32", 200, 32, 4, 4, (32, 24, 16, 8), K_g, min(6, 4 * K_g), seed=10)
+    inp = make_inputs(wl)
+    _, _, logits32 = oracle_layer(wl, inp)
+    _compare(wl, inp, logits32)
+
+
+def test_maximum_router_width():
+    # N_g = 8 groups of N = 32 experts: 256 expert slots, 8 per lane; K_e = 32 fills every lane
+    wl = Workload("max", "f32", 150, 32, 8, 32, (8,) * 8, 3, 32, seed=11)
+    inp = make_inputs(wl)
+    _, _, logits32 = oracle_layer(wl, inp)
+    _compare(wl, inp, logits32)
+
+
+def test_empty_batch_launches_nothing_and_zeroes_statistics():
+    wl = Workload("empty", "f32", 0, 32, 2, 4, (32, 16), 1, 2)
+    gcfg = gpu_cfg(wl)
+    b = B.LayerBuffers(gcfg, 0)
+    x = torch.zeros(1, 32, device="cuda")
+    wr = torch.zeros(wl.n_logits, 32, device="cuda")
+    w13 = [torch.zeros(4, 2 * w, 32, device="cuda") for w in wl.group_width]
+    w2 = [torch.zeros(4, 32, w, device="cuda") for w in wl.group_width]
+    B.layer_forward(gcfg, b, x, wr, w13, w2)
+    B.layer_backward(gcfg, b, x, wr, w13, w2, x)
+    torch.cuda.synchronize()
+    assert int(b.counts.sum()) == 0 and int(b.aligned[wl.n_experts]) == 0
+    assert float(b.dw_router.abs().max()) == 0.0
+    assert all(float(t.abs().max()) == 0.0 for t in b.dw13 + b.dw2)
+    assert B.mohge_get_device_status(b.ws) == 0
+
+
+def test_out_of_range_expert_index_sets_the_status_word_without_faulting():
+    wl = Workload("badidx", "f32", 64, 32, 2, 4, (32, 16), 1, 2)
+    gcfg = gpu_cfg(wl)
+    b = B.LayerBuffers(gcfg, 64)
+    x = torch.zeros(64, 32, device="cuda")
+    idx = torch.zeros(64, 2, dtype=torch.int32, device="cuda")
+    idx[:, 1] = 1
+    idx[5, 1] = 99                                    # not an expert: skipped and reported
+    B.mohge_dispatch(gcfg, 64, x, idx, b.counts, b.offsets, b.aligned, b.row_of, b.prow_of,
+                     b.src_of, b.x_perm, b.ws)
+    torch.cuda.synchronize()
+    assert B.mohge_get_device_status(b.ws) >> 24 == 2
+    assert int(b.counts.sum()) == 127
