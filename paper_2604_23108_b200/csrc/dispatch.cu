@@ -157,6 +157,9 @@ dispatch_scatter_kernel(const int32_t* __restrict__ expert_idx, int T, int Ke, i
       row_of[(size_t)t * Ke + k] = row;
       prow_of[(size_t)t * Ke + k] = s_pstart[e] + rank;
       src_of[row] = t * Ke + k;
+    } else if (t < T) {
+      row_of[(size_t)t * Ke + k] = -1;         // not an expert: no row (also reported in status)
+      prow_of[(size_t)t * Ke + k] = -1;
     }
   }
 }
@@ -198,7 +201,7 @@ __device__ __forceinline__ Vec16 pack(const float (&f)[8], float) {
 // x_perm[prow_of[t,k], :] = x[t, :]   (row_vecs 16-byte vectors per row)
 __global__ void __launch_bounds__(256)
 permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ prow_of, int T, int Ke,
-                    int row_vecs, Vec16* __restrict__ x_perm) {
+                    int row_vecs, int rows_cap, Vec16* __restrict__ x_perm) {
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   for (int t = blockIdx.x; t < T; t += gridDim.x) {
     __syncthreads();
@@ -206,7 +209,8 @@ permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ pro
     __syncthreads();
     for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
       const Vec16 v = x[(size_t)t * row_vecs + c];
-      for (int k = 0; k < Ke; ++k) x_perm[(size_t)s_row[k] * row_vecs + c] = v;
+      for (int k = 0; k < Ke; ++k)
+        if ((unsigned)s_row[k] < (unsigned)rows_cap) x_perm[(size_t)s_row[k] * row_vecs + c] = v;
     }
   }
 }
@@ -229,7 +233,7 @@ zero_pad_rows_kernel(const int32_t* __restrict__ counts, const int32_t* __restri
 template <typename T>
 __global__ void __launch_bounds__(256)
 combine_kernel(const Vec16* __restrict__ y_perm, const int32_t* __restrict__ prow_of,
-               const float* __restrict__ gate_w, int Tn, int Ke, int row_vecs,
+               const float* __restrict__ gate_w, int Tn, int Ke, int row_vecs, int rows_cap,
                Vec16* __restrict__ y) {
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
@@ -246,6 +250,7 @@ combine_kernel(const Vec16* __restrict__ y_perm, const int32_t* __restrict__ pro
       for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
 #pragma unroll 4
       for (int k = 0; k < Ke; ++k) {
+        if ((unsigned)s_row[k] >= (unsigned)rows_cap) continue;   // invalid slot: contributes nothing
         const Vec16 v = y_perm[(size_t)s_row[k] * row_vecs + c];
         float f[8];
         unpack(v, f, T());
@@ -263,7 +268,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_perm,
                    const int32_t* __restrict__ prow_of, const float* __restrict__ gate_w, int Tn,
-                   int Ke, int row_vecs, Vec16* __restrict__ dy_perm, float* __restrict__ dgate_w) {
+                   int Ke, int row_vecs, int rows_cap, Vec16* __restrict__ dy_perm,
+                   float* __restrict__ dgate_w) {
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_red[MOHGE_MAX_K_EXPERTS][8];
@@ -279,7 +285,8 @@ combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_per
       float part = 0.0f;
       const float g = s_g[k];
       const size_t rbase = (size_t)s_row[k] * row_vecs;
-      for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
+      const bool ok = (unsigned)s_row[k] < (unsigned)rows_cap;
+      for (int c = threadIdx.x; ok && c < row_vecs; c += blockDim.x) {
         const Vec16 dv = dy[(size_t)t * row_vecs + c];
         const Vec16 yv = y_perm[rbase + c];
         float a[8], b[8], o[8];
@@ -333,7 +340,7 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   permute_rows_kernel<<<blocks, block_for(row_vecs), 0, st>>>(
-      (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (Vec16*)x_perm);
+      (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)x_perm);
   MOHGE_LAUNCH_CHECK("permute_rows_kernel");
   if (D.align > 1) {
     zero_pad_rows_kernel<<<dim3(D.Ne, 4), 256, 0, st>>>(counts, aligned, row_vecs, (Vec16*)x_perm);
@@ -350,10 +357,10 @@ int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   if (D.bf16)
     combine_kernel<__nv_bfloat16><<<blocks, block_for(row_vecs), 0, st>>>(
-        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (Vec16*)y);
+        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)y);
   else
     combine_kernel<float><<<blocks, block_for(row_vecs), 0, st>>>(
-        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (Vec16*)y);
+        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)y);
   MOHGE_LAUNCH_CHECK("combine_kernel");
   return MOHGE_OK;
 }
@@ -372,11 +379,11 @@ int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
     const int blocks = T < 148 * 16 ? T : 148 * 16;
     if (D.bf16)
       combine_bwd_kernel<__nv_bfloat16><<<blocks, block_for(row_vecs), 0, st>>>(
-          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs,
+          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
           (Vec16*)dy_perm, dgate_w);
     else
       combine_bwd_kernel<float><<<blocks, block_for(row_vecs), 0, st>>>(
-          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs,
+          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
           (Vec16*)dy_perm, dgate_w);
     MOHGE_LAUNCH_CHECK("combine_bwd_kernel");
   }

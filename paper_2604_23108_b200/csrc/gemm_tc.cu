@@ -1,10 +1,656 @@
-// placeholder until the tcgen05 path lands
+// Ragged grouped GEMMs of the expert layer on the 5th-generation tensor cores (sm_100a):
+// tcgen05.mma kind::f16 (BF16 operands, FP32 accumulators in tensor memory), operands staged in
+// shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), a 4-stage mbarrier pipeline,
+// double-buffered accumulators, and warp-specialised roles:
+//   warp 0      TMA producer (one elected lane)
+//   warp 1      tensor-memory owner and MMA issuer (one elected lane)
+//   warps 2..5  epilogue: tcgen05.ld -> registers -> fused element-wise math -> global memory
+// One persistent CTA per SM walks the device-built, cost-sorted tile list with stride gridDim.x.
+//
+// Six roles share the kernel (C = A . B^T over a contraction index k):
+//   FWD1        [A | U] = Xp . W13^T, fused SwiGLU epilogue writes A, U and H = silu(A) * U.
+//               The gate tile and the up tile of the same hidden columns are two TMA boxes that
+//               land back to back in shared memory, so ONE 128 x (2*BNh) MMA covers both and no
+//               weight repacking is needed.
+//   FWD2        Yp = H . W2^T
+//   DGRAD_DOWN  dH = dYp . W2         (B read MN-major), epilogue turns dH into dA, dU using A, U
+//   DGRAD_13    dXp = [dA | dU] . W13 (B read MN-major)
+//   WGRAD_DOWN  dW2  = dYp^T . H      (A and B read MN-major, contraction over the expert's rows)
+//   WGRAD_13    dW13 = [dA | dU]^T . Xp
+// Expert segments start at multiples of 128 physical rows with zero padding rows, so a 128-row
+// tile never straddles two experts and padding contributes exact zeros to the weight gradients.
+// Hidden widths that are not multiples of the tile are handled by TMA's out-of-bounds zero fill
+// on loads and by column masks on stores.
+//
+// Every wait is bounded: after about one second without progress the waiting thread records
+// (1 << 24 | site) in the status word, raises a CTA-wide abort flag and every role leaves its
+// loop; the CTA then lets copies in flight land, frees its tensor memory and returns.
+
+#include <cuda.h>
+
 #include "common.cuh"
+
 namespace mohge {
-int32_t launch_tc_grouped(const Dims&, int, const GroupPtrs&, const void*, const void*, void*, void*,
-                          const int32_t*, const int32_t*, int, int32_t*, Tile*, int64_t, int32_t*,
-                          cudaStream_t) {
-  set_error("tensor-core path not built");
-  return MOHGE_ERR_UNSUPPORTED;
+namespace {
+
+constexpr int BM = 128;          // UMMA M (rows of an output tile)
+constexpr int BK = 64;           // contraction elements per pipeline stage (128 bytes of BF16)
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;          // 16 KiB
+constexpr int kBBytesMax = 256 * BK * 2;      // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytesMax;
+constexpr int kThreads = 192;
+constexpr int kAccCols = 256;                 // tensor-memory columns per accumulator buffer
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+
+enum Epi { EPI_BF16 = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2, EPI_F32 = 3 };
+
+template <int ROLE> struct RoleTraits;
+template <> struct RoleTraits<ROLE_FWD1>       { static constexpr int A_MN = 0, B_MN = 0, EPI = EPI_SWIGLU_FWD; };
+template <> struct RoleTraits<ROLE_FWD2>       { static constexpr int A_MN = 0, B_MN = 0, EPI = EPI_BF16; };
+template <> struct RoleTraits<ROLE_DGRAD_DOWN> { static constexpr int A_MN = 0, B_MN = 1, EPI = EPI_SWIGLU_BWD; };
+template <> struct RoleTraits<ROLE_DGRAD_13>   { static constexpr int A_MN = 0, B_MN = 1, EPI = EPI_BF16; };
+template <> struct RoleTraits<ROLE_WGRAD_DOWN> { static constexpr int A_MN = 1, B_MN = 1, EPI = EPI_F32; };
+template <> struct RoleTraits<ROLE_WGRAD_13>   { static constexpr int A_MN = 1, B_MN = 1, EPI = EPI_F32; };
+
+struct TcParams {
+  CUtensorMap mapA[MOHGE_MAX_GROUPS];
+  CUtensorMap mapB[MOHGE_MAX_GROUPS];
+  GroupShape gs;
+  GroupPtrs gp;
+  int BN[MOHGE_MAX_GROUPS];      // UMMA N per group (FWD1: gate half + up half)
+  const int32_t* aligned;
+  const int32_t* tile_count;
+  const Tile* tiles;
+  __nv_bfloat16* C;              // FWD1: au, FWD2: y_perm, DGRAD_DOWN: dau, DGRAD_13: dx_perm
+  __nv_bfloat16* C2;             // FWD1: h
+  const __nv_bfloat16* E;        // DGRAD_DOWN: au_saved
+  int accumulate;
+  int32_t* status;
+};
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+constexpr uint64_t kWaitBudgetNs = 1000ull * 1000ull * 1000ull;
+
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status, int site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > kWaitBudgetNs) {
+        atomicCAS(status, 0, (1 << 24) | site);
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the mbarrier once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (128-byte swizzle, descriptor version of sm_100).
+//   K-major  : rows of 64 elements (128 B); 8-row groups 1024 B apart (stride byte offset)
+//   MN-major : blocks of 64 MN-elements x 64 k-rows (one TMA box, 8 KiB, leading byte offset);
+//              inside a block k-rows are 128 B apart and 8-row groups 1024 B apart
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
+         ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+__device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+// 32 consecutive BF16 of one row; only the first `valid` (multiple of 8) columns exist
+__device__ __forceinline__ void store_row32(__nv_bfloat16* p, const float (&v)[32], int valid) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    if (q * 8 < valid) {
+      uint4 o;
+      o.x = pack2(v[q * 8 + 0], v[q * 8 + 1]);
+      o.y = pack2(v[q * 8 + 2], v[q * 8 + 3]);
+      o.z = pack2(v[q * 8 + 4], v[q * 8 + 5]);
+      o.w = pack2(v[q * 8 + 6], v[q * 8 + 7]);
+      *reinterpret_cast<uint4*>(p + q * 8) = o;
+    }
+  }
+}
+__device__ __forceinline__ void load_row32(const __nv_bfloat16* p, float (&v)[32], int valid) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint4 o = make_uint4(0, 0, 0, 0);
+    if (q * 8 < valid) o = *reinterpret_cast<const uint4*>(p + q * 8);
+    v[q * 8 + 0] = bf_lo(o.x); v[q * 8 + 1] = bf_hi(o.x);
+    v[q * 8 + 2] = bf_lo(o.y); v[q * 8 + 3] = bf_hi(o.y);
+    v[q * 8 + 4] = bf_lo(o.z); v[q * 8 + 5] = bf_hi(o.z);
+    v[q * 8 + 6] = bf_lo(o.w); v[q * 8 + 7] = bf_hi(o.w);
+  }
+}
+
+struct TileGeom {
+  int e, g, i, W, bn, m0, n0, num_kb, r0;
+};
+
+template <int ROLE>
+__device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) {
+  TileGeom q;
+  q.e = t.e;
+  q.g = t.e / p.gs.N;
+  q.i = t.e % p.gs.N;
+  q.W = p.gs.W[q.g];
+  q.bn = p.BN[q.g];
+  q.m0 = t.m0;
+  q.n0 = t.n0;
+  q.r0 = 0;
+  if (ROLE == ROLE_FWD1 || ROLE == ROLE_DGRAD_DOWN) q.num_kb = (p.gs.d + BK - 1) / BK;
+  else if (ROLE == ROLE_FWD2) q.num_kb = (q.W + BK - 1) / BK;
+  else if (ROLE == ROLE_DGRAD_13) q.num_kb = (2 * q.W + BK - 1) / BK;
+  else {
+    q.num_kb = t.ext / BK;
+    q.r0 = p.aligned[t.e];
+  }
+  return q;
+}
+
+template <int ROLE>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_grouped_kernel(const __grid_constant__ TcParams p) {
+  using RT = RoleTraits<ROLE>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  // barrier block after the stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * kStageBytes);
+  const uint32_t bar0 = smem_base + kStages * kStageBytes;
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total = *p.tile_count;
+
+  if (warp == 0) {
+    // ================= TMA producer =================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
+        const Tile t = p.tiles[ti];
+        const TileGeom q = tile_geom<ROLE>(p, t);
+        const CUtensorMap* mA = &p.mapA[q.g];
+        const CUtensorMap* mB = &p.mapB[q.g];
+        const uint32_t tx = kABytes + (uint32_t)q.bn * BK * 2;
+        for (int kb = 0; kb < q.num_kb; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { alive = false; break; }
+          const uint32_t sA = smem_base + stage * kStageBytes;
+          const uint32_t sB = sA + kABytes;
+          const uint32_t fb = full_bar(stage);
+          mbar_expect_tx(fb, tx);
+          const int k0 = kb * BK;
+          if (RT::A_MN) {
+            tma_load_2d(sA, mA, fb, q.m0, q.r0 + k0);
+            tma_load_2d(sA + 8192, mA, fb, q.m0 + 64, q.r0 + k0);
+          } else {
+            tma_load_2d(sA, mA, fb, k0, q.m0);
+          }
+          if (ROLE == ROLE_FWD1) {
+            const int half = q.bn >> 1;
+            tma_load_3d(sB, mB, fb, k0, q.n0, 2 * q.i);
+            tma_load_3d(sB + half * 128, mB, fb, k0, q.n0, 2 * q.i + 1);
+          } else if (ROLE == ROLE_FWD2) {
+            tma_load_3d(sB, mB, fb, k0, q.n0, q.i);
+          } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
+            for (int j = 0; j < q.bn / 64; ++j) tma_load_3d(sB + j * 8192, mB, fb, q.n0 + 64 * j, k0, q.i);
+          } else {
+            for (int j = 0; j < q.bn / 64; ++j) tma_load_2d(sB + j * 8192, mB, fb, q.n0 + 64 * j, q.r0 + k0);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int buf = 0;
+      uint32_t acc_phase = 0;
+      bool alive = true;
+      for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
+        const Tile t = p.tiles[ti];
+        const TileGeom q = tile_geom<ROLE>(p, t);
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
+                               ((uint32_t)RT::B_MN << 16) | ((uint32_t)(q.bn >> 3) << 17) |
+                               ((uint32_t)(BM >> 4) << 24);
+        if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag, p.status, 2)) { alive = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * kAccCols;
+        for (int kb = 0; kb < q.num_kb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t sA = smem_base + stage * kStageBytes;
+          const uint32_t sB = sA + kABytes;
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            const uint64_t da = RT::A_MN ? make_desc(sA + kk * 2048, 8192, 1024)
+                                         : make_desc(sA + kk * 32, 16, 1024);
+            const uint64_t db = RT::B_MN ? make_desc(sB + kk * 2048, 8192, 1024)
+                                         : make_desc(sB + kk * 32, 16, 1024);
+            umma_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));     // frees the stage when these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!alive) break;
+        umma_commit(tfull_bar(buf));         // accumulator complete
+        if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ================= epilogue warps =================
+    const int quad = warp & 3;                 // tensor-memory lanes [32*quad, 32*quad + 32)
+    const int row_in_tile = quad * 32 + lane;
+    int buf = 0;
+    uint32_t acc_phase = 0;
+    bool alive = true;
+    for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
+      const Tile t = p.tiles[ti];
+      const TileGeom q = tile_geom<ROLE>(p, t);
+      // the whole warp must agree before the warp-collective tensor-memory loads
+      const bool got = mbar_wait(tfull_bar(buf), acc_phase, abort_flag, p.status, 4);
+      if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kAccCols;
+      const long long d = p.gs.d, pitchAU = 2LL * p.gs.Wmax, pitchH = p.gs.Wmax;
+      if (RT::EPI == EPI_SWIGLU_FWD) {
+        const int half = q.bn >> 1;
+        const long long row = q.m0 + row_in_tile;
+        const bool row_ok = row_in_tile < t.ext;
+        for (int c = 0; c < half; c += 32) {
+          uint32_t ra[32], ru[32];
+          tmem_ld32(taddr + c, ra);
+          tmem_ld32(taddr + half + c, ru);
+          tmem_ld_wait();
+          const int valid = q.W - (q.n0 + c);
+          if (row_ok && valid > 0) {
+            float a[32], u[32], h[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              a[j] = __uint_as_float(ra[j]);
+              u[j] = __uint_as_float(ru[j]);
+              h[j] = a[j] / (1.0f + __expf(-a[j])) * u[j];
+            }
+            __nv_bfloat16* pa = p.C + row * pitchAU + q.n0 + c;
+            store_row32(pa, a, valid);
+            store_row32(pa + q.W, u, valid);
+            store_row32(p.C2 + row * pitchH + q.n0 + c, h, valid);
+          }
+        }
+      } else if (RT::EPI == EPI_BF16) {
+        const long long row = q.m0 + row_in_tile;
+        const bool row_ok = row_in_tile < t.ext;
+        for (int c = 0; c < q.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          const int valid = (int)d - (q.n0 + c);
+          if (row_ok && valid > 0) {
+            float v[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+            store_row32(p.C + row * d + q.n0 + c, v, valid);
+          }
+        }
+      } else if (RT::EPI == EPI_SWIGLU_BWD) {
+        const long long row = q.m0 + row_in_tile;
+        const bool row_ok = row_in_tile < t.ext;
+        for (int c = 0; c < q.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          const int valid = q.W - (q.n0 + c);
+          if (row_ok && valid > 0) {
+            float a[32], u[32], da[32], du[32];
+            const __nv_bfloat16* pe = p.E + row * pitchAU + q.n0 + c;
+            load_row32(pe, a, valid);
+            load_row32(pe + q.W, u, valid);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float dh = __uint_as_float(r[j]);
+              const float sg = 1.0f / (1.0f + __expf(-a[j]));
+              da[j] = dh * u[j] * sg * (1.0f + a[j] * (1.0f - sg));
+              du[j] = dh * a[j] * sg;
+            }
+            __nv_bfloat16* po = p.C + row * pitchAU + q.n0 + c;
+            store_row32(po, da, valid);
+            store_row32(po + q.W, du, valid);
+          }
+        }
+      } else {  // EPI_F32: weight gradients
+        const int Mext = ROLE == ROLE_WGRAD_DOWN ? (int)d : 2 * q.W;
+        const int Next = ROLE == ROLE_WGRAD_DOWN ? q.W : (int)d;
+        float* base = ROLE == ROLE_WGRAD_DOWN ? p.gp.dw2[q.g] + (size_t)q.i * d * q.W
+                                              : p.gp.dw13[q.g] + (size_t)q.i * 2 * q.W * d;
+        const int m = q.m0 + row_in_tile;
+        const bool row_ok = m < Mext;
+        for (int c = 0; c < q.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          const int valid = Next - (q.n0 + c);
+          if (row_ok && valid > 0) {
+            float* po = base + (size_t)m * Next + q.n0 + c;
+#pragma unroll
+            for (int v4 = 0; v4 < 8; ++v4) {
+              if (v4 * 4 < valid) {
+                float4 o = make_float4(__uint_as_float(r[v4 * 4]), __uint_as_float(r[v4 * 4 + 1]),
+                                       __uint_as_float(r[v4 * 4 + 2]), __uint_as_float(r[v4 * 4 + 3]));
+                if (p.accumulate) {
+                  const float4 old = *reinterpret_cast<const float4*>(po + v4 * 4);
+                  o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                }
+                *reinterpret_cast<float4*>(po + v4 * 4) = o;
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---- teardown ----
+  __syncthreads();
+  if (*abort_flag) __nanosleep(200000);    // let copies in flight land before the CTA retires
+  tc_fence_after();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                             CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                             CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode() {
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = (EncodeFn)f;
+  }
+  return fn;
+}
+
+// BF16 tensor of `rank` dims (innermost first); strides in bytes for dims 1..rank-1
+int32_t encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims,
+                   const uint64_t* strides, const uint32_t* box) {
+  EncodeFn fn = get_encode();
+  if (!fn) {
+    set_error("cuTensorMapEncodeTiled is not available from the driver");
+    return MOHGE_ERR_UNSUPPORTED;
+  }
+  cuuint64_t gd[5], gs[5];
+  cuuint32_t bx[5], es[5];
+  for (int i = 0; i < rank; ++i) {
+    gd[i] = dims[i];
+    bx[i] = box[i];
+    es[i] = 1;
+    if (i > 0) gs[i - 1] = strides[i - 1];
+  }
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs,
+                        bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    set_error("cuTensorMapEncodeTiled failed with %d (rank %d, dims %llu x %llu, box %u x %u)", (int)r, rank,
+              (unsigned long long)dims[0], (unsigned long long)dims[1], box[0], box[1]);
+    return MOHGE_ERR_CUDA;
+  }
+  return MOHGE_OK;
+}
+
+// Tile width per group: among the candidates the one that wastes the fewest padded columns
+// (ties go to the wider tile, which keeps the tensor pipe busier per shared-memory byte).
+int pick_bn(int extent, const int* cand, int ncand) {
+  int best = cand[0];
+  long long best_pad = -1;
+  for (int c = 0; c < ncand; ++c) {
+    const long long pad = (long long)((extent + cand[c] - 1) / cand[c]) * cand[c];
+    if (best_pad < 0 || pad < best_pad) {
+      best_pad = pad;
+      best = cand[c];
+    }
+  }
+  return best;
+}
+
+template <int ROLE>
+int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    attr_set = true;
+  }
+  tc_grouped_kernel<ROLE><<<grid, kThreads, kSmemBytes, st>>>(p);
+  MOHGE_LAUNCH_CHECK("tc_grouped_kernel");
+  return MOHGE_OK;
+}
+
+}  // namespace
+
+// Activation operands per role:
+//   FWD1        A = x_perm               C = au_saved, C2 = h_saved
+//   FWD2        A = h_saved              C = y_perm
+//   DGRAD_DOWN  A = dy_perm, B = au_saved (epilogue input)   C = dau
+//   DGRAD_13    A = dau                  C = dx_perm
+//   WGRAD_DOWN  A = dy_perm, B = h_saved     -> dw2
+//   WGRAD_13    A = dau,     B = x_perm      -> dw13
+int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
+                          const void* B, void* C, void* C2, const int32_t* /*counts*/,
+                          const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
+                          int64_t tiles_cap, int32_t* status, cudaStream_t st) {
+  static int sm_count = 0;
+  if (!sm_count) {
+    int dev = 0;
+    MOHGE_CUDA(cudaGetDevice(&dev));
+    cudaDeviceProp prop;
+    MOHGE_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) {
+      set_error("the BF16 path needs an sm_100 device (found sm_%d%d)", prop.major, prop.minor);
+      return MOHGE_ERR_UNSUPPORTED;
+    }
+    sm_count = prop.multiProcessorCount;
+  }
+  TcParams p;
+  memset(&p, 0, sizeof(p));
+  p.gs = make_group_shape(D);
+  p.gp = P;
+  p.aligned = aligned; p.tile_count = tile_count; p.tiles = tiles;
+  p.C = (__nv_bfloat16*)C; p.C2 = (__nv_bfloat16*)C2; p.E = nullptr;
+  p.accumulate = accumulate; p.status = status;
+
+  const uint64_t d = D.d, rows = D.Rcap, pitchAU = 2ull * D.Wmax * 2, pitchH = (uint64_t)D.Wmax * 2;
+  const int cand_n[3] = {256, 192, 128};
+  const int cand_h[3] = {128, 96, 64};
+  int bn_plan[MOHGE_MAX_GROUPS];
+  int32_t rc = MOHGE_OK;
+  for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) { p.BN[g] = 128; bn_plan[g] = 128; }
+  for (int g = 0; g < D.Ng && rc == MOHGE_OK; ++g) {
+    const uint64_t W = D.W[g], N = D.N;
+    uint64_t dims[3], str[2];
+    uint32_t box[3];
+    switch (role) {
+      case ROLE_FWD1: {
+        const int half = pick_bn(D.W[g], cand_h, 3);
+        p.BN[g] = 2 * half; bn_plan[g] = half;
+        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
+        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (rc) break;
+        dims[0] = d; dims[1] = W; dims[2] = 2 * N; str[0] = d * 2; str[1] = W * d * 2;
+        box[0] = BK; box[1] = half; box[2] = 1;
+        rc = encode_map(&p.mapB[g], P.w13[g], 3, dims, str, box);
+      } break;
+      case ROLE_FWD2: {
+        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, 3);
+        dims[0] = W; dims[1] = rows; str[0] = pitchH; box[0] = BK; box[1] = BM;
+        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (rc) break;
+        dims[0] = W; dims[1] = d; dims[2] = N; str[0] = W * 2; str[1] = d * W * 2;
+        box[0] = BK; box[1] = p.BN[g]; box[2] = 1;
+        rc = encode_map(&p.mapB[g], P.w2[g], 3, dims, str, box);
+      } break;
+      case ROLE_DGRAD_DOWN: {
+        p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, 3);
+        p.E = (const __nv_bfloat16*)B;
+        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
+        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (rc) break;
+        dims[0] = W; dims[1] = d; dims[2] = N; str[0] = W * 2; str[1] = d * W * 2;
+        box[0] = 64; box[1] = BK; box[2] = 1;
+        rc = encode_map(&p.mapB[g], P.w2[g], 3, dims, str, box);
+      } break;
+      case ROLE_DGRAD_13: {
+        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, 3);
+        dims[0] = 2 * W; dims[1] = rows; str[0] = pitchAU; box[0] = BK; box[1] = BM;
+        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (rc) break;
+        dims[0] = d; dims[1] = 2 * W; dims[2] = N; str[0] = d * 2; str[1] = 2 * W * d * 2;
+        box[0] = 64; box[1] = BK; box[2] = 1;
+        rc = encode_map(&p.mapB[g], P.w13[g], 3, dims, str, box);
+      } break;
+      case ROLE_WGRAD_DOWN: {
+        p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, 3);
+        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = 64; box[1] = BK;
+        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (rc) break;
+        dims[0] = W; dims[1] = rows; str[0] = pitchH; box[0] = 64; box[1] = BK;
+        rc = encode_map(&p.mapB[g], B, 2, dims, str, box);
+      } break;
+      default: {  // ROLE_WGRAD_13
+        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, 3);
+        dims[0] = 2 * W; dims[1] = rows; str[0] = pitchAU; box[0] = 64; box[1] = BK;
+        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (rc) break;
+        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = 64; box[1] = BK;
+        rc = encode_map(&p.mapB[g], B, 2, dims, str, box);
+      } break;
+    }
+  }
+  if (rc) return rc;
+  rc = launch_build_tiles_plan(make_plan(D, role, BM, bn_plan, role == ROLE_FWD1), aligned, tile_count,
+                               tiles, tiles_cap, status, st);
+  if (rc) return rc;
+  switch (role) {
+    case ROLE_FWD1: return launch_role<ROLE_FWD1>(p, sm_count, st);
+    case ROLE_FWD2: return launch_role<ROLE_FWD2>(p, sm_count, st);
+    case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN>(p, sm_count, st);
+    case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13>(p, sm_count, st);
+    case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN>(p, sm_count, st);
+    default: return launch_role<ROLE_WGRAD_13>(p, sm_count, st);
+  }
+}
+
 }  // namespace mohge
