@@ -1,0 +1,354 @@
+#!/usr/bin/env python
+"""Benchmark of the MoHGE expert layer forward + backward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole hot path over one batch: route (logits GEMM + two-level
+selection), auxiliary statistics, dispatch, grouped SwiGLU experts forward, combine, and the full
+backward (combine, experts dgrad + wgrad, dispatch, router).  The metric is tokens/s of that
+step.  With N > 1 every rank runs an independent replica of the layer (the path does not shard:
+"replicas only"), timed as the maximum over ranks.
+
+`--impl reference` times the fp64 numpy oracle on the host cores on a bounded sample of the
+same workload (there is no reference implementation of this layer to run).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2604_23108_b200.inputs import WORKLOADS, Workload, zipf_logit_bias  # noqa: E402
+
+METRIC = "MoHGE layer fwd+bwd tokens/s"
+UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "cfg5_bf16_large"
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return dict(hbm=d["hbm_gbs"], tf_burst=d["bf16_tflops"], tf_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+def device_inputs(wl: Workload, device, seed=None):
+    """Seeded synthetic tensors drawn on the device (same distributions as inputs.make_inputs)."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(wl.seed if seed is None else seed)
+    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+
+    def normal(shape, std):
+        return (torch.randn(shape, generator=gen, dtype=torch.float32, device=device) * std).to(dt)
+
+    d = wl.d_model
+    inp = dict(x=normal((wl.T, d), 1.0), w_router=normal((wl.n_logits, d), 0.02),
+               dy=normal((wl.T, d), 1.0))
+    inp["w13"] = [normal((wl.experts_per_group, 2 * w, d), 0.02) for w in wl.group_width]
+    inp["w2"] = [normal((wl.experts_per_group, d, w), 0.02) for w in wl.group_width]
+    b = zipf_logit_bias(wl)
+    inp["logit_bias"] = None if b is None else b.to(device)
+    return inp
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "200"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            c = [v.strip() for v in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                smax.append(float(c[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def oracle_sample_run(wl: Workload, sample_tokens: int, steps: int, warmup: int, inp_cpu=None):
+    """Times the oracle (as it stands) on `sample_tokens` tokens of the workload; tokens/s."""
+    import numpy as np
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import oracle as O
+    from _util import oracle_cfg, to_np64
+    from paper_2604_23108_b200.inputs import make_inputs
+    if inp_cpu is None:
+        inp_cpu = make_inputs(wl, T=sample_tokens)
+    ocfg = oracle_cfg(wl)
+    x, w_r, dy = to_np64(inp_cpu["x"][:sample_tokens]), to_np64(inp_cpu["w_router"]), to_np64(inp_cpu["dy"][:sample_tokens])
+    bias = None if inp_cpu.get("logit_bias") is None else to_np64(inp_cpu["logit_bias"])
+    w13, w2 = inp_cpu["w13"], inp_cpu["w2"]       # converted to fp64 expert by expert inside the oracle
+    w13n = [w.to(torch.float32).numpy() for w in w13]
+    w2n = [w.to(torch.float32).numpy() for w in w2]
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        fwd = O.layer_forward(ocfg, x, w_r, w13n, w2n, logit_bias=bias, mode="spec")
+        O.layer_backward(fwd, w13n, w2n, dy, with_aux=True)
+        t1 = time.perf_counter()
+        if it >= warmup:
+            times.append(t1 - t0)
+    per = sum(times) / len(times)
+    return sample_tokens / per, per
+
+
+def run_reference(args, wl: Workload, rank: int):
+    if rank != 0:
+        return
+    sample = min(wl.T, args.ref_sample)
+    cores = torch.get_num_threads()
+    val, per = oracle_sample_run(wl, sample, max(1, args.steps), min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "T": wl.T, "d_model": wl.d_model,
+                   "sample": "first %d tokens, all experts" % sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "oracle fwd+bwd on the first %d tokens of the workload" % sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def flops_per_step(wl: Workload, counts) -> float:
+    """Algorithmic FLOPs of the six expert GEMMs: 18 * d * sum_e M_e * W_g(e) (fwd 6, bwd 12)."""
+    N = wl.experts_per_group
+    tot = 0.0
+    for e, m in enumerate(counts):
+        tot += float(m) * wl.group_width[e // N]
+    return 18.0 * wl.d_model * tot
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-sample", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, wl, rank)
+        return
+
+    from paper_2604_23108_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=dev)
+
+    gcfg = B.Config(d_model=wl.d_model, n_groups=wl.n_groups, experts_per_group=wl.experts_per_group,
+                    k_groups=wl.k_groups, k_experts=wl.k_experts, group_width=list(wl.group_width),
+                    dtype=wl.dtype, row_align=128 if wl.dtype == "bf16" else 1)
+    inp = device_inputs(wl, dev, seed=wl.seed + rank)
+    buf = B.LayerBuffers(gcfg, wl.T, device=dev)
+    T = wl.T
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    gemm_marks = []
+
+    def step(mark=False):
+        B.mohge_route(gcfg, T, inp["x"], inp["w_router"], inp["logit_bias"], None, buf.logits,
+                      buf.group_idx, buf.expert_idx, buf.gate_w, buf.gs, buf.esp, buf.ws)
+        B.mohge_aux_stats(gcfg, T, buf.gs, buf.esp, buf.group_idx, buf.expert_idx, buf.group_count,
+                          buf.group_psum, buf.cnt_routed, buf.cnt_lit, buf.expert_psum, buf.loss, buf.ws)
+        B.mohge_dispatch(gcfg, T, inp["x"], buf.expert_idx, buf.counts, buf.offsets, buf.aligned,
+                         buf.row_of, buf.prow_of, buf.src_of, buf.x_perm, buf.ws)
+        if mark:
+            e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+            e0.record()
+        B.mohge_expert_fwd(gcfg, T, buf.x_perm, buf.counts, buf.aligned, inp["w13"], inp["w2"],
+                           buf.au, buf.h, buf.y_perm, buf.ws)
+        if mark:
+            e1.record()
+        B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, buf.y)
+        B.mohge_combine_bwd(gcfg, T, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.counts,
+                            buf.aligned, buf.dy_perm, buf.dgate)
+        if mark:
+            e2.record()
+        B.mohge_expert_bwd(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts, buf.aligned,
+                           inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13, buf.dw2, 0, buf.ws)
+        if mark:
+            e3.record()
+            gemm_marks.append((e0, e1, e2, e3))
+        B.mohge_dispatch_bwd(gcfg, T, buf.dx_perm, buf.prow_of, buf.dx)
+        cnt_e = buf.cnt_lit if gcfg.fe_mode == 0 else buf.cnt_routed
+        B.mohge_route_bwd(gcfg, T, inp["x"], inp["w_router"], buf.dgate, buf.gs, buf.esp,
+                          buf.group_idx, buf.expert_idx, buf.group_count, cnt_e, buf.dlogits,
+                          buf.dx, buf.dw_router, buf.ws)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    status = B.mohge_get_device_status(buf.ws)
+    if status != 0:
+        raise SystemExit("device status word = 0x%x after warm-up" % status)
+    counts = buf.counts.cpu().tolist()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    l0 = B.mohge_launch_count()
+    barrier()
+    t_start, t_end = ev(), ev()
+    t_start.record()
+    for _ in range(args.steps):
+        step(mark=True)
+    t_end.record()
+    barrier()
+    launches = B.mohge_launch_count() - l0
+    clocks = sampler.stop() if sampler else None
+    ms_total = t_start.elapsed_time(t_end)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * T / (ms_step * 1e-3)
+    gemm_ms = [a.elapsed_time(b) + c.elapsed_time(d_) for a, b, c, d_ in gemm_marks]
+    gemm_ms_step = sum(gemm_ms) / len(gemm_ms)
+
+    # ---- end to end: host (pinned) inputs in, results back to the host, every step ----
+    e2e = None
+    if not args.no_e2e:
+        hx = inp["x"].cpu().pin_memory()
+        hdy = inp["dy"].cpu().pin_memory()
+        hy = torch.empty_like(hx).pin_memory()
+        hdx = torch.empty_like(hx).pin_memory()
+        hloss = torch.empty(4, dtype=torch.float32).pin_memory()
+
+        def e2e_step():
+            inp["x"].copy_(hx, non_blocking=True)
+            inp["dy"].copy_(hdy, non_blocking=True)
+            step()
+            hy.copy_(buf.y, non_blocking=True)
+            hdx.copy_(buf.dx, non_blocking=True)
+            hloss.copy_(buf.loss, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        s0, s1 = ev(), ev()
+        n_e2e = max(2, min(args.steps, 5))
+        s0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        s1.record()
+        barrier()
+        ms = s0.elapsed_time(s1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        es = hx.element_size()
+        e2e = {"value": world * T / (ms / n_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": 2 * hx.numel() * es,
+               "d2h_bytes_per_step": 2 * hx.numel() * es + 16}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    pk = _peaks()
+    flops = flops_per_step(wl, counts)
+    achieved = flops / (gemm_ms_step * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": pk["tf_sustained"], "unit": "TFLOP/s",
+                "frac": achieved / pk["tf_sustained"], "traffic": None,
+                "kernel": "tc_grouped_kernel (6 launches per step: fwd1, fwd2, dgrad x2, wgrad x2)",
+                "of": pk["source"], "flops_per_step": flops, "gemm_ms_per_step": gemm_ms_step,
+                "frac_of_nominal_2250": achieved / 2250.0}
+    if wl.dtype != "bf16":
+        roofline.update(bound="alu", peak=None, frac=None,
+                        kernel="simt_grouped_kernel (FP32 FMA; correctness configuration)")
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        sample = min(wl.T, args.ref_sample)
+        cpu_inp = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in inp.items()
+                   if k not in ("w13", "w2")}
+        cpu_inp["w13"] = [w.cpu() for w in inp["w13"]]
+        cpu_inp["w2"] = [w.cpu() for w in inp["w2"]]
+        val, per = oracle_sample_run(wl, sample, 1, 0, inp_cpu=cpu_inp)
+        cpu_baseline = {"value": val, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                        "sample": "oracle fwd+bwd on the first %d tokens of the workload (%.1f s)" % (sample, per)}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "T": T, "d_model": wl.d_model, "n_groups": wl.n_groups,
+                   "experts_per_group": wl.experts_per_group, "group_width": list(wl.group_width),
+                   "k_groups": wl.k_groups, "k_experts": wl.k_experts,
+                   "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+        "roofline": roofline, "cpu_baseline": cpu_baseline,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -80,6 +80,10 @@ typedef struct mohge_config {
 /* Text of the last error raised on the calling thread ("" if none). HOST. */
 const char* mohge_last_error(void);
 
+/* Diagnostics (no paper counterpart): number of kernels this library has launched so far in
+ * the calling process, counted on the host at launch time. */
+int64_t mohge_launch_count(void);
+
 /* Bytes of workspace needed for T tokens (0 on invalid config). */
 int64_t mohge_workspace_bytes(const mohge_config* cfg, int64_t T);
 

@@ -37,6 +37,7 @@ _lib = None
 
 _P = C.c_void_p
 _SIGS = {
+    "mohge_launch_count": (C.c_int64, []),
     "mohge_workspace_bytes": (C.c_int64, [C.POINTER(mohge_config), C.c_int64]),
     "mohge_perm_rows": (C.c_int64, [C.POINTER(mohge_config), C.c_int64]),
     "mohge_workspace_init": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, _P, _P]),
@@ -136,6 +137,10 @@ class Config:
     @property
     def torch_dtype(self):
         return torch.bfloat16 if self.dtype == "bf16" else torch.float32
+
+
+def mohge_launch_count() -> int:
+    return int(lib().mohge_launch_count())
 
 
 def mohge_workspace_bytes(cfg: Config, T: int) -> int:

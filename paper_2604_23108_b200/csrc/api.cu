@@ -10,6 +10,7 @@
 namespace mohge {
 
 static thread_local char g_err[512] = "";
+unsigned long long g_launches = 0;
 
 void set_error(const char* fmt, ...) {
   va_list ap;
@@ -143,6 +144,8 @@ using namespace mohge;
 extern "C" {
 
 const char* mohge_last_error(void) { return g_err; }
+
+int64_t mohge_launch_count(void) { return (int64_t)g_launches; }
 
 int64_t mohge_workspace_bytes(const mohge_config* cfg, int64_t T) {
   Dims D;

@@ -28,10 +28,13 @@ int32_t cuda_fail(cudaError_t e, const char* what);
     if (e__ != cudaSuccess) return ::mohge::cuda_fail(e__, #call); \
   } while (0)
 
+extern unsigned long long g_launches;   // kernels launched by this library (host-side count)
+
 #define MOHGE_LAUNCH_CHECK(name)                                   \
   do {                                                             \
     cudaError_t e__ = cudaGetLastError();                          \
     if (e__ != cudaSuccess) return ::mohge::cuda_fail(e__, name);  \
+    ++::mohge::g_launches;                                         \
   } while (0)
 
 // ---------------------------------------------------------------- derived sizes
