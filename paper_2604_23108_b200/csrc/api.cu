@@ -76,7 +76,8 @@ WsLayout ws_layout(const Dims& D) {
   L.stats_off = 256;
   L.hist_off = L.stats_off + up256((int64_t)kStatsBlocks * D.NL * 8);
   L.base_off = L.hist_off + up256((int64_t)(L.chunks + 1) * D.Ne * 4);
-  L.tiles_off = L.base_off + up256((int64_t)(L.chunks + 1) * D.Ne * 4);
+  L.dl16_off = L.base_off + up256((int64_t)(L.chunks + 1) * D.Ne * 4);
+  L.tiles_off = L.dl16_off + up256((D.T + 1) * (int64_t)((D.NL + 7) / 8 * 8) * 2);
   // tile capacity: the smallest tile either path uses is 64 x 64
   const int64_t mt = D.Rcap / 64 + D.Ne + 1;
   const int64_t wide = (D.d > 2 * D.Wmax ? D.d : 2 * D.Wmax);
@@ -92,6 +93,7 @@ struct Ws {
   double* stats;
   int32_t* hist;
   int32_t* base;
+  __nv_bfloat16* dl16;
   int32_t* tile_count;
   Tile* tiles;
   int64_t tiles_cap;
@@ -105,6 +107,7 @@ static Ws carve(const Dims& D, void* ws) {
   w.stats = (double*)(p + L.stats_off);
   w.hist = (int32_t*)(p + L.hist_off);
   w.base = (int32_t*)(p + L.base_off);
+  w.dl16 = (__nv_bfloat16*)(p + L.dl16_off);
   w.tile_count = (int32_t*)(p + L.tiles_off);
   w.tiles = (Tile*)(p + L.tiles_off + 256);
   w.tiles_cap = L.tiles_cap;
@@ -189,8 +192,11 @@ int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const voi
   if (!logits_in) {
     REQ_PTR(x); REQ_PTR(w_router); REQ_PTR(logits_out); OPT_PTR(logit_bias);
     const int f32 = D.bf16 ? 0 : 1;
-    rc = launch_simt_plain((int)T, D.NL, D.d, x, f32, D.d, 1, w_router, f32, D.d, 1, logits_out, 1,
-                           D.NL, logit_bias, 0, st);
+    if (D.bf16 && !force_simt())
+      rc = launch_tc_plain(D, ROLE_LOGITS, x, w_router, 0, logits_out, logit_bias, carve(D, ws).status, st);
+    else
+      rc = launch_simt_plain((int)T, D.NL, D.d, x, f32, D.d, 1, w_router, f32, D.d, 1, logits_out, 1,
+                             D.NL, logit_bias, 0, st);
     if (rc) return rc;
     logits = logits_out;
   } else {
@@ -374,13 +380,23 @@ int32_t mohge_route_bwd(const mohge_config* cfg, int64_t T, const void* x, const
   MOHGE_CHECK_ARG((group_count == nullptr) == (expert_count == nullptr),
                   "group_count and expert_count must both be given or both be NULL");
   cudaStream_t st = (cudaStream_t)stream;
+  const bool tc = D.bf16 && !force_simt();
+  const Ws w = carve(D, ws);
+  const int pitch16 = (D.NL + 7) / 8 * 8;
   rc = launch_router_bwd_elementwise(D, *cfg, dgate_w, nullptr, gs_saved, esp_saved, group_idx,
-                                     expert_idx, group_count, expert_count, dlogits, st);
+                                     expert_idx, group_count, expert_count, dlogits,
+                                     tc ? w.dl16 : nullptr, pitch16, st);
   if (rc) return rc;
   const int f32 = D.bf16 ? 0 : 1;
   if (T == 0) {
     MOHGE_CUDA(cudaMemsetAsync(dw_router, 0, sizeof(float) * D.NL * D.d, st));
     return MOHGE_OK;
+  }
+  if (tc) {
+    // BF16 copy of dlogits feeds both router-backward GEMMs on the tensor cores
+    rc = launch_tc_plain(D, ROLE_ROUTER_DW, x, w.dl16, pitch16, dw_router, nullptr, w.status, st);
+    if (rc) return rc;
+    return launch_tc_plain(D, ROLE_ROUTER_DX, w.dl16, w_router, pitch16, dx, nullptr, w.status, st);
   }
   // dw_router[NL, d] = dlogits^T . x
   rc = launch_simt_plain(D.NL, D.d, (int)T, dlogits, 1, 1, D.NL, x, f32, 1, D.d, dw_router, 1, D.d,

@@ -53,12 +53,13 @@ static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b)
 // [0, 256)            device status word (int32) and padding
 // stats partials      double [kStatsBlocks][NL]
 // dispatch histogram  int32 [chunks][Ne] (per-chunk counts) and the same size of chunk bases
+// dlogits (BF16)      [T][NLp], NLp = NL rounded up to 8 (operand of the router-backward GEMMs)
 // tile list           int32 count (+pad to 16 B) followed by int4 entries
 constexpr int kStatsBlocks = 296;
 constexpr int kDispatchChunk = 256;  // tokens per dispatch block
 
 struct WsLayout {
-  int64_t status_off, stats_off, hist_off, base_off, tiles_off, total;
+  int64_t status_off, stats_off, hist_off, base_off, dl16_off, tiles_off, total;
   int64_t tiles_cap;
   int chunks;
 };
@@ -88,6 +89,9 @@ enum GemmRole {
   ROLE_DGRAD_13 = 3,    // dXp[rows, d]   = dAU[rows, 2W]  . W13
   ROLE_WGRAD_DOWN = 4,  // dW2[d, W]      = dYp^T . H      (contraction over the expert's rows)
   ROLE_WGRAD_13 = 5,    // dW13[2W, d]    = dAU^T . Xp
+  ROLE_LOGITS = 6,      // logits[T, NL]  = x . W_r^T            (router, single problem)
+  ROLE_ROUTER_DW = 7,   // dW_r[NL, d]    = dlogits^T . x
+  ROLE_ROUTER_DX = 8,   // dx[T, d]      += dlogits . W_r
 };
 
 // Parameters of the device-side tile scheduler (build_tiles_kernel).
@@ -116,7 +120,8 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
                                       const float* gate_unused, const float* gs, const float* esp,
                                       const int32_t* group_idx, const int32_t* expert_idx,
                                       const int32_t* group_count, const int32_t* expert_count,
-                                      float* dlogits, cudaStream_t st);
+                                      float* dlogits, __nv_bfloat16* dl16, int dl16_pitch,
+                                      cudaStream_t st);
 
 // dispatch.cu
 int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx, int32_t* counts,
@@ -154,5 +159,8 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
                           const void* B, void* C, void* C2, const int32_t* counts,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
                           int64_t tiles_cap, int32_t* status, cudaStream_t st);
+
+int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
+                        void* C, const float* bias, int32_t* status, cudaStream_t st);
 
 }  // namespace mohge

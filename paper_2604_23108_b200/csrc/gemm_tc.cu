@@ -43,7 +43,7 @@ constexpr int kThreads = 192;
 constexpr int kAccCols = 256;                 // tensor-memory columns per accumulator buffer
 constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
 
-enum Epi { EPI_BF16 = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2, EPI_F32 = 3 };
+enum Epi { EPI_BF16 = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2, EPI_F32 = 3, EPI_LOGITS = 4, EPI_F32_T = 5, EPI_BF16_ACC = 6 };
 
 template <int ROLE> struct RoleTraits;
 template <> struct RoleTraits<ROLE_FWD1>       { static constexpr int A_MN = 0, B_MN = 0, EPI = EPI_SWIGLU_FWD; };
@@ -52,6 +52,11 @@ template <> struct RoleTraits<ROLE_DGRAD_DOWN> { static constexpr int A_MN = 0, 
 template <> struct RoleTraits<ROLE_DGRAD_13>   { static constexpr int A_MN = 0, B_MN = 1, EPI = EPI_BF16; };
 template <> struct RoleTraits<ROLE_WGRAD_DOWN> { static constexpr int A_MN = 1, B_MN = 1, EPI = EPI_F32; };
 template <> struct RoleTraits<ROLE_WGRAD_13>   { static constexpr int A_MN = 1, B_MN = 1, EPI = EPI_F32; };
+// single-problem ("plain") GEMMs of the router: tiles are decoded from the tile index
+template <> struct RoleTraits<ROLE_LOGITS>     { static constexpr int A_MN = 0, B_MN = 0, EPI = EPI_LOGITS; };
+template <> struct RoleTraits<ROLE_ROUTER_DW>  { static constexpr int A_MN = 1, B_MN = 1, EPI = EPI_F32_T; };
+template <> struct RoleTraits<ROLE_ROUTER_DX>  { static constexpr int A_MN = 0, B_MN = 1, EPI = EPI_BF16_ACC; };
+template <int ROLE> __host__ __device__ constexpr bool is_plain() { return ROLE >= ROLE_LOGITS; }
 
 struct TcParams {
   CUtensorMap mapA[MOHGE_MAX_GROUPS];
@@ -67,6 +72,10 @@ struct TcParams {
   const __nv_bfloat16* E;        // DGRAD_DOWN: au_saved
   int accumulate;
   int32_t* status;
+  // plain roles: C[M, N] over contraction K; tile ti -> (ti / ntn, ti % ntn)
+  int plain_total, plain_ntn, plain_M, plain_N, plain_K;
+  float* Cf;                     // LOGITS: logits [T, NL]; ROUTER_DW: dw_router [NL, d]
+  const float* bias;             // LOGITS: optional logit bias [NL]
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -203,8 +212,26 @@ struct TileGeom {
 };
 
 template <int ROLE>
+__device__ __forceinline__ Tile fetch_tile(const TcParams& p, int ti) {
+  if (is_plain<ROLE>()) {
+    Tile t;
+    t.e = 0;
+    t.m0 = (ti / p.plain_ntn) * BM;
+    t.n0 = (ti % p.plain_ntn) * p.BN[0];
+    t.ext = p.plain_M - t.m0 < BM ? p.plain_M - t.m0 : BM;
+    return t;
+  }
+  return p.tiles[ti];
+}
+
+template <int ROLE>
 __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) {
   TileGeom q;
+  if (is_plain<ROLE>()) {
+    q.e = 0; q.g = 0; q.i = 0; q.W = 0; q.bn = p.BN[0]; q.m0 = t.m0; q.n0 = t.n0; q.r0 = 0;
+    q.num_kb = (p.plain_K + BK - 1) / BK;
+    return q;
+  }
   q.e = t.e;
   q.g = t.e / p.gs.N;
   q.i = t.e % p.gs.N;
@@ -262,7 +289,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total = *p.tile_count;
+  const int total = is_plain<ROLE>() ? p.plain_total : *p.tile_count;
 
   if (warp == 0) {
     // ================= TMA producer =================
@@ -271,7 +298,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       uint32_t phase = 0;
       bool alive = true;
       for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
-        const Tile t = p.tiles[ti];
+        const Tile t = fetch_tile<ROLE>(p, ti);
         const TileGeom q = tile_geom<ROLE>(p, t);
         const CUtensorMap* mA = &p.mapA[q.g];
         const CUtensorMap* mB = &p.mapB[q.g];
@@ -293,6 +320,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             const int half = q.bn >> 1;
             tma_load_3d(sB, mB, fb, k0, q.n0, 2 * q.i);
             tma_load_3d(sB + half * 128, mB, fb, k0, q.n0, 2 * q.i + 1);
+          } else if (ROLE == ROLE_LOGITS) {
+            tma_load_2d(sB, mB, fb, k0, q.n0);
           } else if (ROLE == ROLE_FWD2) {
             tma_load_3d(sB, mB, fb, k0, q.n0, q.i);
           } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
@@ -313,7 +342,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       uint32_t acc_phase = 0;
       bool alive = true;
       for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
-        const Tile t = p.tiles[ti];
+        const Tile t = fetch_tile<ROLE>(p, ti);
         const TileGeom q = tile_geom<ROLE>(p, t);
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
                                ((uint32_t)RT::B_MN << 16) | ((uint32_t)(q.bn >> 3) << 17) |
@@ -350,7 +379,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     uint32_t acc_phase = 0;
     bool alive = true;
     for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
-      const Tile t = p.tiles[ti];
+      const Tile t = fetch_tile<ROLE>(p, ti);
       const TileGeom q = tile_geom<ROLE>(p, t);
       // the whole warp must agree before the warp-collective tensor-memory loads
       const bool got = mbar_wait(tfull_bar(buf), acc_phase, abort_flag, p.status, 4);
@@ -420,6 +449,56 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             __nv_bfloat16* po = p.C + row * pitchAU + q.n0 + c;
             store_row32(po, da, valid);
             store_row32(po + q.W, du, valid);
+          }
+        }
+      } else if (RT::EPI == EPI_LOGITS) {
+        // logits[t, n] = acc + bias[n]; NL is arbitrary, so stores are scalar and masked
+        const long long row = q.m0 + row_in_tile;
+        const bool row_ok = row_in_tile < t.ext;
+        for (int c = 0; c < q.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          if (row_ok) {
+            float* po = p.Cf + row * p.plain_N;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int n = q.n0 + c + j;
+              if (n < p.plain_N) po[n] = __uint_as_float(r[j]) + (p.bias ? p.bias[n] : 0.0f);
+            }
+          }
+        }
+      } else if (RT::EPI == EPI_F32_T) {
+        // transposed store: tile rows are the d index, tile columns the router output index
+        const int m = q.m0 + row_in_tile;
+        const bool row_ok = m < p.plain_M;
+        for (int c = 0; c < q.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int n = q.n0 + c + j;
+              if (n < p.plain_N) p.Cf[(size_t)n * p.plain_M + m] = __uint_as_float(r[j]);
+            }
+          }
+        }
+      } else if (RT::EPI == EPI_BF16_ACC) {
+        const long long row = q.m0 + row_in_tile;
+        const bool row_ok = row_in_tile < t.ext;
+        for (int c = 0; c < q.bn; c += 32) {
+          uint32_t r[32];
+          tmem_ld32(taddr + c, r);
+          tmem_ld_wait();
+          const int valid = p.plain_N - (q.n0 + c);
+          if (row_ok && valid > 0) {
+            float v[32];
+            __nv_bfloat16* po = p.C + row * p.plain_N + q.n0 + c;
+            load_row32(po, v, valid);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
+            store_row32(po, v, valid);
           }
         }
       } else {  // EPI_F32: weight gradients
@@ -540,6 +619,63 @@ int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
 }
 
 }  // namespace
+
+// Router GEMMs on the tensor cores (BF16 layer dtype).
+//   LOGITS     logits[T, NL]  = x . W_r^T + bias                 A = x,          B = w_router
+//   ROUTER_DW  dw_router^T[d, NL] = x^T . dl16  (stored transposed)  A = x,       B = dl16 [T, NLp]
+//   ROUTER_DX  dx[T, d]      += dl16 . W_r                       A = dl16,       B = w_router
+int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
+                        void* C, const float* bias, int32_t* status, cudaStream_t st) {
+  static int sm_count = 0;
+  if (!sm_count) {
+    int dev = 0;
+    MOHGE_CUDA(cudaGetDevice(&dev));
+    MOHGE_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+  }
+  if (D.T == 0) return MOHGE_OK;
+  TcParams p;
+  memset(&p, 0, sizeof(p));
+  p.gs = make_group_shape(D);
+  p.status = status;
+  p.bias = bias;
+  const uint64_t d = D.d, T = D.T, NL = D.NL;
+  uint64_t dims[2], str[1];
+  uint32_t box[2];
+  int32_t rc;
+  if (role == ROLE_LOGITS) {
+    p.plain_M = (int)T; p.plain_N = D.NL; p.plain_K = D.d;
+    p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 15) / 16 * 16;
+    p.Cf = (float*)C;
+    dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = BK; box[1] = BM;
+    if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
+    dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = BK; box[1] = p.BN[0];
+    if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+  } else if (role == ROLE_ROUTER_DW) {
+    p.plain_M = D.d; p.plain_N = D.NL; p.plain_K = (int)T;
+    p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 63) / 64 * 64;
+    p.Cf = (float*)C;
+    dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = 64; box[1] = BK;
+    if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
+    dims[0] = NL; dims[1] = T; str[0] = (uint64_t)b_pitch_elems * 2; box[0] = 64; box[1] = BK;
+    if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+  } else {  // ROLE_ROUTER_DX
+    p.plain_M = (int)T; p.plain_N = D.d; p.plain_K = D.NL;
+    p.BN[0] = D.d >= 256 ? 256 : (D.d + 63) / 64 * 64;
+    p.C = (__nv_bfloat16*)C;
+    dims[0] = NL; dims[1] = T; str[0] = (uint64_t)b_pitch_elems * 2; box[0] = BK; box[1] = BM;
+    if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
+    dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = 64; box[1] = BK;
+    if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+  }
+  p.plain_ntn = (p.plain_N + p.BN[0] - 1) / p.BN[0];
+  p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn;
+  const int grid = p.plain_total < sm_count ? p.plain_total : sm_count;
+  switch (role) {
+    case ROLE_LOGITS: return launch_role<ROLE_LOGITS>(p, grid, st);
+    case ROLE_ROUTER_DW: return launch_role<ROLE_ROUTER_DW>(p, grid, st);
+    default: return launch_role<ROLE_ROUTER_DX>(p, grid, st);
+  }
+}
 
 // Activation operands per role:
 //   FWD1        A = x_perm               C = au_saved, C2 = h_saved

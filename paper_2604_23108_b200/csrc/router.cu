@@ -300,7 +300,7 @@ router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
                   const float* __restrict__ gs, const float* __restrict__ esp,
                   const int32_t* __restrict__ group_idx, const int32_t* __restrict__ expert_idx,
                   const int32_t* __restrict__ group_count, const int32_t* __restrict__ expert_count,
-                  float* __restrict__ dlogits) {
+                  float* __restrict__ dlogits, __nv_bfloat16* __restrict__ dl16, int dl16_pitch) {
   __shared__ float s_dkey[kBwdWarps][256];
   __shared__ float s_dgs[kBwdWarps][MOHGE_MAX_GROUPS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -358,7 +358,11 @@ router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
         inner += __shfl_xor_sync(kFull, inner, mask);
         dgs += __shfl_xor_sync(kFull, dgs, mask);
       }
-      if (valid) dlogits[(size_t)t * s.NL + s.Ng + e] = ev * (desp - inner);
+      if (valid) {
+        const float dl = ev * (desp - inner);
+        dlogits[(size_t)t * s.NL + s.Ng + e] = dl;
+        if (dl16) dl16[(size_t)t * dl16_pitch + s.Ng + e] = __float2bfloat16(dl);
+      }
       if (valid && i == 0) s_dgs[warp][g] = dgs;
     }
     __syncwarp();
@@ -377,7 +381,11 @@ router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
       }
       dG += bp.alpha_g * invT * (cg / Ss - cs / (Ss * Ss));
     }
-    if (lane < s.Ng) dlogits[(size_t)t * s.NL + lane] = dG * gv * (1.0f - gv);
+    if (lane < s.Ng) {
+      const float dl = dG * gv * (1.0f - gv);
+      dlogits[(size_t)t * s.NL + lane] = dl;
+      if (dl16) dl16[(size_t)t * dl16_pitch + lane] = __float2bfloat16(dl);
+    }
     __syncwarp();
   }
 }
@@ -453,7 +461,8 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
                                       const float*, const float* gs, const float* esp,
                                       const int32_t* group_idx, const int32_t* expert_idx,
                                       const int32_t* group_count, const int32_t* expert_count,
-                                      float* dlogits, cudaStream_t st) {
+                                      float* dlogits, __nv_bfloat16* dl16, int dl16_pitch,
+                                      cudaStream_t st) {
   if (D.T == 0) return MOHGE_OK;
   const RouterShape s = make_shape(D);
   BwdParams bp;
@@ -467,7 +476,7 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
   MOHGE_DISPATCH_J(slots_per_lane(D),
                    (router_bwd_kernel<JJ><<<blocks, kBwdWarps * 32, 0, st>>>(
                        s, bp, dgate, gs, esp, group_idx, expert_idx, group_count, expert_count,
-                       dlogits)));
+                       dlogits, dl16, dl16_pitch)));
   MOHGE_LAUNCH_CHECK("router_bwd_kernel");
   return MOHGE_OK;
 }
