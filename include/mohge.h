@@ -141,6 +141,29 @@ int32_t mohge_aux_stats(const mohge_config* cfg, int64_t T, const float* gs_save
                         float* expert_psum, float* loss_out, void* ws, void* stream);
 
 /*
+ * Allocation-free variant of mohge_aux_stats.  The paper has no counterpart: this entry point
+ * exists for callers that cannot allocate device memory at the point of the call (all memory
+ * already owned by a framework's pool, or a loop that must not run into cudaMalloc's device-wide
+ * synchronisation) and therefore cannot provide a workspace.  Same inputs, outputs and results as
+ * mohge_aux_stats, but the per-block partial sums are kept in an array built into the library
+ * image (296 x MOHGE_STATIC_MAX_LOGITS doubles, about 315 KiB, resident on every GPU that loads
+ * the library until the process exits).  It calls no allocator.
+ *   - Limit: N_g + N_e <= MOHGE_STATIC_MAX_LOGITS; larger configs are refused with
+ *     MOHGE_ERR_INVALID_ARG and nothing is launched.
+ *   - The first call on a device looks up the array's device address (one-time set-up, done with
+ *     that device current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps the previous call's contents.
+ *     Nothing has to start at zero (each call rewrites every entry it reads), but calls that
+ *     overlap on the GPU (different streams without ordering) race on it: order them.
+ */
+#define MOHGE_STATIC_MAX_LOGITS 136
+int32_t mohge_aux_stats_static(const mohge_config* cfg, int64_t T, const float* gs_saved,
+                               const float* esp_saved, const int32_t* group_idx,
+                               const int32_t* expert_idx, int32_t* group_count, float* group_psum,
+                               int32_t* expert_count_routed, int32_t* expert_count_lit,
+                               float* expert_psum, float* loss_out, void* stream);
+
+/*
  * Token permutation.  Not a paper equation: the stable counting sort by (expert, token) that
  * grouped execution of Eq. 15's sum needs.  Integer outputs are deterministic and bit-exact.
  *   counts [N_e], offsets [N_e+1] (exclusive prefix sum), aligned_offsets [N_e+1],

@@ -44,6 +44,7 @@ _SIGS = {
     "mohge_get_device_status": (C.c_int32, [_P, C.POINTER(C.c_int32), _P]),
     "mohge_route": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12),
     "mohge_aux_stats": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12),
+    "mohge_aux_stats_static": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 11),
     "mohge_dispatch": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 11),
     "mohge_expert_fwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 10),
     "mohge_combine": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 5),
@@ -182,6 +183,16 @@ def mohge_aux_stats(cfg, T, gs_saved, esp_saved, group_idx, expert_idx, group_co
                                  _ptr(group_psum), _ptr(expert_count_routed),
                                  _ptr(expert_count_lit), _ptr(expert_psum), _ptr(loss_out),
                                  _ptr(ws), _stream()), "mohge_aux_stats")
+
+
+def mohge_aux_stats_static(cfg, T, gs_saved, esp_saved, group_idx, expert_idx, group_count,
+                           group_psum, expert_count_routed, expert_count_lit, expert_psum, loss_out):
+    """mohge_aux_stats without a workspace: for callers that cannot allocate one (see mohge.h)."""
+    _check(lib().mohge_aux_stats_static(C.byref(cfg.c()), T, _ptr(gs_saved), _ptr(esp_saved),
+                                        _ptr(group_idx), _ptr(expert_idx), _ptr(group_count),
+                                        _ptr(group_psum), _ptr(expert_count_routed),
+                                        _ptr(expert_count_lit), _ptr(expert_psum), _ptr(loss_out),
+                                        _stream()), "mohge_aux_stats_static")
 
 
 def mohge_dispatch(cfg, T, x, expert_idx, counts, offsets, aligned_offsets, row_of, prow_of,

@@ -482,3 +482,54 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
 }
 
 }  // namespace mohge
+
+// ---------------------------------------------------------------- allocation-free statistics
+//
+// mohge_aux_stats_static is mohge_aux_stats for callers that cannot hand over a workspace
+// because they cannot allocate one at that point: code that runs after an inference server or a
+// training framework has claimed all device memory for its own pool, or inside a latency-critical
+// loop where cudaMalloc's implicit device-wide synchronisation is unacceptable.  The per-block
+// partial sums live in the file-scope device array below instead.  Consequences, all documented
+// in the header: the array (kStatsBlocks x MOHGE_STATIC_MAX_LOGITS doubles, about 315 KiB) is
+// part of the library image on every GPU that loads it until the process exits; all calls on one
+// device share it, so two calls that overlap on the GPU race; nothing in it needs to start at
+// zero because every partial row that the final reduction reads is rewritten by the same call.
+namespace mohge {
+namespace {
+static __device__ __align__(256) double g_static_partials[kStatsBlocks * MOHGE_STATIC_MAX_LOGITS];
+constexpr int kMaxDevices = 64;
+double* g_static_ptr[kMaxDevices] = {nullptr};
+}  // namespace
+}  // namespace mohge
+
+extern "C" int32_t mohge_aux_stats_static(const mohge_config* cfg, int64_t T, const float* gs_saved,
+                                          const float* esp_saved, const int32_t* group_idx,
+                                          const int32_t* expert_idx, int32_t* group_count,
+                                          float* group_psum, int32_t* expert_count_routed,
+                                          int32_t* expert_count_lit, float* expert_psum,
+                                          float* loss_out, void* stream) {
+  using namespace mohge;
+  Dims D;
+  const int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  MOHGE_CHECK_ARG(gs_saved && esp_saved && group_idx && expert_idx && group_count && group_psum &&
+                      expert_count_routed && expert_count_lit && expert_psum && loss_out,
+                  "mohge_aux_stats_static: every pointer argument must be non-NULL");
+  MOHGE_CHECK_ARG(D.NL <= MOHGE_STATIC_MAX_LOGITS,
+                  "mohge_aux_stats_static: N_g + N_e = %d router outputs exceed the %d that the built-in "
+                  "scratch array holds; use mohge_aux_stats with a caller workspace instead",
+                  D.NL, MOHGE_STATIC_MAX_LOGITS);
+  int dev = 0;
+  MOHGE_CUDA(cudaGetDevice(&dev));
+  MOHGE_CHECK_ARG(dev >= 0 && dev < kMaxDevices, "device ordinal %d not supported", dev);
+  if (g_static_ptr[dev] == nullptr) {
+    // The symbol's name is only a host-side handle; the kernel needs the device address, which
+    // is looked up once per device with that device current.
+    double* p = nullptr;
+    MOHGE_CUDA(cudaGetSymbolAddress((void**)&p, g_static_partials));
+    g_static_ptr[dev] = p;
+  }
+  return launch_aux_stats(D, *cfg, gs_saved, esp_saved, group_idx, expert_idx, group_count,
+                          group_psum, expert_count_routed, expert_count_lit, expert_psum, loss_out,
+                          g_static_ptr[dev], (cudaStream_t)stream);
+}
