@@ -90,7 +90,7 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, smax, reasons = [], [], set()
+        sm, smax, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             c = [v.strip() for v in line.split(",")]
@@ -99,6 +99,7 @@ class ClockSampler:
             try:
                 sm.append(float(c[1]))
                 smax.append(float(c[2]))
+                pw.append(float(c[3]))
             except ValueError:
                 continue
             for n, v in zip(names, c[5:9]):
@@ -107,7 +108,8 @@ class ClockSampler:
         self.f.close()
         os.unlink(self.f.name)
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm),
+                       power_w=statistics.median(pw))
         out["reasons"] = sorted(reasons)
         return out
 

@@ -35,13 +35,20 @@ namespace {
 
 constexpr int BM = 128;          // UMMA M (rows of an output tile)
 constexpr int BK = 64;           // contraction elements per pipeline stage (128 bytes of BF16)
-constexpr int kStages = 4;
-constexpr int kABytes = BM * BK * 2;          // 16 KiB
-constexpr int kBBytesMax = 256 * BK * 2;      // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytesMax;
+constexpr int kABytes = BM * BK * 2;          // 16 KiB: 128 rows of A per CTA and stage
 constexpr int kThreads = 192;
 constexpr int kAccCols = 256;                 // tensor-memory columns per accumulator buffer
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+
+// CG = CTAs per MMA (tcgen05 cta_group).  CG = 2 pairs the two CTAs of a cluster on one
+// 256 x N tile: each CTA stages its own 128 rows of A and HALF of B, so operand traffic per FLOP
+// drops by a third and the smaller stages allow a six-deep pipeline.
+template <int CG> struct Geo {
+  static constexpr int kStages = CG == 1 ? 4 : 6;
+  static constexpr int kBBytes = 256 / CG * BK * 2;          // 32 KiB or 16 KiB
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+  static constexpr int kTileM = BM * CG;
+};
 
 enum Epi { EPI_BF16 = 0, EPI_SWIGLU_FWD = 1, EPI_SWIGLU_BWD = 2, EPI_F32 = 3, EPI_LOGITS = 4, EPI_F32_T = 5, EPI_BF16_ACC = 6 };
 
@@ -136,6 +143,59 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// ---- CTA-pair (cluster of 2) helpers
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar_cluster, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(bar_cluster), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+// loads of the pair signal the barrier of the leader CTA (cluster address)
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+template <int CG>
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  if (CG == 2) tma2_load_2d(dst, map, bar, c0, c1); else tma_load_2d(dst, map, bar, c0, c1);
+}
+template <int CG>
+__device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+  if (CG == 2) tma2_load_3d(dst, map, bar, c0, c1, c2); else tma_load_3d(dst, map, bar, c0, c1, c2);
+}
+__device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives on the same barrier offset in both CTAs of the pair
+__device__ __forceinline__ void umma2_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -250,10 +310,14 @@ __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) 
   return q;
 }
 
-template <int ROLE>
+template <int ROLE, int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_grouped_kernel(const __grid_constant__ TcParams p) {
   using RT = RoleTraits<ROLE>;
+  constexpr int kStages = Geo<CG>::kStages;
+  constexpr int kStageBytes = Geo<CG>::kStageBytes;
+  const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;   // position in the CTA pair
+  const int unit = blockIdx.x / CG, unit_stride = gridDim.x / CG;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -271,22 +335,28 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(full_bar(s), 1);
+      mbar_init(full_bar(s), CG);       // one arrive.expect_tx per CTA of the pair
       mbar_init(empty_bar(s), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 4);
+      mbar_init(tempty_bar(b), 4 * CG);  // four epilogue warps per CTA
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CG == 2) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (CG == 2) cluster_sync_all();     // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int total = is_plain<ROLE>() ? p.plain_total : *p.tile_count;
@@ -297,37 +367,45 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
+      for (int ti = unit; ti < total && alive; ti += unit_stride) {
         const Tile t = fetch_tile<ROLE>(p, ti);
         const TileGeom q = tile_geom<ROLE>(p, t);
         const CUtensorMap* mA = &p.mapA[q.g];
         const CUtensorMap* mB = &p.mapB[q.g];
-        const uint32_t tx = kABytes + (uint32_t)q.bn * BK * 2;
+        const int nb = q.bn / CG;                          // B rows staged by this CTA
+        const uint32_t tx = kABytes + (uint32_t)nb * BK * 2;
+        const int am0 = q.m0 + BM * (int)cta_rank;         // this CTA's 128 rows of the tile
+        const int bn0 = q.n0 + nb * (int)cta_rank;         // this CTA's slice of the tile columns
         for (int kb = 0; kb < q.num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { alive = false; break; }
           const uint32_t sA = smem_base + stage * kStageBytes;
           const uint32_t sB = sA + kABytes;
-          const uint32_t fb = full_bar(stage);
-          mbar_expect_tx(fb, tx);
+          // CG == 2: both CTAs report to the full barrier of the pair's leader (rank 0)
+          const uint32_t fb = CG == 2 ? mapa_rank(full_bar(stage), 0) : full_bar(stage);
+          if (CG == 2) mbar_expect_tx_cluster(fb, tx); else mbar_expect_tx(fb, tx);
           const int k0 = kb * BK;
           if (RT::A_MN) {
-            tma_load_2d(sA, mA, fb, q.m0, q.r0 + k0);
-            tma_load_2d(sA + 8192, mA, fb, q.m0 + 64, q.r0 + k0);
+            tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0);
+            tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0);
           } else {
-            tma_load_2d(sA, mA, fb, k0, q.m0);
+            tma_2d<CG>(sA, mA, fb, k0, am0);
           }
           if (ROLE == ROLE_FWD1) {
             const int half = q.bn >> 1;
-            tma_load_3d(sB, mB, fb, k0, q.n0, 2 * q.i);
-            tma_load_3d(sB + half * 128, mB, fb, k0, q.n0, 2 * q.i + 1);
+            if (CG == 2) {          // leader stages the gate rows, its peer the up rows
+              tma_3d<CG>(sB, mB, fb, k0, q.n0, 2 * q.i + (int)cta_rank);
+            } else {
+              tma_3d<CG>(sB, mB, fb, k0, q.n0, 2 * q.i);
+              tma_3d<CG>(sB + half * 128, mB, fb, k0, q.n0, 2 * q.i + 1);
+            }
           } else if (ROLE == ROLE_LOGITS) {
-            tma_load_2d(sB, mB, fb, k0, q.n0);
+            tma_2d<CG>(sB, mB, fb, k0, bn0);
           } else if (ROLE == ROLE_FWD2) {
-            tma_load_3d(sB, mB, fb, k0, q.n0, q.i);
+            tma_3d<CG>(sB, mB, fb, k0, bn0, q.i);
           } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
-            for (int j = 0; j < q.bn / 64; ++j) tma_load_3d(sB + j * 8192, mB, fb, q.n0 + 64 * j, k0, q.i);
+            for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i);
           } else {
-            for (int j = 0; j < q.bn / 64; ++j) tma_load_2d(sB + j * 8192, mB, fb, q.n0 + 64 * j, q.r0 + k0);
+            for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -335,18 +413,18 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     }
   } else if (warp == 1) {
     // ================= MMA issuer =================
-    if (lane == 0) {
+    if (lane == 0 && cta_rank == 0) {      // the leader issues for the pair
       int stage = 0;
       uint32_t phase = 0;
       int buf = 0;
       uint32_t acc_phase = 0;
       bool alive = true;
-      for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
+      for (int ti = unit; ti < total && alive; ti += unit_stride) {
         const Tile t = fetch_tile<ROLE>(p, ti);
         const TileGeom q = tile_geom<ROLE>(p, t);
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
                                ((uint32_t)RT::B_MN << 16) | ((uint32_t)(q.bn >> 3) << 17) |
-                               ((uint32_t)(BM >> 4) << 24);
+                               ((uint32_t)(Geo<CG>::kTileM >> 4) << 24);
         if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag, p.status, 2)) { alive = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * kAccCols;
@@ -361,24 +439,26 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
                                          : make_desc(sA + kk * 32, 16, 1024);
             const uint64_t db = RT::B_MN ? make_desc(sB + kk * 2048, 8192, 1024)
                                          : make_desc(sB + kk * 32, 16, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+            if (CG == 2) umma2_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+            else umma_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
-          umma_commit(empty_bar(stage));     // frees the stage when these MMAs have read it
+          // frees the stage (in both CTAs of a pair) when these MMAs have read it
+          if (CG == 2) umma2_commit(empty_bar(stage)); else umma_commit(empty_bar(stage));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!alive) break;
-        umma_commit(tfull_bar(buf));         // accumulator complete
+        if (CG == 2) umma2_commit(tfull_bar(buf)); else umma_commit(tfull_bar(buf));   // accumulator complete
         if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
       }
     }
   } else {
     // ================= epilogue warps =================
     const int quad = warp & 3;                 // tensor-memory lanes [32*quad, 32*quad + 32)
-    const int row_in_tile = quad * 32 + lane;
+    const int row_in_tile = BM * (int)cta_rank + quad * 32 + lane;   // row of the (pair's) tile
     int buf = 0;
     uint32_t acc_phase = 0;
     bool alive = true;
-    for (int ti = blockIdx.x; ti < total && alive; ti += gridDim.x) {
+    for (int ti = unit; ti < total && alive; ti += unit_stride) {
       const Tile t = fetch_tile<ROLE>(p, ti);
       const TileGeom q = tile_geom<ROLE>(p, t);
       // the whole warp must agree before the warp-collective tensor-memory loads
@@ -532,7 +612,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(buf));
+      if (lane == 0) {
+        if (CG == 2) mbar_arrive_cluster(mapa_rank(tempty_bar(buf), 0)); else mbar_arrive(tempty_bar(buf));
+      }
       if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
     }
   }
@@ -540,9 +622,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   // ---- teardown ----
   __syncthreads();
   if (*abort_flag) __nanosleep(200000);    // let copies in flight land before the CTA retires
+  if (CG == 2) cluster_sync_all();         // the peer may still signal this CTA's barriers until here
   tc_fence_after();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    if (CG == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
   }
 }
 
@@ -606,16 +692,49 @@ int pick_bn(int extent, const int* cand, int ncand) {
   return best;
 }
 
-template <int ROLE>
+template <int ROLE, int CG>
 int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    Geo<CG>::kSmemBytes));
     attr_set = true;
   }
-  tc_grouped_kernel<ROLE><<<grid, kThreads, kSmemBytes, st>>>(p);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(grid / CG * CG);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = Geo<CG>::kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CG;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (CG == 2) {
+    // Persistent kernel: launch exactly as many CTA pairs as can be resident at once (SMs that
+    // cannot be paired stay idle); a pair that had to wait for a free slot would run its whole
+    // share of the tile list after everyone else.
+    static int max_clusters = 0;
+    if (!max_clusters) {
+      cfg.gridDim = dim3(grid / CG * CG);
+      MOHGE_CUDA(cudaOccupancyMaxActiveClusters(&max_clusters, tc_grouped_kernel<ROLE, CG>, &cfg));
+      if (max_clusters < 1) max_clusters = 1;
+    }
+    const int want = grid / CG < max_clusters ? grid / CG : max_clusters;
+    cfg.gridDim = dim3(want * CG);
+  }
+  MOHGE_CUDA(cudaLaunchKernelEx(&cfg, tc_grouped_kernel<ROLE, CG>, p));
   MOHGE_LAUNCH_CHECK("tc_grouped_kernel");
   return MOHGE_OK;
+}
+
+// CTAs per MMA for the grouped roles (debugging switch MOHGE_TC_CG=1 keeps the single-CTA form)
+int cta_group_size() {
+  const char* e = getenv("MOHGE_TC_CG");
+  return (e && e[0] == '1') ? 1 : 2;
 }
 
 }  // namespace
@@ -671,9 +790,9 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
   p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn;
   const int grid = p.plain_total < sm_count ? p.plain_total : sm_count;
   switch (role) {
-    case ROLE_LOGITS: return launch_role<ROLE_LOGITS>(p, grid, st);
-    case ROLE_ROUTER_DW: return launch_role<ROLE_ROUTER_DW>(p, grid, st);
-    default: return launch_role<ROLE_ROUTER_DX>(p, grid, st);
+    case ROLE_LOGITS: return launch_role<ROLE_LOGITS, 1>(p, grid, st);
+    case ROLE_ROUTER_DW: return launch_role<ROLE_ROUTER_DW, 1>(p, grid, st);
+    default: return launch_role<ROLE_ROUTER_DX, 1>(p, grid, st);
   }
 }
 
@@ -709,7 +828,13 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   p.accumulate = accumulate; p.status = status;
 
   const uint64_t d = D.d, rows = D.Rcap, pitchAU = 2ull * D.Wmax * 2, pitchH = (uint64_t)D.Wmax * 2;
-  const int cand_n[3] = {256, 192, 128};
+  const int CG = cta_group_size();
+  // UMMA N candidates.  A CTA pair splits B in halves, and an MN-major half must stay a multiple
+  // of the 64-element swizzle block, so N = 192 is only available to the single-CTA form.
+  const int cand_n1[3] = {256, 192, 128};
+  const int cand_n2[2] = {256, 128};
+  const int* cand_n = CG == 2 ? cand_n2 : cand_n1;
+  const int ncand = CG == 2 ? 2 : 3;
   const int cand_h[3] = {128, 96, 64};
   int bn_plan[MOHGE_MAX_GROUPS];
   int32_t rc = MOHGE_OK;
@@ -720,7 +845,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
     uint32_t box[3];
     switch (role) {
       case ROLE_FWD1: {
-        const int half = pick_bn(D.W[g], cand_h, 3);
+        const int half = pick_bn(D.W[g], cand_h, CG == 2 ? 1 : 3) ;
         p.BN[g] = 2 * half; bn_plan[g] = half;
         dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
@@ -730,16 +855,16 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         rc = encode_map(&p.mapB[g], P.w13[g], 3, dims, str, box);
       } break;
       case ROLE_FWD2: {
-        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, 3);
+        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
         dims[0] = W; dims[1] = rows; str[0] = pitchH; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
         if (rc) break;
         dims[0] = W; dims[1] = d; dims[2] = N; str[0] = W * 2; str[1] = d * W * 2;
-        box[0] = BK; box[1] = p.BN[g]; box[2] = 1;
+        box[0] = BK; box[1] = p.BN[g] / CG; box[2] = 1;
         rc = encode_map(&p.mapB[g], P.w2[g], 3, dims, str, box);
       } break;
       case ROLE_DGRAD_DOWN: {
-        p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, 3);
+        p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
         p.E = (const __nv_bfloat16*)B;
         dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
@@ -749,7 +874,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         rc = encode_map(&p.mapB[g], P.w2[g], 3, dims, str, box);
       } break;
       case ROLE_DGRAD_13: {
-        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, 3);
+        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
         dims[0] = 2 * W; dims[1] = rows; str[0] = pitchAU; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
         if (rc) break;
@@ -758,7 +883,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         rc = encode_map(&p.mapB[g], P.w13[g], 3, dims, str, box);
       } break;
       case ROLE_WGRAD_DOWN: {
-        p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, 3);
+        p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
         dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = 64; box[1] = BK;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
         if (rc) break;
@@ -766,7 +891,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         rc = encode_map(&p.mapB[g], B, 2, dims, str, box);
       } break;
       default: {  // ROLE_WGRAD_13
-        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, 3);
+        p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
         dims[0] = 2 * W; dims[1] = rows; str[0] = pitchAU; box[0] = 64; box[1] = BK;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
         if (rc) break;
@@ -776,16 +901,26 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
     }
   }
   if (rc) return rc;
-  rc = launch_build_tiles_plan(make_plan(D, role, BM, bn_plan, role == ROLE_FWD1), aligned, tile_count,
+  rc = launch_build_tiles_plan(make_plan(D, role, BM * CG, bn_plan, role == ROLE_FWD1), aligned, tile_count,
                                tiles, tiles_cap, status, st);
   if (rc) return rc;
+  if (CG == 2) {
+    switch (role) {
+      case ROLE_FWD1: return launch_role<ROLE_FWD1, 2>(p, sm_count, st);
+      case ROLE_FWD2: return launch_role<ROLE_FWD2, 2>(p, sm_count, st);
+      case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 2>(p, sm_count, st);
+      case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 2>(p, sm_count, st);
+      case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 2>(p, sm_count, st);
+      default: return launch_role<ROLE_WGRAD_13, 2>(p, sm_count, st);
+    }
+  }
   switch (role) {
-    case ROLE_FWD1: return launch_role<ROLE_FWD1>(p, sm_count, st);
-    case ROLE_FWD2: return launch_role<ROLE_FWD2>(p, sm_count, st);
-    case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN>(p, sm_count, st);
-    case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13>(p, sm_count, st);
-    case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN>(p, sm_count, st);
-    default: return launch_role<ROLE_WGRAD_13>(p, sm_count, st);
+    case ROLE_FWD1: return launch_role<ROLE_FWD1, 1>(p, sm_count, st);
+    case ROLE_FWD2: return launch_role<ROLE_FWD2, 1>(p, sm_count, st);
+    case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 1>(p, sm_count, st);
+    case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 1>(p, sm_count, st);
+    case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 1>(p, sm_count, st);
+    default: return launch_role<ROLE_WGRAD_13, 1>(p, sm_count, st);
   }
 }
 
