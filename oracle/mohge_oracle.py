@@ -39,7 +39,8 @@ __all__ = [
     "OracleConfig", "router_logits", "topk_rounds", "route_definition",
     "route_values", "gates_from_selection", "exp_spec", "sigmoid_spec",
     "tree_sum_f32", "route_spec", "aux_stats", "dispatch", "permute_rows",
-    "swiglu_ffn", "layer_forward", "layer_backward", "layer_loss",
+    "swiglu_ffn", "expert_backward", "layer_forward", "layer_backward", "layer_loss",
+    "aux_losses",
 ]
 
 
@@ -354,6 +355,23 @@ def _as64(a):
     return np.asarray(a, np.float64)
 
 
+def expert_backward(xe, w13_e, w2_e, A, U, H, dY):
+    """Gradients of one SwiGLU expert given dY = d<loss>/dY for its rows.
+
+    With Y = H W_down^T, H = silu(A) * U, A = X W_gate^T, U = X W_up^T:
+    dH = dY W_down; dW_down = dY^T H; dA = dH * U * silu'(A); dU = dH * silu(A);
+    dW13 = [dA | dU]^T X; dX = dA W_gate + dU W_up."""
+    W = w2_e.shape[1]
+    dH = dY @ w2_e
+    dw2 = dY.T @ H
+    sg = _sigmoid(A)
+    dA = dH * U * sg * (1.0 + A * (1.0 - sg))
+    dU = dH * A * sg
+    dw13 = np.concatenate([dA.T @ xe, dU.T @ xe], axis=0)
+    dx = dA @ w13_e[:W] + dU @ w13_e[W:]
+    return dict(dH=dH, dA=dA, dU=dU, dw2=dw2, dw13=dw13, dx=dx)
+
+
 def layer_forward(cfg: OracleConfig, x, w_r, w13: List, w2: List, logit_bias=None,
                   logits=None, mode="definition"):
     """Forward of the whole layer.
@@ -427,14 +445,10 @@ def layer_backward(fwd, w13: List, w2: List, dy, with_aux=True, aux_counts=None)
         w13_e, w2_e = _as64(w13[g][i]), _as64(w2[g][i])
         dgate[t_idx, k_idx] = np.sum(dy[t_idx] * Y, axis=1)
         dY = gate[t_idx, k_idx][:, None] * dy[t_idx]
-        dH = dY @ w2_e
-        dw2[g][i] = dY.T @ H
-        sg = _sigmoid(A)
-        dA = dH * U * sg * (1.0 + A * (1.0 - sg))
-        dU = dH * A * sg
-        dw13[g][i][:W] = dA.T @ x[t_idx]
-        dw13[g][i][W:] = dU.T @ x[t_idx]
-        np.add.at(dx, t_idx, dA @ w13_e[:W] + dU @ w13_e[W:])
+        eb = expert_backward(x[t_idx], w13_e, w2_e, A, U, H, dY)
+        dw2[g][i] = eb["dw2"]
+        dw13[g][i] = eb["dw13"]
+        np.add.at(dx, t_idx, eb["dx"])
     # ---- router: Eq. 6 -> Eq. 4 -> Eq. 3 -> Eq. 2 ----
     GS, ESp, ESpp = fwd["GS"], fwd["ESp"], fwd["ESpp"]
     key = np.take_along_axis(ESpp, expert_idx.astype(np.int64), axis=1)

@@ -30,6 +30,21 @@ def test_single_expert_is_a_dense_swiglu_ffn():
     np.testing.assert_allclose(f["y"], ref.numpy(), rtol=1e-12, atol=1e-13)
 
 
+def test_expert_backward_matches_autograd_of_a_dense_swiglu_ffn():
+    rng = np.random.default_rng(3)
+    n, d, W = 7, 10, 6
+    x, w13, w2, dY = (rng.normal(size=s) for s in ((n, d), (2 * W, d), (d, W), (n, d)))
+    A, U, H, Y = O.swiglu_ffn(x, w13, w2)
+    got = O.expert_backward(x, w13, w2, A, U, H, dY)
+    tx, t13, t2 = (torch.tensor(a, requires_grad=True) for a in (x, w13, w2))
+    ty = (torch.nn.functional.silu(tx @ t13[:W].T) * (tx @ t13[W:].T)) @ t2.T
+    (ty * torch.tensor(dY)).sum().backward()
+    np.testing.assert_allclose(Y, ty.detach().numpy(), rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(got["dx"], tx.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(got["dw13"], t13.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(got["dw2"], t2.grad.numpy(), rtol=1e-10, atol=1e-12)
+
+
 def _torch_dense_forward(cfg, x, w_r, w13, w2, G):
     """Independent forward: every expert is evaluated on every token and mixed
     with a dense [T, N_e] gate matrix built with torch.topk / torch.softmax."""
