@@ -28,7 +28,7 @@ sys.path.insert(0, ROOT)
 
 import torch  # noqa: E402
 
-from paper_2604_23108_b200.inputs import WORKLOADS, Workload, zipf_logit_bias  # noqa: E402
+from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs  # noqa: E402
 
 METRIC = "MoHGE layer fwd+bwd tokens/s"
 UNIT = "tokens/s"
@@ -43,25 +43,6 @@ def _peaks():
         return dict(hbm=d["hbm_gbs"], tf_burst=d["bf16_tflops"], tf_sustained=d["bf16_tflops_sustained"],
                     source="measured")
     return dict(hbm=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
-
-
-def device_inputs(wl: Workload, device, seed=None):
-    """Seeded synthetic tensors drawn on the device (same distributions as inputs.make_inputs)."""
-    gen = torch.Generator(device=device)
-    gen.manual_seed(wl.seed if seed is None else seed)
-    dt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
-
-    def normal(shape, std):
-        return (torch.randn(shape, generator=gen, dtype=torch.float32, device=device) * std).to(dt)
-
-    d = wl.d_model
-    inp = dict(x=normal((wl.T, d), 1.0), w_router=normal((wl.n_logits, d), 0.02),
-               dy=normal((wl.T, d), 1.0))
-    inp["w13"] = [normal((wl.experts_per_group, 2 * w, d), 0.02) for w in wl.group_width]
-    inp["w2"] = [normal((wl.experts_per_group, d, w), 0.02) for w in wl.group_width]
-    b = zipf_logit_bias(wl)
-    inp["logit_bias"] = None if b is None else b.to(device)
-    return inp
 
 
 class ClockSampler:
@@ -204,7 +185,7 @@ def main():
     gcfg = B.Config(d_model=wl.d_model, n_groups=wl.n_groups, experts_per_group=wl.experts_per_group,
                     k_groups=wl.k_groups, k_experts=wl.k_experts, group_width=list(wl.group_width),
                     dtype=wl.dtype, row_align=128 if wl.dtype == "bf16" else 1)
-    inp = device_inputs(wl, dev, seed=wl.seed + rank)
+    inp = make_device_inputs(wl, dev, seed=wl.seed + rank)
     buf = B.LayerBuffers(gcfg, wl.T, device=dev)
     T = wl.T
     ev = lambda: torch.cuda.Event(enable_timing=True)

@@ -19,7 +19,7 @@ from typing import List, Optional
 
 import torch
 
-__all__ = ["Workload", "WORKLOADS", "make_inputs", "zipf_logit_bias"]
+__all__ = ["Workload", "WORKLOADS", "make_inputs", "make_device_inputs", "zipf_logit_bias"]
 
 
 @dataclass(frozen=True)
@@ -96,4 +96,25 @@ def make_inputs(wl: Workload, seed: Optional[int] = None, T: Optional[int] = Non
         out["w13"] = [normal((wl.experts_per_group, 2 * w, d), 0.02) for w in wl.group_width]
         out["w2"] = [normal((wl.experts_per_group, d, w), 0.02) for w in wl.group_width]
     out["logit_bias"] = zipf_logit_bias(wl)
+    return out
+
+
+def make_device_inputs(wl: Workload, device, seed: Optional[int] = None):
+    """The same recipe drawn with a generator on `device` (used at the full benchmark sizes,
+    where drawing gigabytes on the host would take minutes).  Same keys as `make_inputs`;
+    the values differ from the CPU stream but have the same distributions and draw order."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(wl.seed if seed is None else seed)
+    dt = _torch_dtype(wl.dtype)
+    d = wl.d_model
+
+    def normal(shape, std):
+        return (torch.randn(shape, generator=gen, dtype=torch.float32, device=device) * std).to(dt)
+
+    out = {"x": normal((wl.T, d), 1.0), "w_router": normal((wl.n_logits, d), 0.02),
+           "dy": normal((wl.T, d), 1.0)}
+    out["w13"] = [normal((wl.experts_per_group, 2 * w, d), 0.02) for w in wl.group_width]
+    out["w2"] = [normal((wl.experts_per_group, d, w), 0.02) for w in wl.group_width]
+    b = zipf_logit_bias(wl)
+    out["logit_bias"] = None if b is None else b.to(device)
     return out
