@@ -1,10 +1,12 @@
 // Ragged grouped GEMMs of the expert layer on the 5th-generation tensor cores (sm_100a):
 // tcgen05.mma kind::f16 (BF16 operands, FP32 accumulators in tensor memory), operands staged in
-// shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), a 4-stage mbarrier pipeline,
+// shared memory by TMA (cp.async.bulk.tensor, 128-byte swizzle), a multi-stage mbarrier pipeline,
 // double-buffered accumulators, and warp-specialised roles:
 //   warp 0      TMA producer (one elected lane)
 //   warp 1      tensor-memory owner and MMA issuer (one elected lane)
-//   warps 2..5  epilogue: tcgen05.ld -> registers -> fused element-wise math -> global memory
+//   warps 2..5  epilogue: tcgen05.ld -> registers -> fused element-wise math -> swizzled staging
+//               buffers in shared memory -> TMA stores (every global write of the expert roles is
+//               a full 128-byte row piece; the SwiGLU backward also reads A and U through TMA)
 // One persistent CTA per SM walks the device-built, cost-sorted tile list with stride gridDim.x.
 //
 // Six roles share the kernel (C = A . B^T over a contraction index k):
@@ -42,11 +44,17 @@ constexpr int kAccCols = 256;                 // tensor-memory columns per accum
 // CG = CTAs per MMA (tcgen05 cta_group).  CG = 2 pairs the two CTAs of a cluster on one
 // 256 x N tile: each CTA stages its own 128 rows of A and HALF of B, so operand traffic per FLOP
 // drops by a third and the smaller stages allow a six-deep pipeline.
+// Epilogue staging: each of the four epilogue warps owns a ring of four 4 KiB buffers
+// (32 rows x 128 bytes, 128-byte swizzle: the layout a TMA box of 32 rows expects).
+constexpr int kStgBufBytes = 4096;
+constexpr int kStgBufs = 4;
+constexpr int kStgBytes = 4 * kStgBufs * kStgBufBytes;       // 64 KiB per CTA
+
 template <int CG> struct Geo {
-  static constexpr int kStages = CG == 1 ? 4 : 6;
+  static constexpr int kStages = CG == 1 ? 3 : 5;
   static constexpr int kBBytes = 256 / CG * BK * 2;          // 32 KiB or 16 KiB
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kStgBytes + 1024 + 512;
   static constexpr int kTileM = BM * CG;
 };
 
@@ -68,6 +76,10 @@ template <int ROLE> __host__ __device__ constexpr bool is_plain() { return ROLE 
 struct TcParams {
   CUtensorMap mapA[MOHGE_MAX_GROUPS];
   CUtensorMap mapB[MOHGE_MAX_GROUPS];
+  // epilogue outputs, boxes of 32 rows x 128 bytes.  FWD1: A, U, H regions per group;
+  // FWD2 / DGRAD_13: [0][0]; DGRAD_DOWN: dA, dU regions per group; WGRAD: FP32 [N, rows, cols]
+  CUtensorMap mapO[3][MOHGE_MAX_GROUPS];
+  CUtensorMap mapE[2][MOHGE_MAX_GROUPS];   // DGRAD_DOWN epilogue inputs: saved A and U regions
   GroupShape gs;
   GroupPtrs gp;
   int BN[MOHGE_MAX_GROUPS];      // UMMA N per group (FWD1: gate half + up half)
@@ -143,6 +155,41 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// ---- TMA stores from the epilogue staging buffers (bulk async-groups, one per store)
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+// element-wise FP32 add into global memory (each output element is touched by exactly one box)
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// generic-proxy writes to shared memory become visible to the async proxy (TMA)
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Address of 16-byte piece j of row r in a staging buffer (32 rows x 128 B, 128-byte swizzle)
+__device__ __forceinline__ uint32_t stg_addr(uint32_t buf, int r, int j) {
+  return buf + (uint32_t)r * 128u + (uint32_t)((j ^ (r & 7)) << 4);
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
 }
 
 // ---- CTA-pair (cluster of 2) helpers
@@ -321,14 +368,16 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  // barrier block after the stages
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * kStageBytes);
-  const uint32_t bar0 = smem_base + kStages * kStageBytes;
+  // layout: pipeline stages | epilogue staging (4 warps x 4 buffers x 4 KiB) | barriers
+  const uint32_t stg0 = smem_base + kStages * kStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * kStageBytes + kStgBytes);
+  const uint32_t bar0 = stg0 + kStgBytes;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  auto ein_bar = [&](int quad, int set) { return bar0 + 8u * (2 * kStages + 4 + quad * 2 + set); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -342,6 +391,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       mbar_init(tfull_bar(b), 1);
       mbar_init(tempty_bar(b), 4 * CG);  // four epilogue warps per CTA
     }
+    for (int i = 0; i < 8; ++i) mbar_init(ein_bar(i >> 1, i & 1), 1);   // epilogue input loads
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -455,80 +505,170 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     // ================= epilogue warps =================
     const int quad = warp & 3;                 // tensor-memory lanes [32*quad, 32*quad + 32)
     const int row_in_tile = BM * (int)cta_rank + quad * 32 + lane;   // row of the (pair's) tile
+    const uint32_t stg = stg0 + (uint32_t)quad * (kStgBufs * kStgBufBytes);   // this warp's staging ring
+    uint32_t n_store = 0;                      // stores issued so far: ring slot = n_store % 4
+    uint32_t n_chunk = 0;                      // SwiGLU backward: input chunks consumed so far
     int buf = 0;
     uint32_t acc_phase = 0;
     bool alive = true;
     for (int ti = unit; ti < total && alive; ti += unit_stride) {
       const Tile t = fetch_tile<ROLE>(p, ti);
       const TileGeom q = tile_geom<ROLE>(p, t);
+      // row-tiled expert roles: first row of this warp; segments are 128-row aligned, so the
+      // rows of one CTA are either all inside the expert's segment or all outside
+      const int row0 = q.m0 + BM * (int)cta_rank + quad * 32;
+      const bool rows_ok = BM * (int)cta_rank < t.ext;
+      int nch_in = 0;
+      if (RT::EPI == EPI_SWIGLU_BWD) {
+        // A and U of the first 64 columns are fetched while the MMAs of this tile still run
+        if (rows_ok) { const int left = q.W - q.n0; nch_in = ((left < q.bn ? left : q.bn) + 63) / 64; }
+        if (nch_in > 0 && lane == 0) {
+          bulk_wait_read<0>();
+          const uint32_t set = n_chunk & 1u, bar = ein_bar(quad, set);
+          mbar_expect_tx(bar, 2 * kStgBufBytes);
+          tma_load_2d(stg + set * 2 * kStgBufBytes, &p.mapE[0][q.g], bar, q.n0, row0);
+          tma_load_2d(stg + (set * 2 + 1) * kStgBufBytes, &p.mapE[1][q.g], bar, q.n0, row0);
+        }
+      }
       // the whole warp must agree before the warp-collective tensor-memory loads
       const bool got = mbar_wait(tfull_bar(buf), acc_phase, abort_flag, p.status, 4);
       if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kAccCols;
-      const long long d = p.gs.d, pitchAU = 2LL * p.gs.Wmax, pitchH = p.gs.Wmax;
+      const long long d = p.gs.d;
       if (RT::EPI == EPI_SWIGLU_FWD) {
         const int half = q.bn >> 1;
-        const long long row = q.m0 + row_in_tile;
-        const bool row_ok = row_in_tile < t.ext;
-        for (int c = 0; c < half; c += 32) {
-          uint32_t ra[32], ru[32];
-          tmem_ld32(taddr + c, ra);
-          tmem_ld32(taddr + half + c, ru);
-          tmem_ld_wait();
-          const int valid = q.W - (q.n0 + c);
-          if (row_ok && valid > 0) {
-            float a[32], u[32], h[32];
+        for (int c = 0; rows_ok && c < half && q.n0 + c < q.W; c += 64) {
+          if (lane == 0) bulk_wait_read<1>();          // three of the four ring slots are free
+          __syncwarp();
+          const uint32_t bA = stg + ((n_store & 3u) << 12), bU = stg + (((n_store + 1) & 3u) << 12),
+                         bH = stg + (((n_store + 2) & 3u) << 12);
+          n_store += 3;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              a[j] = __uint_as_float(ra[j]);
-              u[j] = __uint_as_float(ru[j]);
-              h[j] = a[j] / (1.0f + __expf(-a[j])) * u[j];
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t ra[32], ru[32];
+            tmem_ld32(taddr + c + 32 * hh, ra);
+            tmem_ld32(taddr + half + c + 32 * hh, ru);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j4 = 0; j4 < 4; ++j4) {
+              uint32_t pa[4], pu[4], ph[4];
+#pragma unroll
+              for (int e2 = 0; e2 < 4; ++e2) {
+                const float a0 = __uint_as_float(ra[j4 * 8 + 2 * e2]), a1 = __uint_as_float(ra[j4 * 8 + 2 * e2 + 1]);
+                const float u0 = __uint_as_float(ru[j4 * 8 + 2 * e2]), u1 = __uint_as_float(ru[j4 * 8 + 2 * e2 + 1]);
+                const float h0 = a0 / (1.0f + __expf(-a0)) * u0, h1 = a1 / (1.0f + __expf(-a1)) * u1;
+                pa[e2] = pack2(a0, a1); pu[e2] = pack2(u0, u1); ph[e2] = pack2(h0, h1);
+              }
+              st_shared_v4(stg_addr(bA, lane, hh * 4 + j4), pa[0], pa[1], pa[2], pa[3]);
+              st_shared_v4(stg_addr(bU, lane, hh * 4 + j4), pu[0], pu[1], pu[2], pu[3]);
+              st_shared_v4(stg_addr(bH, lane, hh * 4 + j4), ph[0], ph[1], ph[2], ph[3]);
             }
-            __nv_bfloat16* pa = p.C + row * pitchAU + q.n0 + c;
-            store_row32(pa, a, valid);
-            store_row32(pa + q.W, u, valid);
-            store_row32(p.C2 + row * pitchH + q.n0 + c, h, valid);
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&p.mapO[0][q.g], bA, q.n0 + c, row0); bulk_commit();
+            tma_store_2d(&p.mapO[1][q.g], bU, q.n0 + c, row0); bulk_commit();
+            tma_store_2d(&p.mapO[2][q.g], bH, q.n0 + c, row0); bulk_commit();
           }
         }
       } else if (RT::EPI == EPI_BF16) {
-        const long long row = q.m0 + row_in_tile;
-        const bool row_ok = row_in_tile < t.ext;
-        for (int c = 0; c < q.bn; c += 32) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c, r);
+        for (int c = 0; rows_ok && c < q.bn && q.n0 + c < (int)d; c += 64) {
+          if (lane == 0) bulk_wait_read<3>();
+          __syncwarp();
+          const uint32_t bO = stg + ((n_store & 3u) << 12);
+          n_store += 1;
+          uint32_t r0[32], r1[32];
+          tmem_ld32(taddr + c, r0);
+          tmem_ld32(taddr + c + 32, r1);
           tmem_ld_wait();
-          const int valid = (int)d - (q.n0 + c);
-          if (row_ok && valid > 0) {
-            float v[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-            store_row32(p.C + row * d + q.n0 + c, v, valid);
+          for (int j4 = 0; j4 < 4; ++j4) {
+            st_shared_v4(stg_addr(bO, lane, j4),
+                         pack2(__uint_as_float(r0[j4 * 8 + 0]), __uint_as_float(r0[j4 * 8 + 1])),
+                         pack2(__uint_as_float(r0[j4 * 8 + 2]), __uint_as_float(r0[j4 * 8 + 3])),
+                         pack2(__uint_as_float(r0[j4 * 8 + 4]), __uint_as_float(r0[j4 * 8 + 5])),
+                         pack2(__uint_as_float(r0[j4 * 8 + 6]), __uint_as_float(r0[j4 * 8 + 7])));
+            st_shared_v4(stg_addr(bO, lane, 4 + j4),
+                         pack2(__uint_as_float(r1[j4 * 8 + 0]), __uint_as_float(r1[j4 * 8 + 1])),
+                         pack2(__uint_as_float(r1[j4 * 8 + 2]), __uint_as_float(r1[j4 * 8 + 3])),
+                         pack2(__uint_as_float(r1[j4 * 8 + 4]), __uint_as_float(r1[j4 * 8 + 5])),
+                         pack2(__uint_as_float(r1[j4 * 8 + 6]), __uint_as_float(r1[j4 * 8 + 7])));
           }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) { tma_store_2d(&p.mapO[0][0], bO, q.n0 + c, row0); bulk_commit(); }
         }
       } else if (RT::EPI == EPI_SWIGLU_BWD) {
-        const long long row = q.m0 + row_in_tile;
-        const bool row_ok = row_in_tile < t.ext;
-        for (int c = 0; c < q.bn; c += 32) {
+        // per 64-column chunk: A and U arrive by TMA in one of two buffer pairs, dA and dU are
+        // written over them in place and leave by TMA; the next chunk's loads fly meanwhile
+        for (int ci = 0; ci < nch_in; ++ci, ++n_chunk) {
+          const int c = ci * 64;
+          const uint32_t set = n_chunk & 1u;
+          if (ci + 1 < nch_in && lane == 0) {
+            bulk_wait_read<0>();                       // the other pair's last stores have left
+            const uint32_t bar = ein_bar(quad, set ^ 1u);
+            mbar_expect_tx(bar, 2 * kStgBufBytes);
+            tma_load_2d(stg + (set ^ 1u) * 2 * kStgBufBytes, &p.mapE[0][q.g], bar, q.n0 + c + 64, row0);
+            tma_load_2d(stg + ((set ^ 1u) * 2 + 1) * kStgBufBytes, &p.mapE[1][q.g], bar, q.n0 + c + 64, row0);
+          }
+          const bool in_ok = mbar_wait(ein_bar(quad, set), (n_chunk >> 1) & 1u, abort_flag, p.status, 5);
+          if (!__all_sync(0xffffffffu, in_ok)) { alive = false; break; }
+          const uint32_t bA = stg + set * 2 * kStgBufBytes, bU = bA + kStgBufBytes;
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c + 32 * hh, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j4 = 0; j4 < 4; ++j4) {
+              const uint32_t aa = stg_addr(bA, lane, hh * 4 + j4), ua = stg_addr(bU, lane, hh * 4 + j4);
+              const uint4 va = ld_shared_v4(aa), vu = ld_shared_v4(ua);
+              const uint32_t wa[4] = {va.x, va.y, va.z, va.w}, wu[4] = {vu.x, vu.y, vu.z, vu.w};
+              uint32_t oa[4], ou[4];
+#pragma unroll
+              for (int e2 = 0; e2 < 4; ++e2) {
+                const float a0 = bf_lo(wa[e2]), a1 = bf_hi(wa[e2]), u0 = bf_lo(wu[e2]), u1 = bf_hi(wu[e2]);
+                const float dh0 = __uint_as_float(r[j4 * 8 + 2 * e2]), dh1 = __uint_as_float(r[j4 * 8 + 2 * e2 + 1]);
+                const float s0 = 1.0f / (1.0f + __expf(-a0)), s1 = 1.0f / (1.0f + __expf(-a1));
+                oa[e2] = pack2(dh0 * u0 * s0 * (1.0f + a0 * (1.0f - s0)), dh1 * u1 * s1 * (1.0f + a1 * (1.0f - s1)));
+                ou[e2] = pack2(dh0 * a0 * s0, dh1 * a1 * s1);
+              }
+              st_shared_v4(aa, oa[0], oa[1], oa[2], oa[3]);
+              st_shared_v4(ua, ou[0], ou[1], ou[2], ou[3]);
+            }
+          }
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&p.mapO[0][q.g], bA, q.n0 + c, row0);
+            tma_store_2d(&p.mapO[1][q.g], bU, q.n0 + c, row0);
+            bulk_commit();
+          }
+        }
+        if (!alive) break;
+      } else if (RT::EPI == EPI_F32) {
+        // weight gradients: FP32 boxes of 32 rows x 32 columns into [expert, rows, columns]
+        const int Mext = ROLE == ROLE_WGRAD_DOWN ? (int)d : 2 * q.W;
+        const int Next = ROLE == ROLE_WGRAD_DOWN ? q.W : (int)d;
+        for (int c = 0; row0 < Mext && c < q.bn && q.n0 + c < Next; c += 32) {
+          if (lane == 0) bulk_wait_read<3>();
+          __syncwarp();
+          const uint32_t bO = stg + ((n_store & 3u) << 12);
+          n_store += 1;
           uint32_t r[32];
           tmem_ld32(taddr + c, r);
           tmem_ld_wait();
-          const int valid = q.W - (q.n0 + c);
-          if (row_ok && valid > 0) {
-            float a[32], u[32], da[32], du[32];
-            const __nv_bfloat16* pe = p.E + row * pitchAU + q.n0 + c;
-            load_row32(pe, a, valid);
-            load_row32(pe + q.W, u, valid);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float dh = __uint_as_float(r[j]);
-              const float sg = 1.0f / (1.0f + __expf(-a[j]));
-              da[j] = dh * u[j] * sg * (1.0f + a[j] * (1.0f - sg));
-              du[j] = dh * a[j] * sg;
-            }
-            __nv_bfloat16* po = p.C + row * pitchAU + q.n0 + c;
-            store_row32(po, da, valid);
-            store_row32(po + q.W, du, valid);
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(stg_addr(bO, lane, j), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            if (p.accumulate) tma_reduce_add_3d(&p.mapO[0][q.g], bO, q.n0 + c, row0, q.i);
+            else tma_store_3d(&p.mapO[0][q.g], bO, q.n0 + c, row0, q.i);
+            bulk_commit();
           }
         }
       } else if (RT::EPI == EPI_LOGITS) {
@@ -581,34 +721,6 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             store_row32(po, v, valid);
           }
         }
-      } else {  // EPI_F32: weight gradients
-        const int Mext = ROLE == ROLE_WGRAD_DOWN ? (int)d : 2 * q.W;
-        const int Next = ROLE == ROLE_WGRAD_DOWN ? q.W : (int)d;
-        float* base = ROLE == ROLE_WGRAD_DOWN ? p.gp.dw2[q.g] + (size_t)q.i * d * q.W
-                                              : p.gp.dw13[q.g] + (size_t)q.i * 2 * q.W * d;
-        const int m = q.m0 + row_in_tile;
-        const bool row_ok = m < Mext;
-        for (int c = 0; c < q.bn; c += 32) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c, r);
-          tmem_ld_wait();
-          const int valid = Next - (q.n0 + c);
-          if (row_ok && valid > 0) {
-            float* po = base + (size_t)m * Next + q.n0 + c;
-#pragma unroll
-            for (int v4 = 0; v4 < 8; ++v4) {
-              if (v4 * 4 < valid) {
-                float4 o = make_float4(__uint_as_float(r[v4 * 4]), __uint_as_float(r[v4 * 4 + 1]),
-                                       __uint_as_float(r[v4 * 4 + 2]), __uint_as_float(r[v4 * 4 + 3]));
-                if (p.accumulate) {
-                  const float4 old = *reinterpret_cast<const float4*>(po + v4 * 4);
-                  o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                }
-                *reinterpret_cast<float4*>(po + v4 * 4) = o;
-              }
-            }
-          }
-        }
       }
       tc_fence_before();
       __syncwarp();
@@ -617,6 +729,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       }
       if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) bulk_wait_all();            // staged stores have left before the CTA retires
   }
 
   // ---- teardown ----
@@ -650,9 +763,9 @@ EncodeFn get_encode() {
   return fn;
 }
 
-// BF16 tensor of `rank` dims (innermost first); strides in bytes for dims 1..rank-1
+// Tensor of `rank` dims (innermost first), BF16 unless `f32`; strides in bytes for dims 1..rank-1
 int32_t encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims,
-                   const uint64_t* strides, const uint32_t* box) {
+                   const uint64_t* strides, const uint32_t* box, bool f32 = false) {
   EncodeFn fn = get_encode();
   if (!fn) {
     set_error("cuTensorMapEncodeTiled is not available from the driver");
@@ -666,7 +779,8 @@ int32_t encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* d
     es[i] = 1;
     if (i > 0) gs[i - 1] = strides[i - 1];
   }
-  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gd, gs,
+  const CUresult r = fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                        (cuuint32_t)rank, const_cast<void*>(base), gd, gs,
                         bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -675,6 +789,19 @@ int32_t encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* d
     return MOHGE_ERR_CUDA;
   }
   return MOHGE_OK;
+}
+
+// [cols, rows] BF16 region with a row pitch in bytes, as 32-row x 64-column staging boxes
+int32_t encode_stage_map(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes) {
+  const uint64_t dims[2] = {cols, rows}, str[1] = {pitch_bytes};
+  const uint32_t box[2] = {64, 32};
+  return encode_map(m, base, 2, dims, str, box);
+}
+// [cols, rows, experts] FP32 weight-gradient tensor as 32 x 32 staging boxes
+int32_t encode_stage_map_f32(CUtensorMap* m, const void* base, uint64_t cols, uint64_t rows, uint64_t n) {
+  const uint64_t dims[3] = {cols, rows, n}, str[2] = {cols * 4, cols * rows * 4};
+  const uint32_t box[3] = {32, 32, 1};
+  return encode_map(m, base, 3, dims, str, box, true);
 }
 
 // Tile width per group: among the candidates the one that wastes the fewest padded columns
@@ -829,13 +956,11 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
 
   const uint64_t d = D.d, rows = D.Rcap, pitchAU = 2ull * D.Wmax * 2, pitchH = (uint64_t)D.Wmax * 2;
   const int CG = cta_group_size();
-  // UMMA N candidates.  A CTA pair splits B in halves, and an MN-major half must stay a multiple
-  // of the 64-element swizzle block, so N = 192 is only available to the single-CTA form.
-  const int cand_n1[3] = {256, 192, 128};
-  const int cand_n2[2] = {256, 128};
-  const int* cand_n = CG == 2 ? cand_n2 : cand_n1;
-  const int ncand = CG == 2 ? 2 : 3;
-  const int cand_h[3] = {128, 96, 64};
+  // UMMA N candidates: multiples of 128 so that a CTA pair's half of an MN-major B stays a
+  // multiple of the 64-element swizzle block and the epilogue's 64-column boxes tile the width.
+  const int cand_n[2] = {256, 128};
+  const int ncand = 2;
+  const int cand_h[2] = {128, 64};
   int bn_plan[MOHGE_MAX_GROUPS];
   int32_t rc = MOHGE_OK;
   for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) { p.BN[g] = 128; bn_plan[g] = 128; }
@@ -845,7 +970,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
     uint32_t box[3];
     switch (role) {
       case ROLE_FWD1: {
-        const int half = pick_bn(D.W[g], cand_h, CG == 2 ? 1 : 3) ;
+        const int half = pick_bn(D.W[g], cand_h, CG == 2 ? 1 : 2);
         p.BN[g] = 2 * half; bn_plan[g] = half;
         dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
@@ -853,6 +978,12 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         dims[0] = d; dims[1] = W; dims[2] = 2 * N; str[0] = d * 2; str[1] = W * d * 2;
         box[0] = BK; box[1] = half; box[2] = 1;
         rc = encode_map(&p.mapB[g], P.w13[g], 3, dims, str, box);
+        if (rc) break;
+        rc = encode_stage_map(&p.mapO[0][g], C, W, rows, pitchAU);
+        if (rc) break;
+        rc = encode_stage_map(&p.mapO[1][g], (const char*)C + W * 2, W, rows, pitchAU);
+        if (rc) break;
+        rc = encode_stage_map(&p.mapO[2][g], C2, W, rows, pitchH);
       } break;
       case ROLE_FWD2: {
         p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
@@ -862,6 +993,8 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         dims[0] = W; dims[1] = d; dims[2] = N; str[0] = W * 2; str[1] = d * W * 2;
         box[0] = BK; box[1] = p.BN[g] / CG; box[2] = 1;
         rc = encode_map(&p.mapB[g], P.w2[g], 3, dims, str, box);
+        if (rc || g > 0) break;
+        rc = encode_stage_map(&p.mapO[0][0], C, d, rows, d * 2);
       } break;
       case ROLE_DGRAD_DOWN: {
         p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
@@ -872,6 +1005,14 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         dims[0] = W; dims[1] = d; dims[2] = N; str[0] = W * 2; str[1] = d * W * 2;
         box[0] = 64; box[1] = BK; box[2] = 1;
         rc = encode_map(&p.mapB[g], P.w2[g], 3, dims, str, box);
+        if (rc) break;
+        rc = encode_stage_map(&p.mapE[0][g], B, W, rows, pitchAU);
+        if (rc) break;
+        rc = encode_stage_map(&p.mapE[1][g], (const char*)B + W * 2, W, rows, pitchAU);
+        if (rc) break;
+        rc = encode_stage_map(&p.mapO[0][g], C, W, rows, pitchAU);
+        if (rc) break;
+        rc = encode_stage_map(&p.mapO[1][g], (const char*)C + W * 2, W, rows, pitchAU);
       } break;
       case ROLE_DGRAD_13: {
         p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
@@ -881,6 +1022,8 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         dims[0] = d; dims[1] = 2 * W; dims[2] = N; str[0] = d * 2; str[1] = 2 * W * d * 2;
         box[0] = 64; box[1] = BK; box[2] = 1;
         rc = encode_map(&p.mapB[g], P.w13[g], 3, dims, str, box);
+        if (rc || g > 0) break;
+        rc = encode_stage_map(&p.mapO[0][0], C, d, rows, d * 2);
       } break;
       case ROLE_WGRAD_DOWN: {
         p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
@@ -889,6 +1032,8 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         if (rc) break;
         dims[0] = W; dims[1] = rows; str[0] = pitchH; box[0] = 64; box[1] = BK;
         rc = encode_map(&p.mapB[g], B, 2, dims, str, box);
+        if (rc) break;
+        rc = encode_stage_map_f32(&p.mapO[0][g], P.dw2[g], W, d, N);
       } break;
       default: {  // ROLE_WGRAD_13
         p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
@@ -897,6 +1042,8 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         if (rc) break;
         dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = 64; box[1] = BK;
         rc = encode_map(&p.mapB[g], B, 2, dims, str, box);
+        if (rc) break;
+        rc = encode_stage_map_f32(&p.mapO[0][g], P.dw13[g], d, 2 * W, N);
       } break;
     }
   }
