@@ -157,14 +157,33 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
-// ---- TMA stores from the epilogue staging buffers (bulk async-groups, one per store)
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+// L2 eviction priorities.  Epilogue outputs are written once and not read again by the same
+// launch, so they are marked evict-first: left at normal priority they push the operand tiles,
+// which every CTA of a wave re-reads, out of L2.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
-  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
-               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
+// ---- TMA stores from the epilogue staging buffers (bulk async-groups)
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1, uint64_t pol) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, uint64_t pol) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(pol) : "memory");
 }
 // element-wise FP32 add into global memory (each output element is touched by exactly one box)
 __device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
@@ -280,6 +299,12 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes,
   return (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
          ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
+
+// sigmoid and silu from the hardware exp2 and reciprocal approximations (about 2 ulp each):
+// the epilogue warps run one per scheduler with nothing to hide latency behind, so the IEEE
+// division sequence would cost more than the tile's MMAs.  exp overflow gives 1/inf = 0.
+__device__ __forceinline__ float sigmoid_fast(float a) { return __fdividef(1.0f, 1.0f + __expf(-a)); }
+__device__ __forceinline__ float silu_fast(float a) { return __fdividef(a, 1.0f + __expf(-a)); }
 
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -508,6 +533,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     const uint32_t stg = stg0 + (uint32_t)quad * (kStgBufs * kStgBufBytes);   // this warp's staging ring
     uint32_t n_store = 0;                      // stores issued so far: ring slot = n_store % 4
     uint32_t n_chunk = 0;                      // SwiGLU backward: input chunks consumed so far
+    const uint64_t pol_stream = l2_policy_evict_first();
     int buf = 0;
     uint32_t acc_phase = 0;
     bool alive = true;
@@ -526,8 +552,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           bulk_wait_read<0>();
           const uint32_t set = n_chunk & 1u, bar = ein_bar(quad, set);
           mbar_expect_tx(bar, 2 * kStgBufBytes);
-          tma_load_2d(stg + set * 2 * kStgBufBytes, &p.mapE[0][q.g], bar, q.n0, row0);
-          tma_load_2d(stg + (set * 2 + 1) * kStgBufBytes, &p.mapE[1][q.g], bar, q.n0, row0);
+          tma_load_2d_hint(stg + set * 2 * kStgBufBytes, &p.mapE[0][q.g], bar, q.n0, row0, pol_stream);
+          tma_load_2d_hint(stg + (set * 2 + 1) * kStgBufBytes, &p.mapE[1][q.g], bar, q.n0, row0, pol_stream);
         }
       }
       // the whole warp must agree before the warp-collective tensor-memory loads
@@ -557,7 +583,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               for (int e2 = 0; e2 < 4; ++e2) {
                 const float a0 = __uint_as_float(ra[j4 * 8 + 2 * e2]), a1 = __uint_as_float(ra[j4 * 8 + 2 * e2 + 1]);
                 const float u0 = __uint_as_float(ru[j4 * 8 + 2 * e2]), u1 = __uint_as_float(ru[j4 * 8 + 2 * e2 + 1]);
-                const float h0 = a0 / (1.0f + __expf(-a0)) * u0, h1 = a1 / (1.0f + __expf(-a1)) * u1;
+                const float h0 = silu_fast(a0) * u0, h1 = silu_fast(a1) * u1;
                 pa[e2] = pack2(a0, a1); pu[e2] = pack2(u0, u1); ph[e2] = pack2(h0, h1);
               }
               st_shared_v4(stg_addr(bA, lane, hh * 4 + j4), pa[0], pa[1], pa[2], pa[3]);
@@ -568,9 +594,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            tma_store_2d(&p.mapO[0][q.g], bA, q.n0 + c, row0); bulk_commit();
-            tma_store_2d(&p.mapO[1][q.g], bU, q.n0 + c, row0); bulk_commit();
-            tma_store_2d(&p.mapO[2][q.g], bH, q.n0 + c, row0); bulk_commit();
+            tma_store_2d(&p.mapO[0][q.g], bA, q.n0 + c, row0, pol_stream); bulk_commit();
+            tma_store_2d(&p.mapO[1][q.g], bU, q.n0 + c, row0, pol_stream); bulk_commit();
+            tma_store_2d(&p.mapO[2][q.g], bH, q.n0 + c, row0, pol_stream); bulk_commit();
           }
         }
       } else if (RT::EPI == EPI_BF16) {
@@ -598,7 +624,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           }
           fence_async_smem();
           __syncwarp();
-          if (lane == 0) { tma_store_2d(&p.mapO[0][0], bO, q.n0 + c, row0); bulk_commit(); }
+          if (lane == 0) { tma_store_2d(&p.mapO[0][0], bO, q.n0 + c, row0, pol_stream); bulk_commit(); }
         }
       } else if (RT::EPI == EPI_SWIGLU_BWD) {
         // per 64-column chunk: A and U arrive by TMA in one of two buffer pairs, dA and dU are
@@ -610,8 +636,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             bulk_wait_read<0>();                       // the other pair's last stores have left
             const uint32_t bar = ein_bar(quad, set ^ 1u);
             mbar_expect_tx(bar, 2 * kStgBufBytes);
-            tma_load_2d(stg + (set ^ 1u) * 2 * kStgBufBytes, &p.mapE[0][q.g], bar, q.n0 + c + 64, row0);
-            tma_load_2d(stg + ((set ^ 1u) * 2 + 1) * kStgBufBytes, &p.mapE[1][q.g], bar, q.n0 + c + 64, row0);
+            tma_load_2d_hint(stg + (set ^ 1u) * 2 * kStgBufBytes, &p.mapE[0][q.g], bar, q.n0 + c + 64, row0, pol_stream);
+            tma_load_2d_hint(stg + ((set ^ 1u) * 2 + 1) * kStgBufBytes, &p.mapE[1][q.g], bar, q.n0 + c + 64, row0, pol_stream);
           }
           const bool in_ok = mbar_wait(ein_bar(quad, set), (n_chunk >> 1) & 1u, abort_flag, p.status, 5);
           if (!__all_sync(0xffffffffu, in_ok)) { alive = false; break; }
@@ -631,7 +657,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               for (int e2 = 0; e2 < 4; ++e2) {
                 const float a0 = bf_lo(wa[e2]), a1 = bf_hi(wa[e2]), u0 = bf_lo(wu[e2]), u1 = bf_hi(wu[e2]);
                 const float dh0 = __uint_as_float(r[j4 * 8 + 2 * e2]), dh1 = __uint_as_float(r[j4 * 8 + 2 * e2 + 1]);
-                const float s0 = 1.0f / (1.0f + __expf(-a0)), s1 = 1.0f / (1.0f + __expf(-a1));
+                const float s0 = sigmoid_fast(a0), s1 = sigmoid_fast(a1);
                 oa[e2] = pack2(dh0 * u0 * s0 * (1.0f + a0 * (1.0f - s0)), dh1 * u1 * s1 * (1.0f + a1 * (1.0f - s1)));
                 ou[e2] = pack2(dh0 * a0 * s0, dh1 * a1 * s1);
               }
@@ -642,8 +668,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            tma_store_2d(&p.mapO[0][q.g], bA, q.n0 + c, row0);
-            tma_store_2d(&p.mapO[1][q.g], bU, q.n0 + c, row0);
+            tma_store_2d(&p.mapO[0][q.g], bA, q.n0 + c, row0, pol_stream);
+            tma_store_2d(&p.mapO[1][q.g], bU, q.n0 + c, row0, pol_stream);
             bulk_commit();
           }
         }
@@ -667,7 +693,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           __syncwarp();
           if (lane == 0) {
             if (p.accumulate) tma_reduce_add_3d(&p.mapO[0][q.g], bO, q.n0 + c, row0, q.i);
-            else tma_store_3d(&p.mapO[0][q.g], bO, q.n0 + c, row0, q.i);
+            else tma_store_3d(&p.mapO[0][q.g], bO, q.n0 + c, row0, q.i, pol_stream);
             bulk_commit();
           }
         }
