@@ -83,6 +83,10 @@ struct TcParams {
   GroupShape gs;
   GroupPtrs gp;
   int BN[MOHGE_MAX_GROUPS];      // UMMA N per group (FWD1: gate half + up half)
+  // MN-major operands whose MN extent is a multiple of 64 are mapped with one more dimension
+  // (64 elements, k rows, 64-element blocks[, expert]) so that ONE box brings all the 8 KiB
+  // swizzle blocks of a stage; otherwise each block is a box of its own
+  unsigned char a_blk[MOHGE_MAX_GROUPS], b_blk[MOHGE_MAX_GROUPS];
   const int32_t* aligned;
   const int32_t* tile_count;
   const Tile* tiles;
@@ -243,6 +247,20 @@ __device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* ma
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+template <int CG>
+__device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  if (CG == 2) tma2_load_4d(dst, map, bar, c0, c1, c2, c3); else tma_load_4d(dst, map, bar, c0, c1, c2, c3);
+}
 template <int CG>
 __device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
   if (CG == 2) tma2_load_2d(dst, map, bar, c0, c1); else tma_load_2d(dst, map, bar, c0, c1);
@@ -337,6 +355,16 @@ __device__ __forceinline__ void load_row32(const __nv_bfloat16* p, float (&v)[32
     v[q * 8 + 4] = bf_lo(o.z); v[q * 8 + 5] = bf_hi(o.z);
     v[q * 8 + 6] = bf_lo(o.w); v[q * 8 + 7] = bf_hi(o.w);
   }
+}
+
+// Epilogue pacing.  A tile's output leaves while the MMAs of the CTA's next tile run; sent as
+// one burst it delays that tile's operand loads (both share the SM's path to L2) by about as
+// long as the burst lasts.  The store-heavy roles therefore spread their chunks over
+// kPacePct % of the next tile's MMA time (512 clocks per 64-deep k-block at full rate).
+constexpr int kPacePct = 75;
+__device__ __forceinline__ void pace(long long t0, int i, int n, int next_num_kb) {
+  const long long target = t0 + (long long)next_num_kb * (512 * kPacePct / 100) * i / n;
+  while (clock64() < target) __nanosleep(64);
 }
 
 struct TileGeom {
@@ -460,8 +488,12 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           if (CG == 2) mbar_expect_tx_cluster(fb, tx); else mbar_expect_tx(fb, tx);
           const int k0 = kb * BK;
           if (RT::A_MN) {
-            tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0);
-            tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0);
+            if (p.a_blk[q.g]) {
+              tma_3d<CG>(sA, mA, fb, 0, q.r0 + k0, am0 >> 6);
+            } else {
+              tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0);
+              tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0);
+            }
           } else {
             tma_2d<CG>(sA, mA, fb, k0, am0);
           }
@@ -478,9 +510,11 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           } else if (ROLE == ROLE_FWD2) {
             tma_3d<CG>(sB, mB, fb, k0, bn0, q.i);
           } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
-            for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i);
+            if (p.b_blk[q.g]) tma_4d<CG>(sB, mB, fb, 0, k0, bn0 >> 6, q.i);
+            else for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i);
           } else {
-            for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0);
+            if (p.b_blk[q.g]) tma_3d<CG>(sB, mB, fb, 0, q.r0 + k0, bn0 >> 6);
+            else for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -562,6 +596,11 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kAccCols;
       const long long d = p.gs.d;
+      // pacing reference: now, and the k-blocks of the tile whose MMAs overlap this epilogue
+      const long long t_epi = clock64();
+      int next_kb = 0;
+      if ((RT::EPI == EPI_BF16 || RT::EPI == EPI_F32) && ti + unit_stride < total)
+        next_kb = tile_geom<ROLE>(p, fetch_tile<ROLE>(p, ti + unit_stride)).num_kb;
       if (RT::EPI == EPI_SWIGLU_FWD) {
         const int half = q.bn >> 1;
         for (int c = 0; rows_ok && c < half && q.n0 + c < q.W; c += 64) {
@@ -601,6 +640,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         }
       } else if (RT::EPI == EPI_BF16) {
         for (int c = 0; rows_ok && c < q.bn && q.n0 + c < (int)d; c += 64) {
+          pace(t_epi, c, q.bn, next_kb);
           if (lane == 0) bulk_wait_read<3>();
           __syncwarp();
           const uint32_t bO = stg + ((n_store & 3u) << 12);
@@ -679,6 +719,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         const int Mext = ROLE == ROLE_WGRAD_DOWN ? (int)d : 2 * q.W;
         const int Next = ROLE == ROLE_WGRAD_DOWN ? q.W : (int)d;
         for (int c = 0; row0 < Mext && c < q.bn && q.n0 + c < Next; c += 32) {
+          pace(t_epi, c, q.bn, next_kb);
           if (lane == 0) bulk_wait_read<3>();
           __syncwarp();
           const uint32_t bO = stg + ((n_store & 3u) << 12);
@@ -815,6 +856,28 @@ int32_t encode_map(CUtensorMap* m, const void* base, int rank, const uint64_t* d
     return MOHGE_ERR_CUDA;
   }
   return MOHGE_OK;
+}
+
+// MN-major operand [k_rows, mn] (mn contiguous, row pitch in bytes), optionally one matrix per
+// expert.  `blocks` = 64-element swizzle blocks one stage needs.  When mn is a multiple of 64
+// the blocks become a dimension and one box covers them all (*blocked = 1).
+int32_t encode_mn_map(CUtensorMap* m, const void* base, uint64_t mn, uint64_t k_rows, uint64_t pitch_bytes,
+                      uint64_t n_experts, uint64_t expert_stride_bytes, int blocks, unsigned char* blocked) {
+  uint64_t dims[4], str[3];
+  uint32_t box[4];
+  if (mn % 64 == 0) {
+    *blocked = 1;
+    dims[0] = 64; dims[1] = k_rows; dims[2] = mn / 64; str[0] = pitch_bytes; str[1] = 128;
+    box[0] = 64; box[1] = BK; box[2] = (uint32_t)blocks;
+    if (n_experts == 0) return encode_map(m, base, 3, dims, str, box);
+    dims[3] = n_experts; str[2] = expert_stride_bytes; box[3] = 1;
+    return encode_map(m, base, 4, dims, str, box);
+  }
+  *blocked = 0;
+  dims[0] = mn; dims[1] = k_rows; str[0] = pitch_bytes; box[0] = 64; box[1] = BK;
+  if (n_experts == 0) return encode_map(m, base, 2, dims, str, box);
+  dims[2] = n_experts; str[1] = expert_stride_bytes; box[2] = 1;
+  return encode_map(m, base, 3, dims, str, box);
 }
 
 // [cols, rows] BF16 region with a row pitch in bytes, as 32-row x 64-column staging boxes
@@ -1028,9 +1091,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
         if (rc) break;
-        dims[0] = W; dims[1] = d; dims[2] = N; str[0] = W * 2; str[1] = d * W * 2;
-        box[0] = 64; box[1] = BK; box[2] = 1;
-        rc = encode_map(&p.mapB[g], P.w2[g], 3, dims, str, box);
+        rc = encode_mn_map(&p.mapB[g], P.w2[g], W, d, W * 2, N, d * W * 2, p.BN[g] / CG / 64, &p.b_blk[g]);
         if (rc) break;
         rc = encode_stage_map(&p.mapE[0][g], B, W, rows, pitchAU);
         if (rc) break;
@@ -1045,29 +1106,23 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         dims[0] = 2 * W; dims[1] = rows; str[0] = pitchAU; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
         if (rc) break;
-        dims[0] = d; dims[1] = 2 * W; dims[2] = N; str[0] = d * 2; str[1] = 2 * W * d * 2;
-        box[0] = 64; box[1] = BK; box[2] = 1;
-        rc = encode_map(&p.mapB[g], P.w13[g], 3, dims, str, box);
+        rc = encode_mn_map(&p.mapB[g], P.w13[g], d, 2 * W, d * 2, N, 2 * W * d * 2, p.BN[g] / CG / 64, &p.b_blk[g]);
         if (rc || g > 0) break;
         rc = encode_stage_map(&p.mapO[0][0], C, d, rows, d * 2);
       } break;
       case ROLE_WGRAD_DOWN: {
         p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
-        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = 64; box[1] = BK;
-        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        rc = encode_mn_map(&p.mapA[g], A, d, rows, d * 2, 0, 0, 2, &p.a_blk[g]);
         if (rc) break;
-        dims[0] = W; dims[1] = rows; str[0] = pitchH; box[0] = 64; box[1] = BK;
-        rc = encode_map(&p.mapB[g], B, 2, dims, str, box);
+        rc = encode_mn_map(&p.mapB[g], B, W, rows, pitchH, 0, 0, p.BN[g] / CG / 64, &p.b_blk[g]);
         if (rc) break;
         rc = encode_stage_map_f32(&p.mapO[0][g], P.dw2[g], W, d, N);
       } break;
       default: {  // ROLE_WGRAD_13
         p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
-        dims[0] = 2 * W; dims[1] = rows; str[0] = pitchAU; box[0] = 64; box[1] = BK;
-        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        rc = encode_mn_map(&p.mapA[g], A, 2 * W, rows, pitchAU, 0, 0, 2, &p.a_blk[g]);
         if (rc) break;
-        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = 64; box[1] = BK;
-        rc = encode_map(&p.mapB[g], B, 2, dims, str, box);
+        rc = encode_mn_map(&p.mapB[g], B, d, rows, d * 2, 0, 0, p.BN[g] / CG / 64, &p.b_blk[g]);
         if (rc) break;
         rc = encode_stage_map_f32(&p.mapO[0][g], P.dw13[g], d, 2 * W, N);
       } break;
