@@ -14,6 +14,8 @@ namespace mohge {
 
 namespace {
 
+constexpr int kBandTiles = 8;
+
 __global__ void __launch_bounds__(256)
 build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
                    Tile* __restrict__ tiles, long long cap, int32_t* status) {
@@ -70,8 +72,16 @@ build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __r
     const int ex = s_order[lo];
     const int gg = ex / p.N;
     const int local = i - s_start[lo];
+    // Order inside an expert: bands of kBandTiles m-tiles; inside a band m runs fastest, then n.
+    // The CTAs of a wave then work on a near-square block of the output, so the A rows and the
+    // B rows they share are both few enough to stay in L2 while the wave needs them (a full
+    // column of m-tiles of a large expert would have to survive several waves to be reused).
     const int mt = s_mt[ex];
-    const int tm = local % mt, tn = local / mt;   // m fastest: neighbours share the B operand
+    const int nt = s_nt[ex] / mt;
+    const int band = local / (kBandTiles * nt);
+    const int in_band = local - band * kBandTiles * nt;
+    const int band_m = mt - band * kBandTiles < kBandTiles ? mt - band * kBandTiles : kBandTiles;
+    const int tm = band * kBandTiles + in_band % band_m, tn = in_band / band_m;
     Tile t;
     t.e = ex;
     t.n0 = tn * p.BN[gg];
