@@ -30,6 +30,11 @@ import torch  # noqa: E402
 
 from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs  # noqa: E402
 
+# DRAM bytes (read + written) of the six grouped-GEMM launches of one step, from the 1-pass ncu
+# capture summarised in profiles/launch_list_layer_step_cfg5.md; workloads without a capture of
+# the current kernels report null.
+NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 68.4e9}
+
 METRIC = "MoHGE layer fwd+bwd tokens/s"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg5_bf16_large"
@@ -344,7 +349,8 @@ def main():
     flops = flops_per_step(wl, counts)
     achieved = flops / (gemm_ms_step * 1e-3) / 1e12
     roofline = {"bound": "tensor", "achieved": achieved, "peak": pk["tf_sustained"], "unit": "TFLOP/s",
-                "frac": achieved / pk["tf_sustained"], "traffic": None,
+                "frac": achieved / pk["tf_sustained"], "traffic": NCU_DRAM_TRAFFIC_PER_STEP.get(wl.name),
+                "traffic_unit": "bytes of DRAM traffic per step (six launches)",
                 "kernel": "tc_grouped_kernel (6 launches per step: fwd1, fwd2, dgrad x2, wgrad x2)",
                 "of": pk["source"], "flops_per_step": flops, "gemm_ms_per_step": gemm_ms_step,
                 "frac_of_nominal_2250": achieved / 2250.0}

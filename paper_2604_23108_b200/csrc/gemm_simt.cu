@@ -56,14 +56,15 @@ build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __r
     }
     s_start[p.Ne] = run;
     if (run > cap) {
-      atomicCAS(status, 0, (2 << 24) | 2);
+      if (blockIdx.x == 0) atomicCAS(status, 0, (2 << 24) | 2);
       s_start[p.Ne] = 0;
     }
-    *tile_count = s_start[p.Ne];
+    if (blockIdx.x == 0) *tile_count = s_start[p.Ne];
   }
   __syncthreads();
+  // every block has built the same per-expert table; the entries are written grid-strided
   const int total = s_start[p.Ne];
-  for (int i = threadIdx.x; i < total; i += blockDim.x) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
     int lo = 0, hi = p.Ne - 1;              // last rank whose start <= i
     while (lo < hi) {
       const int mid = (lo + hi + 1) >> 1;
@@ -322,7 +323,7 @@ GroupShape make_group_shape(const Dims& D) {
 
 int32_t launch_build_tiles_plan(const TilePlan& p, const int32_t* aligned, int32_t* tile_count,
                                 Tile* tiles, int64_t tiles_cap, int32_t* status, cudaStream_t st) {
-  build_tiles_kernel<<<1, 256, 0, st>>>(p, aligned, tile_count, tiles, (long long)tiles_cap, status);
+  build_tiles_kernel<<<32, 256, 0, st>>>(p, aligned, tile_count, tiles, (long long)tiles_cap, status);
   MOHGE_LAUNCH_CHECK("build_tiles_kernel");
   return MOHGE_OK;
 }
