@@ -56,6 +56,13 @@ WORKLOADS = {
                                (1536, 1024, 768, 384), 2, 6, zipf_beta=1.0),
     "cfg5_bf16_large": Workload("cfg5_bf16_large", "bf16", 65536, 4096, 4, 32,
                                 (2048, 1536, 1024, 512), 2, 8),
+    # Layer shapes of the paper's own 3B- and 14B-scale MoHGE models (App. A.2, architecture
+    # table): d = 1024, eight groups of distinct width, K_g = 3, K_e = 6, sequences of 4096
+    # tokens (four sequences per batch here; the paper does not state its micro-batch).
+    "paper_3b_layer": Workload("paper_3b_layer", "bf16", 16384, 1024, 8, 8,
+                               (384, 512, 640, 768, 896, 1024, 1152, 1280), 3, 6, seed=6),
+    "paper_14b_layer": Workload("paper_14b_layer", "bf16", 16384, 1024, 8, 16,
+                                (640, 768, 896, 1024, 1152, 1280, 1408, 1536), 3, 6, seed=7),
 }
 
 

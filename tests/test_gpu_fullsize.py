@@ -25,7 +25,7 @@ pytestmark = pytest.mark.gpu
 
 TOL = 2e-2
 FULL_ORACLE = {"cfg2_bf16": True, "cfg3_bf16_aux": True, "cfg4_bf16_skew": True,
-               "cfg5_bf16_large": False}
+               "cfg5_bf16_large": False, "paper_3b_layer": True, "paper_14b_layer": True}
 N_SAMPLE_TOKENS = 48
 
 
