@@ -373,13 +373,18 @@ def expert_backward(xe, w13_e, w2_e, A, U, H, dY):
 
 
 def layer_forward(cfg: OracleConfig, x, w_r, w13: List, w2: List, logit_bias=None,
-                  logits=None, mode="definition"):
+                  logits=None, mode="definition", shared=None):
     """Forward of the whole layer.
 
     y_t = sum over the K_e selected experts of ES_{g,i,t} * E_{g,i}(x_t)
     (appendix Eq. 15 with the gate of Eq. 6).  mode "definition": selection in
     fp64 (Eq. 2-6).  mode "spec": the integer selection comes from the float32
     contract, all real values are still evaluated in fp64 for that selection.
+    `shared` = (w13_s [2*W_s, d], w2_s [d, W_s]): the always-active shared experts of the
+    paper's models (App. A.2 lists N_s = 2 of them without an equation).  Reading: as in the
+    DeepSeek-V2 layer the baseline is adapted from, they are FFNs applied to every token and
+    added to the routed sum with no gate; N_s such FFNs of width W equal one FFN of width
+    N_s * W with the weights concatenated along the hidden axis, which is what is passed here.
     Returns a dict with every intermediate needed by tests and by the backward.
     """
     cfg.check()
@@ -412,8 +417,13 @@ def layer_forward(cfg: OracleConfig, x, w_r, w13: List, w2: List, logit_bias=Non
         A, U, H, Y = swiglu_ffn(x[t_idx], _as64(w13[g][i]), _as64(w2[g][i]))
         np.add.at(y, t_idx, r["gate"][t_idx, k_idx][:, None] * Y)
         per_expert[e] = dict(t=t_idx, k=k_idx, A=A, U=U, H=H, Y=Y)
+    shared_saved = None
+    if shared is not None:
+        A, U, H, Y = swiglu_ffn(x, _as64(shared[0]), _as64(shared[1]))
+        y = y + Y
+        shared_saved = dict(A=A, U=U, H=H, Y=Y)
     return dict(cfg=cfg, x=x, w_r=w_r, logits=logits, y=y, per_expert=per_expert,
-                stats=stats, **r)
+                stats=stats, shared=shared_saved, **r)
 
 
 def layer_loss(fwd, G):
@@ -421,7 +431,7 @@ def layer_loss(fwd, G):
     return float(np.sum(fwd["y"] * _as64(G))) + fwd["stats"]["L_G"] + fwd["stats"]["L_E"]
 
 
-def layer_backward(fwd, w13: List, w2: List, dy, with_aux=True, aux_counts=None):
+def layer_backward(fwd, w13: List, w2: List, dy, with_aux=True, aux_counts=None, shared=None):
     """Gradients of  <y, dy> (+ L_G + L_E when with_aux)  w.r.t. x, the router
     weight and every expert weight.  Top-k choices and the indicator counts
     f^G, f^E are piecewise constant and carry no gradient.
@@ -481,5 +491,14 @@ def layer_backward(fwd, w13: List, w2: List, dy, with_aux=True, aux_counts=None)
     dlogits = np.concatenate([dlG, dlE.reshape(T, N_e)], axis=1)
     dw_r = dlogits.T @ x
     dx_router = dlogits @ w_r
-    return dict(dx=dx + dx_router, dx_experts=dx, dx_router=dx_router, dw_r=dw_r,
-                dw13=dw13, dw2=dw2, dgate=dgate, dlogits=dlogits)
+    out = dict(dx_experts=dx, dx_router=dx_router, dw_r=dw_r, dw13=dw13, dw2=dw2, dgate=dgate,
+               dlogits=dlogits)
+    dx_total = dx + dx_router
+    if shared is not None:
+        # the shared FFN sees every token with unit gate: dY = dy
+        c = fwd["shared"]
+        sb = expert_backward(x, _as64(shared[0]), _as64(shared[1]), c["A"], c["U"], c["H"], dy)
+        dx_total = dx_total + sb["dx"]
+        out.update(shared=sb)
+    out["dx"] = dx_total
+    return out

@@ -172,3 +172,43 @@ def test_sampled_tokens_reproduce_full_batch_rows():
                           aux_counts=(f["stats"]["cG"], f["stats"]["cE_lit"], T))
     np.testing.assert_allclose(fs["y"], f["y"][samp], rtol=1e-13)
     np.testing.assert_allclose(bs["dx"], b["dx"][samp], rtol=1e-12, atol=1e-14)
+
+
+def test_shared_experts_add_an_ungated_dense_ffn_and_its_gradients():
+    # N_s shared FFNs of width W, weights concatenated along the hidden axis, applied to every
+    # token: autograd of (independent dense routed forward + three-line dense FFN) must agree
+    cfg = O.OracleConfig(d_model=10, n_groups=2, experts_per_group=3, k_groups=1, k_experts=2,
+                         group_width=[8, 12], alpha_g=0.7, alpha_e=0.9)
+    T, Ws, Ns = 30, 6, 2
+    x, w_r, w13, w2, dy = _rand_layer(cfg, T, 33)
+    rng = np.random.default_rng(34)
+    sh_g = [rng.normal(size=(Ws, 10)) * 0.3 for _ in range(Ns)]      # per shared expert
+    sh_u = [rng.normal(size=(Ws, 10)) * 0.3 for _ in range(Ns)]
+    sh_d = [rng.normal(size=(10, Ws)) * 0.3 for _ in range(Ns)]
+    w13_s = np.concatenate(sh_g + sh_u, axis=0)                       # [2 * Ns * Ws, d]
+    w2_s = np.concatenate(sh_d, axis=1)                               # [d, Ns * Ws]
+    f = O.layer_forward(cfg, x, w_r, w13, w2, shared=(w13_s, w2_s))
+    b = O.layer_backward(f, w13, w2, dy, shared=(w13_s, w2_s))
+    f0 = O.layer_forward(cfg, x, w_r, w13, w2)
+    # forward: the sum of the N_s separate FFNs
+    extra = sum((torch.nn.functional.silu(torch.tensor(x) @ torch.tensor(g_).T)
+                 * (torch.tensor(x) @ torch.tensor(u_).T)) @ torch.tensor(d_).T
+                for g_, u_, d_ in zip(sh_g, sh_u, sh_d)).numpy()
+    np.testing.assert_allclose(f["y"], f0["y"] + extra, rtol=1e-11, atol=1e-12)
+    # backward: autograd of routed + shared
+    tx = torch.tensor(x, requires_grad=True)
+    twr = torch.tensor(w_r, requires_grad=True)
+    tw13 = [torch.tensor(w, requires_grad=True) for w in w13]
+    tw2 = [torch.tensor(w, requires_grad=True) for w in w2]
+    t13s, t2s = torch.tensor(w13_s, requires_grad=True), torch.tensor(w2_s, requires_grad=True)
+    H = Ns * Ws
+    _, loss, _, _ = _torch_dense_forward(cfg, tx, twr, tw13, tw2, torch.tensor(dy))
+    ys = (torch.nn.functional.silu(tx @ t13s[:H].T) * (tx @ t13s[H:].T)) @ t2s.T
+    (loss + torch.sum(ys * torch.tensor(dy))).backward()
+    tol = dict(rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(b["dx"], tx.grad.numpy(), **tol)
+    np.testing.assert_allclose(b["dw_r"], twr.grad.numpy(), **tol)
+    np.testing.assert_allclose(b["shared"]["dw13"], t13s.grad.numpy(), **tol)
+    np.testing.assert_allclose(b["shared"]["dw2"], t2s.grad.numpy(), **tol)
+    for g in range(2):
+        np.testing.assert_allclose(b["dw13"][g], tw13[g].grad.numpy(), **tol)
