@@ -161,10 +161,11 @@ def replica_seed(wl: Workload, rank: int) -> int:
     return wl.seed + rank
 
 
-def flops_per_step(wl: Workload, counts) -> float:
-    """Algorithmic FLOPs of the six expert GEMMs: 18 * d * sum_e M_e * W_g(e) (fwd 6, bwd 12)."""
+def flops_per_step(wl: Workload, counts, shared_width: int = 0) -> float:
+    """Algorithmic FLOPs of the expert GEMMs: 18 * d * sum_e M_e * W_g(e) (fwd 6, bwd 12), plus
+    18 * d * T * shared_width when shared experts run."""
     N = wl.experts_per_group
-    tot = 0.0
+    tot = float(wl.T) * shared_width
     for e, m in enumerate(counts):
         tot += float(m) * wl.group_width[e // N]
     return 18.0 * wl.d_model * tot
@@ -180,6 +181,9 @@ def main():
     ap.add_argument("--ref-sample", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--shared-width", type=int, default=0,
+                    help="hidden width of the shared experts (N_s FFNs concatenated); 0 = none, "
+                         "the benchmark configurations have none")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
@@ -205,7 +209,11 @@ def main():
                     k_groups=wl.k_groups, k_experts=wl.k_experts, group_width=list(wl.group_width),
                     dtype=wl.dtype, row_align=128 if wl.dtype == "bf16" else 1)
     inp = make_device_inputs(wl, dev, seed=replica_seed(wl, rank))
-    buf = B.LayerBuffers(gcfg, wl.T, device=dev)
+    buf = B.LayerBuffers(gcfg, wl.T, device=dev, shared_width=args.shared_width)
+    shared = None
+    if args.shared_width:
+        from paper_2604_23108_b200.inputs import make_shared_weights
+        shared = make_shared_weights(wl, args.shared_width, device=dev, seed=replica_seed(wl, rank))
     T = wl.T
     ev = lambda: torch.cuda.Event(enable_timing=True)
     gemm_marks = []
@@ -222,19 +230,28 @@ def main():
             e0.record()
         B.mohge_expert_fwd(gcfg, T, buf.x_perm, buf.counts, buf.aligned, inp["w13"], inp["w2"],
                            buf.au, buf.h, buf.y_perm, buf.ws)
+        if shared is not None:
+            B.mohge_shared_fwd(gcfg, T, args.shared_width, inp["x"], shared[0], shared[1], buf.au_sh,
+                               buf.h_sh, buf.y_sh, buf.ws)
         if mark:
             e1.record()
-        B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, buf.y)
+        B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, buf.y,
+                        y_add=buf.y_sh if shared is not None else None)
         B.mohge_combine_bwd(gcfg, T, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.counts,
                             buf.aligned, buf.dy_perm, buf.dgate)
         if mark:
             e2.record()
         B.mohge_expert_bwd(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts, buf.aligned,
                            inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13, buf.dw2, 0, buf.ws)
+        if shared is not None:
+            B.mohge_shared_bwd(gcfg, T, args.shared_width, inp["dy"], inp["x"], buf.au_sh, buf.h_sh,
+                               shared[0], shared[1], buf.dau_sh, buf.dx_sh, buf.dw13_sh, buf.dw2_sh,
+                               0, buf.ws)
         if mark:
             e3.record()
             gemm_marks.append((e0, e1, e2, e3))
-        B.mohge_dispatch_bwd(gcfg, T, buf.dx_perm, buf.prow_of, buf.dx)
+        B.mohge_dispatch_bwd(gcfg, T, buf.dx_perm, buf.prow_of, buf.dx,
+                             dx_add=buf.dx_sh if shared is not None else None)
         cnt_e = buf.cnt_lit if gcfg.fe_mode == 0 else buf.cnt_routed
         B.mohge_route_bwd(gcfg, T, inp["x"], inp["w_router"], buf.dgate, buf.gs, buf.esp,
                           buf.group_idx, buf.expert_idx, buf.group_count, cnt_e, buf.dlogits,
@@ -346,7 +363,7 @@ def main():
         return
 
     pk = _peaks()
-    flops = flops_per_step(wl, counts)
+    flops = flops_per_step(wl, counts, args.shared_width)
     achieved = flops / (gemm_ms_step * 1e-3) / 1e12
     roofline = {"bound": "tensor", "achieved": achieved, "peak": pk["tf_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / pk["tf_sustained"], "traffic": NCU_DRAM_TRAFFIC_PER_STEP.get(wl.name),
@@ -373,7 +390,7 @@ def main():
         "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "T": T, "d_model": wl.d_model, "n_groups": wl.n_groups,
                    "experts_per_group": wl.experts_per_group, "group_width": list(wl.group_width),
-                   "k_groups": wl.k_groups, "k_experts": wl.k_experts,
+                   "k_groups": wl.k_groups, "k_experts": wl.k_experts, "shared_width": args.shared_width,
                    "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu_baseline,

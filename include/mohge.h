@@ -187,11 +187,14 @@ int32_t mohge_expert_fwd(const mohge_config* cfg, int64_t T, const void* x_perm,
                          void* h_saved, void* y_perm, void* ws, void* stream);
 
 /*
- * Weighted combine: y[t, :] = sum_k gate_w[t,k] * y_perm[prow_of[t,k], :]   (Eq. 15 with the
- * gate of Eq. 6), FP32 accumulation.   y [T, d] dtype.
+ * Weighted combine: y[t, :] = sum_k gate_w[t,k] * y_perm[prow_of[t,k], :] (+ y_add[t, :])
+ * (Eq. 15 with the gate of Eq. 6), FP32 accumulation.   y [T, d] dtype.
+ *   y_add [T, d] dtype, nullable: a term added to every token's output in the same pass, i.e.
+ *   the output of the shared experts (mohge_shared_fwd).
  */
 int32_t mohge_combine(const mohge_config* cfg, int64_t T, const void* y_perm,
-                      const int32_t* prow_of, const float* gate_w, void* y, void* stream);
+                      const int32_t* prow_of, const float* gate_w, const void* y_add, void* y,
+                      void* stream);
 
 /*
  * Backward of the combine:  dgate_w[t,k] = <dy[t], y_perm[prow_of[t,k]]>,
@@ -216,9 +219,42 @@ int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm
                          float* const* dw13, float* const* dw2, int32_t accumulate, void* ws,
                          void* stream);
 
-/* Backward of the permutation: dx[t, :] = sum_k dx_perm[prow_of[t,k], :].  dx [T, d] dtype. */
+/*
+ * Backward of the permutation: dx[t, :] = sum_k dx_perm[prow_of[t,k], :] (+ dx_add[t, :]).
+ *   dx [T, d] dtype;  dx_add [T, d] dtype, nullable (the shared experts' input gradient).
+ */
 int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,
-                           const int32_t* prow_of, void* dx, void* stream);
+                           const int32_t* prow_of, const void* dx_add, void* dx, void* stream);
+
+/*
+ * Shared experts (App. A.2 lists N_s = 2 shared experts per layer; the paper gives no equation
+ * for them).  Reading: as in the DeepSeek-V2 layer its baseline is adapted from, every token
+ * passes through them and their output is added to the routed sum with no gate.  N_s FFNs of
+ * width W are one SwiGLU FFN of hidden width shared_width = N_s * W with the weights
+ * concatenated along the hidden axis, which is the form taken here:
+ *   y_shared[t, :] = W_down( silu(W_gate x_t) * (W_up x_t) )
+ *   w13_shared [2*shared_width, d] dtype (gate rows, then up rows); w2_shared [d, shared_width]
+ *   au_shared [T, 2*shared_width] dtype, h_shared [T, shared_width] dtype: saved A | U and H
+ *   y_shared [T, d] dtype: pass it to mohge_combine as y_add.
+ * Runs on the grouped-expert kernels with x as a single segment (no permutation, no copy).
+ * `cfg` and `ws` are the layer's; shared_width must be a multiple of 8 and small enough for
+ * the workspace's tile list (any width up to K_e * W_max fits).
+ */
+int32_t mohge_shared_fwd(const mohge_config* cfg, int64_t T, int32_t shared_width, const void* x,
+                         const void* w13_shared, const void* w2_shared, void* au_shared,
+                         void* h_shared, void* y_shared, void* ws, void* stream);
+
+/*
+ * Backward of the shared experts for the upstream gradient dy [T, d] (unit gate):
+ *   dau_shared [T, 2*shared_width] dtype (dA | dU), dx_shared [T, d] dtype: pass it to
+ *   mohge_dispatch_bwd as dx_add;  dw13_shared [2*shared_width, d] float32,
+ *   dw2_shared [d, shared_width] float32; accumulate != 0 adds into the weight gradients.
+ */
+int32_t mohge_shared_bwd(const mohge_config* cfg, int64_t T, int32_t shared_width, const void* dy,
+                         const void* x, const void* au_shared, const void* h_shared,
+                         const void* w13_shared, const void* w2_shared, void* dau_shared,
+                         void* dx_shared, float* dw13_shared, float* dw2_shared,
+                         int32_t accumulate, void* ws, void* stream);
 
 /*
  * Router backward: dgate_w through Eq. 6, 4, 3, 2 (top-k choices carry no gradient) to the

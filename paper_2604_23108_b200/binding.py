@@ -47,11 +47,14 @@ _SIGS = {
     "mohge_aux_stats_static": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 11),
     "mohge_dispatch": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 11),
     "mohge_expert_fwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 10),
-    "mohge_combine": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 5),
+    "mohge_combine": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 6),
     "mohge_combine_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 9),
     "mohge_expert_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12
                          + [C.c_int32, _P, _P]),
-    "mohge_dispatch_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 4),
+    "mohge_dispatch_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 5),
+    "mohge_shared_fwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 8),
+    "mohge_shared_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 10
+                         + [C.c_int32, _P, _P]),
     "mohge_route_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 14),
 }
 
@@ -210,9 +213,9 @@ def mohge_expert_fwd(cfg, T, x_perm, counts, aligned_offsets, w13, w2, au_saved,
            "mohge_expert_fwd")
 
 
-def mohge_combine(cfg, T, y_perm, prow_of, gate_w, y):
+def mohge_combine(cfg, T, y_perm, prow_of, gate_w, y, y_add=None):
     _check(lib().mohge_combine(C.byref(cfg.c()), T, _ptr(y_perm), _ptr(prow_of), _ptr(gate_w),
-                               _ptr(y), _stream()), "mohge_combine")
+                               _ptr(y_add), _ptr(y), _stream()), "mohge_combine")
 
 
 def mohge_combine_bwd(cfg, T, dy, y_perm, prow_of, gate_w, counts, aligned_offsets, dy_perm, dgate_w):
@@ -231,9 +234,24 @@ def mohge_expert_bwd(cfg, T, dy_perm, x_perm, au_saved, h_saved, counts, aligned
                                   _stream()), "mohge_expert_bwd")
 
 
-def mohge_dispatch_bwd(cfg, T, dx_perm, prow_of, dx):
-    _check(lib().mohge_dispatch_bwd(C.byref(cfg.c()), T, _ptr(dx_perm), _ptr(prow_of), _ptr(dx),
-                                    _stream()), "mohge_dispatch_bwd")
+def mohge_dispatch_bwd(cfg, T, dx_perm, prow_of, dx, dx_add=None):
+    _check(lib().mohge_dispatch_bwd(C.byref(cfg.c()), T, _ptr(dx_perm), _ptr(prow_of),
+                                    _ptr(dx_add), _ptr(dx), _stream()), "mohge_dispatch_bwd")
+
+
+def mohge_shared_fwd(cfg, T, shared_width, x, w13_shared, w2_shared, au_shared, h_shared, y_shared, ws):
+    _check(lib().mohge_shared_fwd(C.byref(cfg.c()), T, int(shared_width), _ptr(x), _ptr(w13_shared),
+                                  _ptr(w2_shared), _ptr(au_shared), _ptr(h_shared), _ptr(y_shared),
+                                  _ptr(ws), _stream()), "mohge_shared_fwd")
+
+
+def mohge_shared_bwd(cfg, T, shared_width, dy, x, au_shared, h_shared, w13_shared, w2_shared,
+                     dau_shared, dx_shared, dw13_shared, dw2_shared, accumulate, ws):
+    _check(lib().mohge_shared_bwd(C.byref(cfg.c()), T, int(shared_width), _ptr(dy), _ptr(x),
+                                  _ptr(au_shared), _ptr(h_shared), _ptr(w13_shared),
+                                  _ptr(w2_shared), _ptr(dau_shared), _ptr(dx_shared),
+                                  _ptr(dw13_shared), _ptr(dw2_shared), int(accumulate), _ptr(ws),
+                                  _stream()), "mohge_shared_bwd")
 
 
 def mohge_route_bwd(cfg, T, x, w_router, dgate_w, gs_saved, esp_saved, group_idx, expert_idx,
@@ -247,8 +265,8 @@ def mohge_route_bwd(cfg, T, x, w_router, dgate_w, gs_saved, esp_saved, group_idx
 class LayerBuffers:
     """Device allocations for one layer step (torch is used for memory only)."""
 
-    def __init__(self, cfg: Config, T: int, device="cuda"):
-        self.cfg, self.T = cfg, T
+    def __init__(self, cfg: Config, T: int, device="cuda", shared_width: int = 0):
+        self.cfg, self.T, self.shared_width = cfg, T, shared_width
         dt, dev = cfg.torch_dtype, device
         Ne, NL, Ke, Kg, d = cfg.n_experts, cfg.n_logits, cfg.k_experts, cfg.k_groups, cfg.d_model
         Wmax = max(cfg.group_width)
@@ -276,12 +294,18 @@ class LayerBuffers:
         self.dw_router = e(NL, d, dtype=f32)
         self.dw13 = [e(cfg.experts_per_group, 2 * w, d, dtype=f32) for w in cfg.group_width]
         self.dw2 = [e(cfg.experts_per_group, d, w, dtype=f32) for w in cfg.group_width]
+        if shared_width:
+            Ws = shared_width
+            self.au_sh, self.h_sh, self.y_sh = e(Tn, 2 * Ws), e(Tn, Ws), e(Tn, d)
+            self.dau_sh, self.dx_sh = e(Tn, 2 * Ws), e(Tn, d)
+            self.dw13_sh, self.dw2_sh = e(2 * Ws, d, dtype=f32), e(d, Ws, dtype=f32)
         mohge_workspace_init(cfg, T, self.ws)
 
 
 def layer_forward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, logit_bias=None,
-                  logits_in=None, aux=True):
-    """route -> aux_stats -> dispatch -> expert_fwd -> combine; results stay in `b`."""
+                  logits_in=None, aux=True, shared=None):
+    """route -> aux_stats -> dispatch -> expert_fwd (-> shared_fwd) -> combine; results stay in
+    `b`.  shared = (w13_shared, w2_shared) adds the shared experts (b.shared_width wide)."""
     T = b.T
     mohge_route(cfg, T, x, w_router, logit_bias, logits_in, b.logits, b.group_idx, b.expert_idx,
                 b.gate_w, b.gs, b.esp, b.ws)
@@ -291,17 +315,25 @@ def layer_forward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, logit_bias
     mohge_dispatch(cfg, T, x, b.expert_idx, b.counts, b.offsets, b.aligned, b.row_of, b.prow_of,
                    b.src_of, b.x_perm, b.ws)
     mohge_expert_fwd(cfg, T, b.x_perm, b.counts, b.aligned, w13, w2, b.au, b.h, b.y_perm, b.ws)
-    mohge_combine(cfg, T, b.y_perm, b.prow_of, b.gate_w, b.y)
+    if shared is not None:
+        mohge_shared_fwd(cfg, T, b.shared_width, x, shared[0], shared[1], b.au_sh, b.h_sh, b.y_sh, b.ws)
+    mohge_combine(cfg, T, b.y_perm, b.prow_of, b.gate_w, b.y,
+                  y_add=b.y_sh if shared is not None else None)
     return b.y
 
 
-def layer_backward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, dy, aux=True, accumulate=False):
-    """combine_bwd -> expert_bwd -> dispatch_bwd -> route_bwd; results stay in `b`."""
+def layer_backward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, dy, aux=True, accumulate=False,
+                   shared=None):
+    """combine_bwd -> expert_bwd (-> shared_bwd) -> dispatch_bwd -> route_bwd; results stay in `b`."""
     T = b.T
     mohge_combine_bwd(cfg, T, dy, b.y_perm, b.prow_of, b.gate_w, b.counts, b.aligned, b.dy_perm, b.dgate)
     mohge_expert_bwd(cfg, T, b.dy_perm, b.x_perm, b.au, b.h, b.counts, b.aligned, w13, w2, b.dau,
                      b.dx_perm, b.dw13, b.dw2, accumulate, b.ws)
-    mohge_dispatch_bwd(cfg, T, b.dx_perm, b.prow_of, b.dx)
+    if shared is not None:
+        mohge_shared_bwd(cfg, T, b.shared_width, dy, x, b.au_sh, b.h_sh, shared[0], shared[1],
+                         b.dau_sh, b.dx_sh, b.dw13_sh, b.dw2_sh, accumulate, b.ws)
+    mohge_dispatch_bwd(cfg, T, b.dx_perm, b.prow_of, b.dx,
+                       dx_add=b.dx_sh if shared is not None else None)
     cnt_e = b.cnt_lit if cfg.fe_mode == 0 else b.cnt_routed
     mohge_route_bwd(cfg, T, x, w_router, b.dgate, b.gs, b.esp, b.group_idx, b.expert_idx,
                     b.group_count if aux else None, cnt_e if aux else None, b.dlogits, b.dx,

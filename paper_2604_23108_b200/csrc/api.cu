@@ -239,21 +239,13 @@ int32_t mohge_dispatch(const mohge_config* cfg, int64_t T, const void* x,
                          x_perm, w.hist, w.base, w.status, (cudaStream_t)stream);
 }
 
-int32_t mohge_expert_fwd(const mohge_config* cfg, int64_t T, const void* x_perm,
-                         const int32_t* counts, const int32_t* aligned_offsets,
-                         const void* const* w13, const void* const* w2, void* au_saved,
-                         void* h_saved, void* y_perm, void* ws, void* stream) {
-  Dims D;
-  int32_t rc = make_dims(cfg, T, &D);
-  if (rc) return rc;
-  REQ_PTR(x_perm); REQ_PTR(counts); REQ_PTR(aligned_offsets); REQ_PTR(au_saved); REQ_PTR(h_saved);
-  REQ_PTR(y_perm); REQ_PTR(ws);
-  MOHGE_CHECK_ARG(w13 && w2, "w13 and w2 must be host arrays of n_groups device pointers");
-  GroupPtrs P;
-  rc = group_ptrs(D, w13, w2, nullptr, nullptr, &P);
-  if (rc) return rc;
-  const Ws w = carve(D, ws);
-  cudaStream_t st = (cudaStream_t)stream;
+// Forward of the grouped SwiGLU experts for already validated arguments.  Shared by the routed
+// experts and by the shared experts (one segment of T rows).
+static int32_t expert_fwd_impl(const Dims& D, const GroupPtrs& P, const void* x_perm,
+                               const int32_t* counts, const int32_t* aligned_offsets,
+                               void* au_saved, void* h_saved, void* y_perm, const Ws& w,
+                               cudaStream_t st) {
+  int32_t rc;
   if (D.bf16 && !force_simt()) {
     MOHGE_CHECK_ARG(D.align == 128, "the BF16 tensor-core path needs row_align = 128");
     rc = launch_tc_grouped(D, ROLE_FWD1, P, x_perm, nullptr, au_saved, h_saved, counts,
@@ -277,13 +269,31 @@ int32_t mohge_expert_fwd(const mohge_config* cfg, int64_t T, const void* x_perm,
                              w.tile_count, w.tiles, st);
 }
 
-int32_t mohge_combine(const mohge_config* cfg, int64_t T, const void* y_perm,
-                      const int32_t* prow_of, const float* gate_w, void* y, void* stream) {
+int32_t mohge_expert_fwd(const mohge_config* cfg, int64_t T, const void* x_perm,
+                         const int32_t* counts, const int32_t* aligned_offsets,
+                         const void* const* w13, const void* const* w2, void* au_saved,
+                         void* h_saved, void* y_perm, void* ws, void* stream) {
   Dims D;
   int32_t rc = make_dims(cfg, T, &D);
   if (rc) return rc;
-  REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(y);
-  return launch_combine(D, y_perm, prow_of, gate_w, y, (cudaStream_t)stream);
+  REQ_PTR(x_perm); REQ_PTR(counts); REQ_PTR(aligned_offsets); REQ_PTR(au_saved); REQ_PTR(h_saved);
+  REQ_PTR(y_perm); REQ_PTR(ws);
+  MOHGE_CHECK_ARG(w13 && w2, "w13 and w2 must be host arrays of n_groups device pointers");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, nullptr, nullptr, &P);
+  if (rc) return rc;
+  return expert_fwd_impl(D, P, x_perm, counts, aligned_offsets, au_saved, h_saved, y_perm,
+                         carve(D, ws), (cudaStream_t)stream);
+}
+
+int32_t mohge_combine(const mohge_config* cfg, int64_t T, const void* y_perm,
+                      const int32_t* prow_of, const float* gate_w, const void* y_add, void* y,
+                      void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(y); OPT_PTR(y_add);
+  return launch_combine(D, y_perm, prow_of, gate_w, y_add, y, (cudaStream_t)stream);
 }
 
 int32_t mohge_combine_bwd(const mohge_config* cfg, int64_t T, const void* dy, const void* y_perm,
@@ -299,23 +309,12 @@ int32_t mohge_combine_bwd(const mohge_config* cfg, int64_t T, const void* dy, co
                             dgate_w, (cudaStream_t)stream);
 }
 
-int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm,
-                         const void* x_perm, const void* au_saved, const void* h_saved,
-                         const int32_t* counts, const int32_t* aligned_offsets,
-                         const void* const* w13, const void* const* w2, void* dau, void* dx_perm,
-                         float* const* dw13, float* const* dw2, int32_t accumulate, void* ws,
-                         void* stream) {
-  Dims D;
-  int32_t rc = make_dims(cfg, T, &D);
-  if (rc) return rc;
-  REQ_PTR(dy_perm); REQ_PTR(x_perm); REQ_PTR(au_saved); REQ_PTR(h_saved); REQ_PTR(counts);
-  REQ_PTR(aligned_offsets); REQ_PTR(dau); REQ_PTR(dx_perm); REQ_PTR(ws);
-  MOHGE_CHECK_ARG(w13 && w2 && dw13 && dw2, "w13, w2, dw13, dw2 must be host arrays of n_groups device pointers");
-  GroupPtrs P;
-  rc = group_ptrs(D, w13, w2, dw13, dw2, &P);
-  if (rc) return rc;
-  const Ws w = carve(D, ws);
-  cudaStream_t st = (cudaStream_t)stream;
+// Backward of the grouped SwiGLU experts for already validated arguments (see expert_fwd_impl).
+static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy_perm,
+                               const void* x_perm, const void* au_saved, const void* h_saved,
+                               const int32_t* counts, const int32_t* aligned_offsets, void* dau,
+                               void* dx_perm, int32_t accumulate, const Ws& w, cudaStream_t st) {
+  int32_t rc;
   if (!accumulate) {
     rc = launch_zero_empty_wgrad(D, P, counts, st);
     if (rc) return rc;
@@ -357,13 +356,110 @@ int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm
   return MOHGE_OK;
 }
 
-int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,
-                           const int32_t* prow_of, void* dx, void* stream) {
+
+int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm,
+                         const void* x_perm, const void* au_saved, const void* h_saved,
+                         const int32_t* counts, const int32_t* aligned_offsets,
+                         const void* const* w13, const void* const* w2, void* dau, void* dx_perm,
+                         float* const* dw13, float* const* dw2, int32_t accumulate, void* ws,
+                         void* stream) {
   Dims D;
   int32_t rc = make_dims(cfg, T, &D);
   if (rc) return rc;
-  REQ_PTR(dx_perm); REQ_PTR(prow_of); REQ_PTR(dx);
-  return launch_unpermute_sum(D, dx_perm, prow_of, dx, (cudaStream_t)stream);
+  REQ_PTR(dy_perm); REQ_PTR(x_perm); REQ_PTR(au_saved); REQ_PTR(h_saved); REQ_PTR(counts);
+  REQ_PTR(aligned_offsets); REQ_PTR(dau); REQ_PTR(dx_perm); REQ_PTR(ws);
+  MOHGE_CHECK_ARG(w13 && w2 && dw13 && dw2, "w13, w2, dw13, dw2 must be host arrays of n_groups device pointers");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, dw13, dw2, &P);
+  if (rc) return rc;
+  return expert_bwd_impl(D, P, dy_perm, x_perm, au_saved, h_saved, counts, aligned_offsets, dau,
+                         dx_perm, accumulate, carve(D, ws), (cudaStream_t)stream);
+}
+
+int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,
+                           const int32_t* prow_of, const void* dx_add, void* dx, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(dx_perm); REQ_PTR(prow_of); REQ_PTR(dx); OPT_PTR(dx_add);
+  return launch_unpermute_sum(D, dx_perm, prow_of, dx_add, dx, (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------- shared experts
+// The shared experts are one dense SwiGLU FFN over all T tokens.  They run through the grouped
+// kernels as a single group with a single expert whose segment is x itself: the segment table
+// {0, T rounded up to row_align} and the count {T} live in the workspace header, and the
+// tensor maps end at row T, so tiles that reach past T read zeros and store nothing.
+namespace {
+__global__ void shared_segment_kernel(int32_t* hdr, int T, int align) {
+  hdr[0] = 0;
+  hdr[1] = (T + align - 1) / align * align;
+  hdr[2] = T;
+}
+
+struct SharedCtx {
+  Dims Dm, Ds;          // the layer's dimensions (workspace layout) and the one-expert view
+  Ws w;
+  int32_t* aligned;     // {0, padded T}
+  int32_t* counts;      // {T}
+};
+
+int32_t shared_ctx(const mohge_config* cfg, int64_t T, int32_t width, void* ws, SharedCtx* c) {
+  int32_t rc = make_dims(cfg, T, &c->Dm);
+  if (rc) return rc;
+  MOHGE_CHECK_ARG(width >= 8 && width % 8 == 0, "shared_width = %d must be a positive multiple of 8", width);
+  MOHGE_CHECK_ARG(ws != nullptr && aligned16(ws), "ws must be a non-NULL 16-byte aligned device pointer");
+  mohge_config one = *cfg;
+  one.n_groups = 1; one.experts_per_group = 1; one.k_groups = 1; one.k_experts = 1;
+  for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) one.group_width[g] = g == 0 ? width : 0;
+  rc = make_dims(&one, T, &c->Ds);
+  if (rc) return rc;
+  c->Ds.Rcap = T > 0 ? T : 1;                       // rows that exist in x, dy and the saved tensors
+  c->w = carve(c->Dm, ws);
+  MOHGE_CHECK_ARG(ws_layout(c->Ds).tiles_cap <= c->w.tiles_cap,
+                  "shared_width = %d needs a larger tile list than this layer's workspace holds", width);
+  c->aligned = c->w.status + 16;                    // bytes 64..75 of the workspace header
+  c->counts = c->w.status + 18;
+  return MOHGE_OK;
+}
+}  // namespace
+
+int32_t mohge_shared_fwd(const mohge_config* cfg, int64_t T, int32_t shared_width, const void* x,
+                         const void* w13_shared, const void* w2_shared, void* au_shared,
+                         void* h_shared, void* y_shared, void* ws, void* stream) {
+  SharedCtx c;
+  int32_t rc = shared_ctx(cfg, T, shared_width, ws, &c);
+  if (rc) return rc;
+  REQ_PTR(x); REQ_PTR(w13_shared); REQ_PTR(w2_shared); REQ_PTR(au_shared); REQ_PTR(h_shared);
+  REQ_PTR(y_shared);
+  cudaStream_t st = (cudaStream_t)stream;
+  shared_segment_kernel<<<1, 1, 0, st>>>(c.aligned, (int)T, c.Ds.align);
+  MOHGE_LAUNCH_CHECK("shared_segment_kernel");
+  GroupPtrs P;
+  memset(&P, 0, sizeof(P));
+  P.w13[0] = w13_shared; P.w2[0] = w2_shared;
+  return expert_fwd_impl(c.Ds, P, x, c.counts, c.aligned, au_shared, h_shared, y_shared, c.w, st);
+}
+
+int32_t mohge_shared_bwd(const mohge_config* cfg, int64_t T, int32_t shared_width, const void* dy,
+                         const void* x, const void* au_shared, const void* h_shared,
+                         const void* w13_shared, const void* w2_shared, void* dau_shared,
+                         void* dx_shared, float* dw13_shared, float* dw2_shared,
+                         int32_t accumulate, void* ws, void* stream) {
+  SharedCtx c;
+  int32_t rc = shared_ctx(cfg, T, shared_width, ws, &c);
+  if (rc) return rc;
+  REQ_PTR(dy); REQ_PTR(x); REQ_PTR(au_shared); REQ_PTR(h_shared); REQ_PTR(w13_shared);
+  REQ_PTR(w2_shared); REQ_PTR(dau_shared); REQ_PTR(dx_shared); REQ_PTR(dw13_shared);
+  REQ_PTR(dw2_shared);
+  cudaStream_t st = (cudaStream_t)stream;
+  shared_segment_kernel<<<1, 1, 0, st>>>(c.aligned, (int)T, c.Ds.align);
+  MOHGE_LAUNCH_CHECK("shared_segment_kernel");
+  GroupPtrs P;
+  memset(&P, 0, sizeof(P));
+  P.w13[0] = w13_shared; P.w2[0] = w2_shared; P.dw13[0] = dw13_shared; P.dw2[0] = dw2_shared;
+  return expert_bwd_impl(c.Ds, P, dy, x, au_shared, h_shared, c.counts, c.aligned, dau_shared,
+                         dx_shared, accumulate, c.w, st);
 }
 
 int32_t mohge_route_bwd(const mohge_config* cfg, int64_t T, const void* x, const void* w_router,

@@ -129,12 +129,12 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
                         int32_t* src_of, void* x_perm, int32_t* hist, int32_t* base,
                         int32_t* status, cudaStream_t st);
 int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of,
-                       const float* gate_w, void* y, cudaStream_t st);
+                       const float* gate_w, const void* add, void* y, cudaStream_t st);
 int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
                            const int32_t* prow_of, const float* gate_w, const int32_t* counts,
                            const int32_t* aligned, void* dy_perm, float* dgate_w, cudaStream_t st);
-int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* prow_of, void* dx,
-                             cudaStream_t st);
+int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* prow_of,
+                             const void* add, void* dx, cudaStream_t st);
 
 // gemm_simt.cu
 int32_t launch_build_tiles(const Dims& D, int role, int BM, int BN, const int32_t* counts,

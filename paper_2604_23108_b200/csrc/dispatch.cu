@@ -229,12 +229,12 @@ zero_pad_rows_kernel(const int32_t* __restrict__ counts, const int32_t* __restri
     p[i] = z;
 }
 
-// y[t] = sum_k gate[t,k] * y_perm[prow[t,k]]   (gate == nullptr: plain sum)
+// y[t] = sum_k gate[t,k] * y_perm[prow[t,k]] (+ add[t])   (gate == nullptr: plain sum)
 template <typename T>
 __global__ void __launch_bounds__(256)
 combine_kernel(const Vec16* __restrict__ y_perm, const int32_t* __restrict__ prow_of,
-               const float* __restrict__ gate_w, int Tn, int Ke, int row_vecs, int rows_cap,
-               Vec16* __restrict__ y) {
+               const float* __restrict__ gate_w, const Vec16* __restrict__ add, int Tn, int Ke,
+               int row_vecs, int rows_cap, Vec16* __restrict__ y) {
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
   for (int t = blockIdx.x; t < Tn; t += gridDim.x) {
@@ -248,6 +248,7 @@ combine_kernel(const Vec16* __restrict__ y_perm, const int32_t* __restrict__ pro
       float acc[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) acc[i] = 0.0f;
+      if (add) unpack(add[(size_t)t * row_vecs + c], acc, T());   // e.g. the shared experts' output
 #pragma unroll 4
       for (int k = 0; k < Ke; ++k) {
         if ((unsigned)s_row[k] >= (unsigned)rows_cap) continue;   // invalid slot: contributes nothing
@@ -350,24 +351,26 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
 }
 
 int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of,
-                       const float* gate_w, void* y, cudaStream_t st) {
+                       const float* gate_w, const void* add, void* y, cudaStream_t st) {
   if (D.T == 0) return MOHGE_OK;
   const int T = (int)D.T;
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   if (D.bf16)
     combine_kernel<__nv_bfloat16><<<blocks, block_for(row_vecs), 0, st>>>(
-        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)y);
+        (const Vec16*)y_perm, prow_of, gate_w, (const Vec16*)add, T, D.Ke, row_vecs, (int)D.Rcap,
+        (Vec16*)y);
   else
     combine_kernel<float><<<blocks, block_for(row_vecs), 0, st>>>(
-        (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)y);
+        (const Vec16*)y_perm, prow_of, gate_w, (const Vec16*)add, T, D.Ke, row_vecs, (int)D.Rcap,
+        (Vec16*)y);
   MOHGE_LAUNCH_CHECK("combine_kernel");
   return MOHGE_OK;
 }
 
-int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* prow_of, void* dx,
-                             cudaStream_t st) {
-  return launch_combine(D, dx_perm, prow_of, nullptr, dx, st);
+int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* prow_of,
+                             const void* add, void* dx, cudaStream_t st) {
+  return launch_combine(D, dx_perm, prow_of, nullptr, add, dx, st);
 }
 
 int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,

@@ -19,7 +19,8 @@ from typing import List, Optional
 
 import torch
 
-__all__ = ["Workload", "WORKLOADS", "make_inputs", "make_device_inputs", "zipf_logit_bias"]
+__all__ = ["Workload", "WORKLOADS", "make_inputs", "make_device_inputs", "make_shared_weights",
+           "zipf_logit_bias"]
 
 
 @dataclass(frozen=True)
@@ -125,3 +126,16 @@ def make_device_inputs(wl: Workload, device, seed: Optional[int] = None):
     b = zipf_logit_bias(wl)
     out["logit_bias"] = None if b is None else b.to(device)
     return out
+
+
+def make_shared_weights(wl: Workload, shared_width: int, device="cpu", seed: Optional[int] = None):
+    """Weights of the shared experts, N(0, 0.02) like every other weight, from a generator of
+    their own (seed + 1000) so that the draws of `make_inputs` do not move:
+    (w13_shared [2*shared_width, d], w2_shared [d, shared_width]) in the layer dtype."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed((wl.seed if seed is None else seed) + 1000)
+    dt = _torch_dtype(wl.dtype)
+    d = wl.d_model
+    w13 = (torch.randn((2 * shared_width, d), generator=gen, dtype=torch.float32, device=device) * 0.02).to(dt)
+    w2 = (torch.randn((d, shared_width), generator=gen, dtype=torch.float32, device=device) * 0.02).to(dt)
+    return w13, w2

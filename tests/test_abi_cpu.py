@@ -51,13 +51,13 @@ def test_sizes_and_validation_without_a_device():
             c = B.Config(**dict(args, group_width=args["group_width"][:8])).c()
             c.n_groups = 9
         assert lib.mohge_workspace_bytes(C.byref(c), 128) == 0, kw
-        rc = lib.mohge_combine(C.byref(c), 128, None, None, None, None, None)
+        rc = lib.mohge_combine(C.byref(c), 128, None, None, None, None, None, None)
         assert rc == -1, kw
         assert len(lib.mohge_last_error()) > 0
     # NULL and misaligned pointers are refused before any launch
     good = cfg.c()
-    assert lib.mohge_combine(C.byref(good), 128, None, None, None, None, None) == -1
+    assert lib.mohge_combine(C.byref(good), 128, None, None, None, None, None, None) == -1
     assert lib.mohge_combine(C.byref(good), 128, C.c_void_p(8), C.c_void_p(16), C.c_void_p(16),
-                             C.c_void_p(16), None) == -1
+                             None, C.c_void_p(16), None) == -1
     assert b"16-byte" in lib.mohge_last_error()
     assert lib.mohge_route(C.byref(good), -5, *([None] * 12)) == -1
