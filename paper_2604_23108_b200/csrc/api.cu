@@ -69,6 +69,17 @@ int32_t make_dims(const mohge_config* c, int64_t T, Dims* D) {
 
 static int64_t up256(int64_t v) { return (v + 255) / 256 * 256; }
 
+int router_dw_splits(const Dims& D) {
+  const int m_tiles = (D.d + 127) / 128;
+  const int64_t k_blocks = (D.T + 63) / 64;
+  int64_t s = 148 / m_tiles;
+  if (s > 32) s = 32;
+  if (s > k_blocks) s = k_blocks;
+  if (s < 1) s = 1;
+  const int64_t chunk = (k_blocks + s - 1) / s;          // k-blocks per split
+  return chunk > 0 ? (int)((k_blocks + chunk - 1) / chunk) : 1;   // no split is empty
+}
+
 WsLayout ws_layout(const Dims& D) {
   WsLayout L;
   L.chunks = ceil_div(D.T, kDispatchChunk);
@@ -77,7 +88,8 @@ WsLayout ws_layout(const Dims& D) {
   L.hist_off = L.stats_off + up256((int64_t)kStatsBlocks * D.NL * 8);
   L.base_off = L.hist_off + up256((int64_t)(L.chunks + 1) * D.Ne * 4);
   L.dl16_off = L.base_off + up256((int64_t)(L.chunks + 1) * D.Ne * 4);
-  L.tiles_off = L.dl16_off + up256((D.T + 1) * (int64_t)((D.NL + 7) / 8 * 8) * 2);
+  L.rdw_off = L.dl16_off + up256((D.T + 1) * (int64_t)((D.NL + 7) / 8 * 8) * 2);
+  L.tiles_off = L.rdw_off + up256((int64_t)router_dw_splits(D) * D.NL * D.d * 4);
   // tile capacity: the smallest tile either path uses is 64 x 64
   const int64_t mt = D.Rcap / 64 + D.Ne + 1;
   const int64_t wide = (D.d > 2 * D.Wmax ? D.d : 2 * D.Wmax);
@@ -94,6 +106,7 @@ struct Ws {
   int32_t* hist;
   int32_t* base;
   __nv_bfloat16* dl16;
+  float* rdw;
   int32_t* tile_count;
   Tile* tiles;
   int64_t tiles_cap;
@@ -108,6 +121,7 @@ static Ws carve(const Dims& D, void* ws) {
   w.hist = (int32_t*)(p + L.hist_off);
   w.base = (int32_t*)(p + L.base_off);
   w.dl16 = (__nv_bfloat16*)(p + L.dl16_off);
+  w.rdw = (float*)(p + L.rdw_off);
   w.tile_count = (int32_t*)(p + L.tiles_off);
   w.tiles = (Tile*)(p + L.tiles_off + 256);
   w.tiles_cap = L.tiles_cap;
@@ -193,7 +207,7 @@ int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const voi
     REQ_PTR(x); REQ_PTR(w_router); REQ_PTR(logits_out); OPT_PTR(logit_bias);
     const int f32 = D.bf16 ? 0 : 1;
     if (D.bf16 && !force_simt())
-      rc = launch_tc_plain(D, ROLE_LOGITS, x, w_router, 0, logits_out, logit_bias, carve(D, ws).status, st);
+      rc = launch_tc_plain(D, ROLE_LOGITS, x, w_router, 0, logits_out, logit_bias, nullptr, carve(D, ws).status, st);
     else
       rc = launch_simt_plain((int)T, D.NL, D.d, x, f32, D.d, 1, w_router, f32, D.d, 1, logits_out, 1,
                              D.NL, logit_bias, 0, st);
@@ -490,9 +504,9 @@ int32_t mohge_route_bwd(const mohge_config* cfg, int64_t T, const void* x, const
   }
   if (tc) {
     // BF16 copy of dlogits feeds both router-backward GEMMs on the tensor cores
-    rc = launch_tc_plain(D, ROLE_ROUTER_DW, x, w.dl16, pitch16, dw_router, nullptr, w.status, st);
+    rc = launch_tc_plain(D, ROLE_ROUTER_DW, x, w.dl16, pitch16, dw_router, nullptr, w.rdw, w.status, st);
     if (rc) return rc;
-    return launch_tc_plain(D, ROLE_ROUTER_DX, w.dl16, w_router, pitch16, dx, nullptr, w.status, st);
+    return launch_tc_plain(D, ROLE_ROUTER_DX, w.dl16, w_router, pitch16, dx, nullptr, nullptr, w.status, st);
   }
   // dw_router[NL, d] = dlogits^T . x
   rc = launch_simt_plain(D.NL, D.d, (int)T, dlogits, 1, 1, D.NL, x, f32, 1, D.d, dw_router, 1, D.d,

@@ -54,16 +54,20 @@ static inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b)
 // stats partials      double [kStatsBlocks][NL]
 // dispatch histogram  int32 [chunks][Ne] (per-chunk counts) and the same size of chunk bases
 // dlogits (BF16)      [T][NLp], NLp = NL rounded up to 8 (operand of the router-backward GEMMs)
+// router dW partials  float [splits][NL][d]: split-K partial sums of dw_router (BF16 path)
 // tile list           int32 count (+pad to 16 B) followed by int4 entries
 constexpr int kStatsBlocks = 296;
 constexpr int kDispatchChunk = 256;  // tokens per dispatch block
 
 struct WsLayout {
-  int64_t status_off, stats_off, hist_off, base_off, dl16_off, tiles_off, total;
+  int64_t status_off, stats_off, hist_off, base_off, dl16_off, rdw_off, tiles_off, total;
   int64_t tiles_cap;
   int chunks;
 };
 WsLayout ws_layout(const Dims& D);
+// Split-K factor of the router weight-gradient GEMM: its output has only d/128 tiles, so the
+// token dimension is cut into this many ranges to occupy the SMs (partials summed in fixed order).
+int router_dw_splits(const Dims& D);
 
 // One unit of GEMM work: expert e, output tile origin (m0, n0), and a role-specific extent.
 struct __align__(16) Tile {
@@ -161,6 +165,6 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
                           int64_t tiles_cap, int32_t* status, cudaStream_t st);
 
 int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
-                        void* C, const float* bias, int32_t* status, cudaStream_t st);
+                        void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st);
 
 }  // namespace mohge

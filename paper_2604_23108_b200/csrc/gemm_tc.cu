@@ -97,6 +97,7 @@ struct TcParams {
   int32_t* status;
   // plain roles: C[M, N] over contraction K; tile ti -> (ti / ntn, ti % ntn)
   int plain_total, plain_ntn, plain_M, plain_N, plain_K;
+  int plain_splits, plain_kchunk;   // split-K of ROUTER_DW: ranges of plain_kchunk k-blocks
   float* Cf;                     // LOGITS: logits [T, NL]; ROUTER_DW: dw_router [NL, d]
   const float* bias;             // LOGITS: optional logit bias [NL]
 };
@@ -375,9 +376,11 @@ template <int ROLE>
 __device__ __forceinline__ Tile fetch_tile(const TcParams& p, int ti) {
   if (is_plain<ROLE>()) {
     Tile t;
-    t.e = 0;
-    t.m0 = (ti / p.plain_ntn) * BM;
-    t.n0 = (ti % p.plain_ntn) * p.BN[0];
+    const int per_m = p.plain_ntn * p.plain_splits;       // tile index = (m, n, split), split fastest
+    const int rem = ti % per_m;
+    t.e = rem % p.plain_splits;                            // split index
+    t.m0 = (ti / per_m) * BM;
+    t.n0 = (rem / p.plain_splits) * p.BN[0];
     t.ext = p.plain_M - t.m0 < BM ? p.plain_M - t.m0 : BM;
     return t;
   }
@@ -388,8 +391,11 @@ template <int ROLE>
 __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) {
   TileGeom q;
   if (is_plain<ROLE>()) {
-    q.e = 0; q.g = 0; q.i = 0; q.W = 0; q.bn = p.BN[0]; q.m0 = t.m0; q.n0 = t.n0; q.r0 = 0;
-    q.num_kb = (p.plain_K + BK - 1) / BK;
+    q.e = t.e; q.g = 0; q.i = 0; q.W = 0; q.bn = p.BN[0]; q.m0 = t.m0; q.n0 = t.n0;
+    const int total_kb = (p.plain_K + BK - 1) / BK;
+    const int kb0 = t.e * p.plain_kchunk;                  // first k-block of this split
+    q.r0 = kb0 * BK;
+    q.num_kb = total_kb - kb0 < p.plain_kchunk ? total_kb - kb0 : p.plain_kchunk;
     return q;
   }
   q.e = t.e;
@@ -759,6 +765,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         // transposed store: tile rows are the d index, tile columns the router output index
         const int m = q.m0 + row_in_tile;
         const bool row_ok = m < p.plain_M;
+        float* cf = p.Cf + (size_t)q.e * p.plain_N * p.plain_M;    // this split's partial sum
         for (int c = 0; c < q.bn; c += 32) {
           uint32_t r[32];
           tmem_ld32(taddr + c, r);
@@ -767,7 +774,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int n = q.n0 + c + j;
-              if (n < p.plain_N) p.Cf[(size_t)n * p.plain_M + m] = __uint_as_float(r[j]);
+              if (n < p.plain_N) cf[(size_t)n * p.plain_M + m] = __uint_as_float(r[j]);
             }
           }
         }
@@ -959,8 +966,20 @@ int cta_group_size() {
 //   LOGITS     logits[T, NL]  = x . W_r^T + bias                 A = x,          B = w_router
 //   ROUTER_DW  dw_router^T[d, NL] = x^T . dl16  (stored transposed)  A = x,       B = dl16 [T, NLp]
 //   ROUTER_DX  dx[T, d]      += dl16 . W_r                       A = dl16,       B = w_router
+namespace {
+// out[i] = part[0][i] + part[1][i] + ... in this fixed order (run-to-run identical bits)
+__global__ void __launch_bounds__(256)
+sum_partials_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    float acc = part[i];
+    for (int s = 1; s < splits; ++s) acc += part[(size_t)s * n + i];
+    out[i] = acc;
+  }
+}
+}  // namespace
+
 int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
-                        void* C, const float* bias, int32_t* status, cudaStream_t st) {
+                        void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st) {
   static int sm_count = 0;
   if (!sm_count) {
     int dev = 0;
@@ -1003,11 +1022,26 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
     if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
   }
   p.plain_ntn = (p.plain_N + p.BN[0] - 1) / p.BN[0];
-  p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn;
+  const int total_kb = (p.plain_K + BK - 1) / BK;
+  p.plain_splits = 1;
+  p.plain_kchunk = total_kb;
+  if (role == ROLE_ROUTER_DW && partials != nullptr) {
+    p.plain_splits = router_dw_splits(D);
+    p.plain_kchunk = (total_kb + p.plain_splits - 1) / p.plain_splits;
+    if (p.plain_splits > 1) p.Cf = partials;
+  }
+  p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn * p.plain_splits;
   const int grid = p.plain_total < sm_count ? p.plain_total : sm_count;
   switch (role) {
     case ROLE_LOGITS: return launch_role<ROLE_LOGITS, 1>(p, grid, st);
-    case ROLE_ROUTER_DW: return launch_role<ROLE_ROUTER_DW, 1>(p, grid, st);
+    case ROLE_ROUTER_DW: {
+      const int32_t rc2 = launch_role<ROLE_ROUTER_DW, 1>(p, grid, st);
+      if (rc2 || p.plain_splits == 1) return rc2;
+      const size_t n = (size_t)D.NL * D.d;
+      sum_partials_kernel<<<(unsigned)((n + 1023) / 1024), 256, 0, st>>>(partials, p.plain_splits, n, (float*)C);
+      MOHGE_LAUNCH_CHECK("sum_partials_kernel");
+      return MOHGE_OK;
+    }
     default: return launch_role<ROLE_ROUTER_DX, 1>(p, grid, st);
   }
 }
