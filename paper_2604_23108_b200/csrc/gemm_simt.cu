@@ -14,7 +14,10 @@ namespace mohge {
 
 namespace {
 
-constexpr int kBandTiles = 8;
+#ifndef MOHGE_BAND_TILES
+#define MOHGE_BAND_TILES 8
+#endif
+constexpr int kBandTiles = MOHGE_BAND_TILES;
 
 __global__ void __launch_bounds__(256)
 build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
