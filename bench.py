@@ -37,6 +37,7 @@ from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs
 NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 108.7e9}
 
 METRIC = "MoHGE layer fwd+bwd tokens/s"
+METRIC_FWD = "MoHGE layer fwd tokens/s"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg5_bf16_large"
 
@@ -182,10 +183,15 @@ def main():
     ap.add_argument("--ref-sample", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--forward-only", action="store_true",
+                    help="time the forward pass alone (inference-shaped workloads); the roofline "
+                         "object then describes mohge_expert_fwd against HBM bandwidth")
     ap.add_argument("--shared-width", type=int, default=0,
                     help="hidden width of the shared experts (N_s FFNs concatenated); 0 = none, "
                          "the benchmark configurations have none")
     args = ap.parse_args()
+    if args.forward_only:          # the end-to-end and CPU arms describe the fwd+bwd step only
+        args.no_e2e = args.no_cpu_baseline = True
     wl = WORKLOADS[args.workload]
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -238,6 +244,10 @@ def main():
             e1.record()
         B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, buf.y,
                         y_add=buf.y_sh if shared is not None else None)
+        if args.forward_only:
+            if mark:
+                gemm_marks.append((e0, e1, e1, e1))
+            return
         B.mohge_combine_bwd(gcfg, T, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.counts,
                             buf.aligned, buf.dy_perm, buf.dgate)
         if mark:
@@ -372,6 +382,18 @@ def main():
                 "kernel": "tc_grouped_kernel (6 launches per step: fwd1, fwd2, dgrad x2, wgrad x2)",
                 "of": pk["source"], "flops_per_step": flops, "gemm_ms_per_step": gemm_ms_step,
                 "frac_of_nominal_2250": achieved / 2250.0}
+    if args.forward_only:
+        # expert forward of a small batch: what has to move is the weights of the experts that
+        # were hit (read once), their rows of x_perm and the saved A, U, H and y_perm rows
+        es = 2 if wl.dtype == "bf16" else 4
+        N = wl.experts_per_group
+        wbytes = sum(3 * wl.d_model * wl.group_width[e // N] * es for e, m in enumerate(counts) if m > 0)
+        rbytes = sum(m * (2 * wl.d_model + 3 * wl.group_width[e // N]) * es for e, m in enumerate(counts))
+        gbs = (wbytes + rbytes) / (gemm_ms_step * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm"], "unit": "GB/s",
+                    "frac": gbs / pk["hbm"], "traffic": None,
+                    "kernel": "tc_grouped_kernel (2 launches per step: fwd1, fwd2)", "of": pk["source"],
+                    "bytes_per_step": wbytes + rbytes, "expert_fwd_ms_per_step": gemm_ms_step}
     if wl.dtype != "bf16":
         roofline.update(bound="alu", peak=None, frac=None,
                         kernel="simt_grouped_kernel (FP32 FMA; correctness configuration)")
@@ -386,12 +408,13 @@ def main():
         cpu_baseline = {"value": val, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                         "sample": "oracle fwd+bwd on the first %d tokens of the workload (%.1f s)" % (sample, per)}
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC_FWD if args.forward_only else METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "T": T, "d_model": wl.d_model, "n_groups": wl.n_groups,
                    "experts_per_group": wl.experts_per_group, "group_width": list(wl.group_width),
                    "k_groups": wl.k_groups, "k_experts": wl.k_experts, "shared_width": args.shared_width,
+                   "pass": "forward only" if args.forward_only else "forward + backward",
                    "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu_baseline,

@@ -62,6 +62,10 @@ WORKLOADS = {
     # tokens (four sequences per batch here; the paper does not state its micro-batch).
     "paper_3b_layer": Workload("paper_3b_layer", "bf16", 16384, 1024, 8, 8,
                                (384, 512, 640, 768, 896, 1024, 1152, 1280), 3, 6, seed=6),
+    # Inference-shaped batch: few tokens against the large configuration's 4 GB of expert
+    # weights, so the forward pass is bound by streaming the weights of the experts that are hit.
+    "decode_256_large": Workload("decode_256_large", "bf16", 256, 4096, 4, 32,
+                                 (2048, 1536, 1024, 512), 2, 8, seed=8),
     "paper_14b_layer": Workload("paper_14b_layer", "bf16", 16384, 1024, 8, 16,
                                 (640, 768, 896, 1024, 1152, 1280, 1408, 1536), 3, 6, seed=7),
 }
