@@ -105,7 +105,11 @@ struct TilePlan {
   int Mext[MOHGE_MAX_GROUPS];   // wgrad only: rows of the output (d or 2W)
   int Next[MOHGE_MAX_GROUPS];   // columns of the output
   int Kcost[MOHGE_MAX_GROUPS];  // row-tiled roles: contraction length (cost of one tile)
+  int wide;                     // 1: pair neighbouring n-tiles into double-width entries (kTileWide)
 };
+// A tile-list entry with this bit set in n0 covers TWO neighbouring n-tiles (n0 and n0 + BN):
+// the CTA pair computes both from one pass over A (the tensor-core path only).
+constexpr int32_t kTileWide = 1 << 30;
 TilePlan make_plan(const Dims& D, int role, int BM, const int* BN, bool fused_swiglu);
 int32_t launch_build_tiles_plan(const TilePlan& p, const int32_t* aligned, int32_t* tile_count,
                                 Tile* tiles, int64_t tiles_cap, int32_t* status, cudaStream_t st);

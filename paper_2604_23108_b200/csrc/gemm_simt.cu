@@ -39,8 +39,10 @@ build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __r
       mt = (rows + p.BM - 1) / p.BM;
       cost = (long long)p.Kcost[g] * p.BN[g];
     }
+    // with wide entries, n-tiles are taken two at a time (plus a single one when nt is odd)
+    const int ne = p.wide ? nt / 2 + (nt & 1) : nt;
     s_mt[e] = mt;
-    s_nt[e] = mt * nt;
+    s_nt[e] = mt * ne;
     s_cost[e] = s_nt[e] > 0 ? cost : -1;
   }
   __syncthreads();
@@ -88,7 +90,12 @@ build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __r
     const int tm = band * kBandTiles + in_band % band_m, tn = in_band / band_m;
     Tile t;
     t.e = ex;
-    t.n0 = tn * p.BN[gg];
+    if (p.wide) {
+      const int nt_full = (p.Next[gg] + p.BN[gg] - 1) / p.BN[gg];
+      t.n0 = tn < nt_full / 2 ? (2 * tn * p.BN[gg]) | kTileWide : (nt_full - 1) * p.BN[gg];
+    } else {
+      t.n0 = tn * p.BN[gg];
+    }
     if (wgrad) {
       t.m0 = tm * p.BM;
       t.ext = aligned[ex + 1] - aligned[ex];
@@ -334,7 +341,7 @@ int32_t launch_build_tiles_plan(const TilePlan& p, const int32_t* aligned, int32
 // Row-tiled roles: output [rows, Next]; wgrad roles: output [Mext, Next] per expert.
 TilePlan make_plan(const Dims& D, int role, int BM, const int* BN /*per group*/, bool fused_swiglu) {
   TilePlan p;
-  p.role = role; p.BM = BM; p.Ng = D.Ng; p.N = D.N; p.Ne = D.Ne; p.d = D.d;
+  p.role = role; p.BM = BM; p.Ng = D.Ng; p.N = D.N; p.Ne = D.Ne; p.d = D.d; p.wide = 0;
   for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) {
     const int W = g < D.Ng ? D.W[g] : 0;
     p.BN[g] = BN[g];

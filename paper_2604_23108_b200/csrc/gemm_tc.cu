@@ -50,10 +50,15 @@ constexpr int kStgBufBytes = 4096;
 constexpr int kStgBufs = 4;
 constexpr int kStgBytes = 4 * kStgBufs * kStgBufBytes;       // 64 KiB per CTA
 
-template <int CG> struct Geo {
-  static constexpr int kStages = CG == 1 ? 3 : 5;
-  static constexpr int kBBytes = 256 / CG * BK * 2;          // 32 KiB or 16 KiB
-  static constexpr int kStageBytes = kABytes + kBBytes;
+// WIDE = 1 (CTA pairs only): the pair works on double-width entries, 256 x 512 outputs from ONE
+// pass over A, the two 256-column halves in the two accumulator buffers.  A stage then holds A
+// and the pair's halves of both B tiles (48 KiB per CTA, three stages), which cuts the operand
+// bytes per FLOP by a quarter; the price is that the epilogue of an entry no longer overlaps
+// the MMAs of the next one.  It pays where the contraction is long (see launch_tc_grouped).
+template <int CG, int WIDE = 0> struct Geo {
+  static constexpr int kStages = (CG == 2 && !WIDE) ? 5 : 3;
+  static constexpr int kBBytes = 256 / CG * BK * 2;          // one B tile per CTA: 32 KiB or 16 KiB
+  static constexpr int kStageBytes = kABytes + kBBytes * (WIDE ? 2 : 1);
   static constexpr int kSmemBytes = kStages * kStageBytes + kStgBytes + 1024 + 512;
   static constexpr int kTileM = BM * CG;
 };
@@ -369,7 +374,7 @@ __device__ __forceinline__ void pace(long long t0, int i, int n, int next_num_kb
 }
 
 struct TileGeom {
-  int e, g, i, W, bn, m0, n0, num_kb, r0;
+  int e, g, i, W, bn, m0, n0, num_kb, r0, wide;
 };
 
 template <int ROLE>
@@ -391,7 +396,7 @@ template <int ROLE>
 __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) {
   TileGeom q;
   if (is_plain<ROLE>()) {
-    q.e = t.e; q.g = 0; q.i = 0; q.W = 0; q.bn = p.BN[0]; q.m0 = t.m0; q.n0 = t.n0;
+    q.e = t.e; q.g = 0; q.i = 0; q.W = 0; q.bn = p.BN[0]; q.m0 = t.m0; q.n0 = t.n0; q.wide = 0;
     const int total_kb = (p.plain_K + BK - 1) / BK;
     const int kb0 = t.e * p.plain_kchunk;                  // first k-block of this split
     q.r0 = kb0 * BK;
@@ -404,7 +409,8 @@ __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) 
   q.W = p.gs.W[q.g];
   q.bn = p.BN[q.g];
   q.m0 = t.m0;
-  q.n0 = t.n0;
+  q.n0 = t.n0 & (kTileWide - 1);
+  q.wide = (t.n0 & kTileWide) ? 1 : 0;
   q.r0 = 0;
   if (ROLE == ROLE_FWD1 || ROLE == ROLE_DGRAD_DOWN) q.num_kb = (p.gs.d + BK - 1) / BK;
   else if (ROLE == ROLE_FWD2) q.num_kb = (q.W + BK - 1) / BK;
@@ -416,12 +422,13 @@ __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) 
   return q;
 }
 
-template <int ROLE, int CG>
+template <int ROLE, int CG, int WIDE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_grouped_kernel(const __grid_constant__ TcParams p) {
   using RT = RoleTraits<ROLE>;
-  constexpr int kStages = Geo<CG>::kStages;
-  constexpr int kStageBytes = Geo<CG>::kStageBytes;
+  using G = Geo<CG, WIDE>;
+  constexpr int kStages = G::kStages;
+  constexpr int kStageBytes = G::kStageBytes;
   const uint32_t cta_rank = CG == 2 ? cluster_ctarank() : 0u;   // position in the CTA pair
   const int unit = blockIdx.x / CG, unit_stride = gridDim.x / CG;
   extern __shared__ uint8_t smem_raw[];
@@ -481,14 +488,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         const TileGeom q = tile_geom<ROLE>(p, t);
         const CUtensorMap* mA = &p.mapA[q.g];
         const CUtensorMap* mB = &p.mapB[q.g];
-        const int nb = q.bn / CG;                          // B rows staged by this CTA
-        const uint32_t tx = kABytes + (uint32_t)nb * BK * 2;
+        const int nb = q.bn / CG;                          // B rows staged by this CTA per B tile
+        const int pieces = (WIDE && q.wide) ? 2 : 1;       // B tiles of this entry
+        const uint32_t tx = kABytes + (uint32_t)pieces * nb * BK * 2;
         const int am0 = q.m0 + BM * (int)cta_rank;         // this CTA's 128 rows of the tile
-        const int bn0 = q.n0 + nb * (int)cta_rank;         // this CTA's slice of the tile columns
         for (int kb = 0; kb < q.num_kb; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { alive = false; break; }
           const uint32_t sA = smem_base + stage * kStageBytes;
-          const uint32_t sB = sA + kABytes;
           // CG == 2: both CTAs report to the full barrier of the pair's leader (rank 0)
           const uint32_t fb = CG == 2 ? mapa_rank(full_bar(stage), 0) : full_bar(stage);
           if (CG == 2) mbar_expect_tx_cluster(fb, tx); else mbar_expect_tx(fb, tx);
@@ -503,24 +509,31 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           } else {
             tma_2d<CG>(sA, mA, fb, k0, am0);
           }
-          if (ROLE == ROLE_FWD1) {
-            const int half = q.bn >> 1;
-            if (CG == 2) {          // leader stages the gate rows, its peer the up rows
-              tma_3d<CG>(sB, mB, fb, k0, q.n0, 2 * q.i + (int)cta_rank);
+          for (int pc = 0; pc < pieces; ++pc) {
+            const uint32_t sB = sA + kABytes + pc * G::kBBytes;
+            if (ROLE == ROLE_FWD1) {
+              const int half = q.bn >> 1;
+              const int h0 = q.n0 + pc * half;               // first hidden column of this piece
+              if (CG == 2) {          // leader stages the gate rows, its peer the up rows
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i + (int)cta_rank);
+              } else {
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i);
+                tma_3d<CG>(sB + half * 128, mB, fb, k0, h0, 2 * q.i + 1);
+              }
             } else {
-              tma_3d<CG>(sB, mB, fb, k0, q.n0, 2 * q.i);
-              tma_3d<CG>(sB + half * 128, mB, fb, k0, q.n0, 2 * q.i + 1);
+              const int bn0 = q.n0 + pc * q.bn + nb * (int)cta_rank;   // this CTA's slice of the columns
+              if (ROLE == ROLE_LOGITS) {
+                tma_2d<CG>(sB, mB, fb, k0, bn0);
+              } else if (ROLE == ROLE_FWD2) {
+                tma_3d<CG>(sB, mB, fb, k0, bn0, q.i);
+              } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
+                if (p.b_blk[q.g]) tma_4d<CG>(sB, mB, fb, 0, k0, bn0 >> 6, q.i);
+                else for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i);
+              } else {
+                if (p.b_blk[q.g]) tma_3d<CG>(sB, mB, fb, 0, q.r0 + k0, bn0 >> 6);
+                else for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0);
+              }
             }
-          } else if (ROLE == ROLE_LOGITS) {
-            tma_2d<CG>(sB, mB, fb, k0, bn0);
-          } else if (ROLE == ROLE_FWD2) {
-            tma_3d<CG>(sB, mB, fb, k0, bn0, q.i);
-          } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
-            if (p.b_blk[q.g]) tma_4d<CG>(sB, mB, fb, 0, k0, bn0 >> 6, q.i);
-            else for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i);
-          } else {
-            if (p.b_blk[q.g]) tma_3d<CG>(sB, mB, fb, 0, q.r0 + k0, bn0 >> 6);
-            else for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -534,36 +547,86 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       int buf = 0;
       uint32_t acc_phase = 0;
       bool alive = true;
+      // MMAs of one k-block into accumulator column base d_tmem from the B tile at sB
+      auto issue_kblock = [&](uint32_t d_tmem, uint32_t sA, uint32_t sB, uint32_t idesc, bool first) {
+#pragma unroll
+        for (int kk = 0; kk < BK / 16; ++kk) {
+          const uint64_t da = RT::A_MN ? make_desc(sA + kk * 2048, 8192, 1024)
+                                       : make_desc(sA + kk * 32, 16, 1024);
+          const uint64_t db = RT::B_MN ? make_desc(sB + kk * 2048, 8192, 1024)
+                                       : make_desc(sB + kk * 32, 16, 1024);
+          const uint32_t acc = (first && kk == 0) ? 0u : 1u;
+          if (CG == 2) umma2_bf16(d_tmem, da, db, idesc, acc);
+          else umma_bf16(d_tmem, da, db, idesc, acc);
+        }
+      };
+      auto free_stage = [&](int st) { if (CG == 2) umma2_commit(empty_bar(st)); else umma_commit(empty_bar(st)); };
+      auto acc_done = [&](int b) { if (CG == 2) umma2_commit(tfull_bar(b)); else umma_commit(tfull_bar(b)); };
       for (int ti = unit; ti < total && alive; ti += unit_stride) {
         const Tile t = fetch_tile<ROLE>(p, ti);
         const TileGeom q = tile_geom<ROLE>(p, t);
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
                                ((uint32_t)RT::B_MN << 16) | ((uint32_t)(q.bn >> 3) << 17) |
-                               ((uint32_t)(Geo<CG>::kTileM >> 4) << 24);
-        if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag, p.status, 2)) { alive = false; break; }
+                               ((uint32_t)(G::kTileM >> 4) << 24);
+        if (!WIDE || !q.wide) {
+          if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag, p.status, 2)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * kAccCols;
+          for (int kb = 0; kb < q.num_kb; ++kb) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
+            tc_fence_after();
+            const uint32_t sA = smem_base + stage * kStageBytes;
+            issue_kblock(d_tmem, sA, sA + kABytes, idesc, kb == 0);
+            free_stage(stage);               // frees the stage (in both CTAs of a pair) once read
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+          if (!alive) break;
+          acc_done(buf);
+          if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
+          continue;
+        }
+        // ---- double-width entry: accumulators b0 (columns n0..) and b1 (columns n0 + bn..).
+        // The epilogue drains b0 first.  The first kDefer k-blocks go to b0 alone while b1 is
+        // still being drained, then b1 catches up on the same stages; after that each
+        // k-block feeds both.
+        const int b0 = buf, b1 = buf ^ 1;
+        const uint32_t ph0 = acc_phase, ph1 = (b1 == 0) ? (acc_phase ^ 1u) : acc_phase;
+        const uint32_t d0 = tmem_base + b0 * kAccCols, d1 = tmem_base + b1 * kAccCols;
+        constexpr int kDefer = 2;
+        const int nd = q.num_kb < kDefer ? q.num_kb : kDefer;
+        if (!mbar_wait(tempty_bar(b0), ph0 ^ 1u, abort_flag, p.status, 2)) { alive = false; break; }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + buf * kAccCols;
-        for (int kb = 0; kb < q.num_kb; ++kb) {
+        int st_d[kDefer];
+        for (int kb = 0; kb < nd; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
           tc_fence_after();
           const uint32_t sA = smem_base + stage * kStageBytes;
-          const uint32_t sB = sA + kABytes;
-#pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            const uint64_t da = RT::A_MN ? make_desc(sA + kk * 2048, 8192, 1024)
-                                         : make_desc(sA + kk * 32, 16, 1024);
-            const uint64_t db = RT::B_MN ? make_desc(sB + kk * 2048, 8192, 1024)
-                                         : make_desc(sB + kk * 32, 16, 1024);
-            if (CG == 2) umma2_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
-            else umma_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
-          }
-          // frees the stage (in both CTAs of a pair) when these MMAs have read it
-          if (CG == 2) umma2_commit(empty_bar(stage)); else umma_commit(empty_bar(stage));
+          issue_kblock(d0, sA, sA + kABytes, idesc, kb == 0);
+          st_d[kb] = stage;
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!alive) break;
-        if (CG == 2) umma2_commit(tfull_bar(buf)); else umma_commit(tfull_bar(buf));   // accumulator complete
-        if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
+        if (!mbar_wait(tempty_bar(b1), ph1 ^ 1u, abort_flag, p.status, 6)) { alive = false; break; }
+        tc_fence_after();
+        for (int kb = 0; kb < nd; ++kb) {
+          const uint32_t sA = smem_base + st_d[kb] * kStageBytes;
+          issue_kblock(d1, sA, sA + kABytes + G::kBBytes, idesc, kb == 0);
+          free_stage(st_d[kb]);
+        }
+        for (int kb = nd; kb < q.num_kb; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
+          tc_fence_after();
+          const uint32_t sA = smem_base + stage * kStageBytes;
+          issue_kblock(d0, sA, sA + kABytes, idesc, false);
+          issue_kblock(d1, sA, sA + kABytes + G::kBBytes, idesc, false);
+          free_stage(stage);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!alive) break;
+        acc_done(b0);
+        acc_done(b1);
+        // two buffers used: the buffer index is unchanged, the phase of both advances
+        if (b0 == 0) acc_phase ^= 1u; else { buf = 1; acc_phase ^= 1u; }
       }
     }
   } else {
@@ -579,7 +642,11 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     bool alive = true;
     for (int ti = unit; ti < total && alive; ti += unit_stride) {
       const Tile t = fetch_tile<ROLE>(p, ti);
-      const TileGeom q = tile_geom<ROLE>(p, t);
+      TileGeom q = tile_geom<ROLE>(p, t);
+      // a double-width entry is drained as two pieces, one accumulator buffer each
+      const int pieces = (WIDE && q.wide) ? 2 : 1;
+      for (int pc = 0; pc < pieces && alive; ++pc) {
+      if (pc) q.n0 += RT::EPI == EPI_SWIGLU_FWD ? (q.bn >> 1) : q.bn;
       // row-tiled expert roles: first row of this warp; segments are 128-row aligned, so the
       // rows of one CTA are either all inside the expert's segment or all outside
       const int row0 = q.m0 + BM * (int)cta_rank + quad * 32;
@@ -605,7 +672,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       // pacing reference: now, and the k-blocks of the tile whose MMAs overlap this epilogue
       const long long t_epi = clock64();
       int next_kb = 0;
-      if ((RT::EPI == EPI_BF16 || RT::EPI == EPI_F32) && ti + unit_stride < total)
+      if ((RT::EPI == EPI_BF16 || RT::EPI == EPI_F32) && !(WIDE && q.wide) && ti + unit_stride < total)
         next_kb = tile_geom<ROLE>(p, fetch_tile<ROLE>(p, ti + unit_stride)).num_kb;
       if (RT::EPI == EPI_SWIGLU_FWD) {
         const int half = q.bn >> 1;
@@ -802,6 +869,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         if (CG == 2) mbar_arrive_cluster(mapa_rank(tempty_bar(buf), 0)); else mbar_arrive(tempty_bar(buf));
       }
       if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
+      }   // pieces
     }
     if (lane == 0) bulk_wait_all();            // staged stores have left before the CTA retires
   }
@@ -915,19 +983,19 @@ int pick_bn(int extent, const int* cand, int ncand) {
   return best;
 }
 
-template <int ROLE, int CG>
+template <int ROLE, int CG, int WIDE = 0>
 int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    Geo<CG>::kSmemBytes));
+    MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE, CG, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    Geo<CG, WIDE>::kSmemBytes));
     attr_set = true;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(grid / CG * CG);
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = Geo<CG>::kSmemBytes;
+  cfg.dynamicSmemBytes = Geo<CG, WIDE>::kSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -943,15 +1011,38 @@ int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
     static int max_clusters = 0;
     if (!max_clusters) {
       cfg.gridDim = dim3(grid / CG * CG);
-      MOHGE_CUDA(cudaOccupancyMaxActiveClusters(&max_clusters, tc_grouped_kernel<ROLE, CG>, &cfg));
+      MOHGE_CUDA(cudaOccupancyMaxActiveClusters(&max_clusters, tc_grouped_kernel<ROLE, CG, WIDE>, &cfg));
       if (max_clusters < 1) max_clusters = 1;
     }
     const int want = grid / CG < max_clusters ? grid / CG : max_clusters;
     cfg.gridDim = dim3(want * CG);
   }
-  MOHGE_CUDA(cudaLaunchKernelEx(&cfg, tc_grouped_kernel<ROLE, CG>, p));
+  MOHGE_CUDA(cudaLaunchKernelEx(&cfg, tc_grouped_kernel<ROLE, CG, WIDE>, p));
   MOHGE_LAUNCH_CHECK("tc_grouped_kernel");
   return MOHGE_OK;
+}
+
+// Double-width entries for a role of a CTA-pair launch.  Default: where the FLOP-weighted mean
+// contraction length of the launch is at least kWideMinK (the exposed epilogue of an entry is
+// then a few percent of its MMA time and the saved operand traffic outweighs it).  The debugging
+// switch MOHGE_TC_WIDE=<bit mask over roles 0..5> overrides the rule.
+constexpr double kWideMinK = 3000.0;
+bool wide_tiles(const Dims& D, int role) {
+  const char* e = getenv("MOHGE_TC_WIDE");
+  if (e && e[0]) return (atoi(e) >> role) & 1;
+  double num = 0.0, den = 0.0;            // mean contraction length, weighted by the group's width
+  for (int g = 0; g < D.Ng; ++g) {
+    double k;
+    switch (role) {
+      case ROLE_FWD1: case ROLE_DGRAD_DOWN: k = D.d; break;
+      case ROLE_FWD2: k = D.W[g]; break;
+      case ROLE_DGRAD_13: k = 2.0 * D.W[g]; break;
+      default: k = (double)D.R / D.Ne; break;            // wgrad: rows of an average expert
+    }
+    num += k * D.W[g];
+    den += D.W[g];
+  }
+  return den > 0.0 && num / den >= kWideMinK;
 }
 
 // CTAs per MMA for the grouped roles (debugging switch MOHGE_TC_CG=1 keeps the single-CTA form)
@@ -1163,9 +1254,21 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
     }
   }
   if (rc) return rc;
-  rc = launch_build_tiles_plan(make_plan(D, role, BM * CG, bn_plan, role == ROLE_FWD1), aligned, tile_count,
-                               tiles, tiles_cap, status, st);
+  TilePlan plan = make_plan(D, role, BM * CG, bn_plan, role == ROLE_FWD1);
+  const bool wide = CG == 2 && wide_tiles(D, role);
+  plan.wide = wide ? 1 : 0;
+  rc = launch_build_tiles_plan(plan, aligned, tile_count, tiles, tiles_cap, status, st);
   if (rc) return rc;
+  if (CG == 2 && wide) {
+    switch (role) {
+      case ROLE_FWD1: return launch_role<ROLE_FWD1, 2, 1>(p, sm_count, st);
+      case ROLE_FWD2: return launch_role<ROLE_FWD2, 2, 1>(p, sm_count, st);
+      case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 2, 1>(p, sm_count, st);
+      case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 2, 1>(p, sm_count, st);
+      case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 2, 1>(p, sm_count, st);
+      default: return launch_role<ROLE_WGRAD_13, 2, 1>(p, sm_count, st);
+    }
+  }
   if (CG == 2) {
     switch (role) {
       case ROLE_FWD1: return launch_role<ROLE_FWD1, 2>(p, sm_count, st);
