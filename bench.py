@@ -32,9 +32,9 @@ from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs
 
 # DRAM bytes (read + written) of the six grouped-GEMM launches of one step, from the 1-pass ncu
 # capture summarised in profiles/launch_list_layer_step_cfg5.md (the L2 hit rate of these launches
-# differs between the GPUs of the pool: captures range from 68 GB to 109 GB); workloads without a
+# differs between the GPUs of the pool: captures of the same build range over tens of GB); workloads without a
 # capture of the current kernels report null.
-NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 108.7e9}
+NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 82.7e9}
 
 METRIC = "MoHGE layer fwd+bwd tokens/s"
 METRIC_FWD = "MoHGE layer fwd tokens/s"
