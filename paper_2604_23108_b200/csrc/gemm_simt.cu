@@ -64,7 +64,20 @@ build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __r
       if (blockIdx.x == 0) atomicCAS(status, 0, (2 << 24) | 2);
       s_start[p.Ne] = 0;
     }
-    if (blockIdx.x == 0) *tile_count = s_start[p.Ne];
+    if (blockIdx.x == 0) {
+      tile_count[0] = s_start[p.Ne];
+      // tile_count[1]: 1 when the costs per tile differ by more than a quarter between experts
+      // (skewed routing, or groups of different contraction length): the persistent CTAs then
+      // walk the sorted list in alternating directions
+      long long lo = -1, hi = -1;
+      for (int r = 0; r < p.Ne; ++r) {
+        const long long c = s_cost[r];
+        if (c <= 0) continue;
+        if (lo < 0 || c < lo) lo = c;
+        if (c > hi) hi = c;
+      }
+      tile_count[1] = (lo > 0 && hi * 4 > lo * 5) ? 1 : 0;
+    }
   }
   __syncthreads();
   // every block has built the same per-expert table; the entries are written grid-strided

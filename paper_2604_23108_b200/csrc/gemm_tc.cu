@@ -476,6 +476,17 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int total = is_plain<ROLE>() ? p.plain_total : *p.tile_count;
+  // Tile of this CTA (pair) in round i.  The list is sorted by cost, heaviest first.  When the
+  // costs differ (zigzag), rounds alternate direction (0..n-1, then n-1..0), so no CTA always gets
+  // the heaviest tile of its round; with equal costs the plain order measured slightly faster.  Returns -1 when the round has no tile left for this CTA (last, partial round).
+  const bool zigzag = (is_plain<ROLE>() || WIDE) ? false : p.tile_count[1] != 0;   // set by the list builder
+  auto tile_of = [&](int i) {
+    const int ti = i * unit_stride + ((zigzag && (i & 1)) ? unit_stride - 1 - unit : unit);
+    return ti < total ? ti : -1;
+  };
+  const int rounds = (total + unit_stride - 1) / unit_stride;
+  // loop variable: the round when zigzag, else the tile index itself
+  const int it0 = zigzag ? 0 : unit, it_step = zigzag ? 1 : unit_stride, it_end = zigzag ? rounds : total;
 
   if (warp == 0) {
     // ================= TMA producer =================
@@ -483,7 +494,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int ti = unit; ti < total && alive; ti += unit_stride) {
+      for (int it = it0; it < it_end && alive; it += it_step) {
+        const int ti = zigzag ? tile_of(it) : it;
+        if (ti < 0) continue;
         const Tile t = fetch_tile<ROLE>(p, ti);
         const TileGeom q = tile_geom<ROLE>(p, t);
         const CUtensorMap* mA = &p.mapA[q.g];
@@ -562,7 +575,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       };
       auto free_stage = [&](int st) { if (CG == 2) umma2_commit(empty_bar(st)); else umma_commit(empty_bar(st)); };
       auto acc_done = [&](int b) { if (CG == 2) umma2_commit(tfull_bar(b)); else umma_commit(tfull_bar(b)); };
-      for (int ti = unit; ti < total && alive; ti += unit_stride) {
+      for (int it = it0; it < it_end && alive; it += it_step) {
+        const int ti = zigzag ? tile_of(it) : it;
+        if (ti < 0) continue;
         const Tile t = fetch_tile<ROLE>(p, ti);
         const TileGeom q = tile_geom<ROLE>(p, t);
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
@@ -640,7 +655,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     int buf = 0;
     uint32_t acc_phase = 0;
     bool alive = true;
-    for (int ti = unit; ti < total && alive; ti += unit_stride) {
+    for (int it = it0; it < it_end && alive; it += it_step) {
+      const int ti = zigzag ? tile_of(it) : it;
+      if (ti < 0) continue;
       const Tile t = fetch_tile<ROLE>(p, ti);
       TileGeom q = tile_geom<ROLE>(p, t);
       // a double-width entry is drained as two pieces, one accumulator buffer each
@@ -672,8 +689,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       // pacing reference: now, and the k-blocks of the tile whose MMAs overlap this epilogue
       const long long t_epi = clock64();
       int next_kb = 0;
-      if ((RT::EPI == EPI_BF16 || RT::EPI == EPI_F32) && !(WIDE && q.wide) && ti + unit_stride < total)
-        next_kb = tile_geom<ROLE>(p, fetch_tile<ROLE>(p, ti + unit_stride)).num_kb;
+      if ((RT::EPI == EPI_BF16 || RT::EPI == EPI_F32) && !(WIDE && q.wide) && it + it_step < it_end &&
+          (zigzag ? tile_of(it + 1) : it + it_step) >= 0)
+        next_kb = tile_geom<ROLE>(p, fetch_tile<ROLE>(p, zigzag ? tile_of(it + 1) : it + it_step)).num_kb;
       if (RT::EPI == EPI_SWIGLU_FWD) {
         const int half = q.bn >> 1;
         for (int c = 0; rows_ok && c < half && q.n0 + c < q.W; c += 64) {
