@@ -680,6 +680,22 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           tma_load_2d_hint(stg + (set * 2 + 1) * kStgBufBytes, &p.mapE[1][q.g], bar, q.n0, row0, pol_stream);
         }
       }
+      int nch_acc = 0;
+      if (RT::EPI == EPI_BF16_ACC) {
+        // dx += ...: all (up to four) 64-column chunks of this warp's 32 rows are fetched at once
+        // into the staging ring, added to in place and stored from there; rows past T are clipped
+        const int left = p.plain_N - q.n0;
+        nch_acc = ((left < q.bn ? left : q.bn) + 63) / 64;
+        if (q.m0 + BM * (int)cta_rank + quad * 32 >= p.plain_M) nch_acc = 0;
+        if (nch_acc > 0 && lane == 0) {
+          bulk_wait_read<0>();
+          const uint32_t bar = ein_bar(quad, 0);
+          mbar_expect_tx(bar, (uint32_t)nch_acc * kStgBufBytes);
+          for (int ci = 0; ci < nch_acc; ++ci)
+            tma_load_2d_hint(stg + ci * kStgBufBytes, &p.mapO[0][0], bar, q.n0 + ci * 64,
+                             q.m0 + quad * 32, pol_stream);
+        }
+      }
       // the whole warp must agree before the warp-collective tensor-memory loads
       const bool got = mbar_wait(tfull_bar(buf), acc_phase, abort_flag, p.status, 4);
       if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
@@ -864,20 +880,36 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           }
         }
       } else if (RT::EPI == EPI_BF16_ACC) {
-        const long long row = q.m0 + row_in_tile;
-        const bool row_ok = row_in_tile < t.ext;
-        for (int c = 0; c < q.bn; c += 32) {
-          uint32_t r[32];
-          tmem_ld32(taddr + c, r);
-          tmem_ld_wait();
-          const int valid = p.plain_N - (q.n0 + c);
-          if (row_ok && valid > 0) {
-            float v[32];
-            __nv_bfloat16* po = p.C + row * p.plain_N + q.n0 + c;
-            load_row32(po, v, valid);
+        if (nch_acc > 0) {
+          const bool in_ok = mbar_wait(ein_bar(quad, 0), n_chunk & 1u, abort_flag, p.status, 5);
+          if (!__all_sync(0xffffffffu, in_ok)) { alive = false; break; }
+          ++n_chunk;                                   // uses of this barrier so far (its phase)
+          for (int ci = 0; ci < nch_acc; ++ci) {
+            const uint32_t bO = stg + ci * kStgBufBytes;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
-            store_row32(po, v, valid);
+            for (int hh = 0; hh < 2; ++hh) {
+              uint32_t r[32];
+              tmem_ld32(taddr + ci * 64 + 32 * hh, r);
+              tmem_ld_wait();
+#pragma unroll
+              for (int j4 = 0; j4 < 4; ++j4) {
+                const uint32_t a = stg_addr(bO, lane, hh * 4 + j4);
+                const uint4 v = ld_shared_v4(a);
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                uint32_t o[4];
+#pragma unroll
+                for (int e2 = 0; e2 < 4; ++e2)
+                  o[e2] = pack2(bf_lo(w[e2]) + __uint_as_float(r[j4 * 8 + 2 * e2]),
+                                bf_hi(w[e2]) + __uint_as_float(r[j4 * 8 + 2 * e2 + 1]));
+                st_shared_v4(a, o[0], o[1], o[2], o[3]);
+              }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&p.mapO[0][0], bO, q.n0 + ci * 64, q.m0 + quad * 32, pol_stream);
+              bulk_commit();
+            }
           }
         }
       }
@@ -1129,6 +1161,7 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
     if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
     dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = 64; box[1] = BK;
     if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+    if ((rc = encode_stage_map(&p.mapO[0][0], C, d, T, d * 2))) return rc;    // dx, read and written
   }
   p.plain_ntn = (p.plain_N + p.BN[0] - 1) / p.BN[0];
   const int total_kb = (p.plain_K + BK - 1) / BK;
