@@ -132,9 +132,23 @@ def oracle_sample_run(wl: Workload, sample_tokens: int, steps: int, warmup: int,
 def run_reference(args, wl: Workload, rank: int):
     if rank != 0:
         return
-    sample = min(wl.T, args.ref_sample)
     cores = torch.get_num_threads()
-    val, per = oracle_sample_run(wl, sample, max(1, args.steps), min(args.warmup, 1))
+    # The oracle's time per step is set by how many distinct experts the sample hits (it converts
+    # each one's weights to fp64).  A two-token probe gives the cost per expert; the sample is then
+    # the largest power of two of tokens (at most --ref-sample) for which steps + warm-up fit in
+    # about 150 s.
+    from paper_2604_23108_b200.inputs import make_inputs
+    inp_cpu = make_inputs(wl, T=min(wl.T, args.ref_sample))
+    Ne, Ke = wl.n_experts, wl.k_experts
+    hits = lambda n: Ne * (1.0 - (1.0 - min(1.0, Ke / Ne)) ** n)
+    probe = min(2, wl.T)
+    _, t_probe = oracle_sample_run(wl, probe, 1, 0, inp_cpu=inp_cpu)
+    per_expert = t_probe / max(1.0, hits(probe))
+    n_steps = max(1, args.steps) + min(args.warmup, 1)
+    sample = min(wl.T, args.ref_sample)
+    while sample > 1 and n_steps * per_expert * hits(sample) > 150.0:
+        sample //= 2
+    val, per = oracle_sample_run(wl, sample, max(1, args.steps), min(args.warmup, 1), inp_cpu=inp_cpu)
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3,
