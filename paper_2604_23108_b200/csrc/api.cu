@@ -96,7 +96,7 @@ WsLayout ws_layout(const Dims& D) {
   const int64_t row_tiled = mt * ((wide + 63) / 64);
   const int64_t wgrad = (int64_t)D.Ne * ((2 * D.Wmax + 63) / 64) * ((D.d + 63) / 64);
   L.tiles_cap = row_tiled > wgrad ? row_tiled : wgrad;
-  L.total = L.tiles_off + 256 + up256(L.tiles_cap * (int64_t)sizeof(Tile));
+  L.total = L.tiles_off + 1024 + (int64_t)kMaxLists * up256(L.tiles_cap * (int64_t)sizeof(Tile));
   return L;
 }
 
@@ -123,7 +123,7 @@ static Ws carve(const Dims& D, void* ws) {
   w.dl16 = (__nv_bfloat16*)(p + L.dl16_off);
   w.rdw = (float*)(p + L.rdw_off);
   w.tile_count = (int32_t*)(p + L.tiles_off);
-  w.tiles = (Tile*)(p + L.tiles_off + 256);
+  w.tiles = (Tile*)(p + L.tiles_off + 1024);   // kMaxLists lists, tiles_cap entries apart
   w.tiles_cap = L.tiles_cap;
   return w;
 }
@@ -262,11 +262,17 @@ static int32_t expert_fwd_impl(const Dims& D, const GroupPtrs& P, const void* x_
   int32_t rc;
   if (D.bf16 && !force_simt()) {
     MOHGE_CHECK_ARG(D.align == 128, "the BF16 tensor-core path needs row_align = 128");
+    // both tile lists with one launch, then the two GEMMs
+    const TilePlan plans[2] = {tc_tile_plan(D, ROLE_FWD1), tc_tile_plan(D, ROLE_FWD2)};
+    rc = launch_build_tiles_multi(plans, 2, aligned_offsets, w.tile_count, w.tiles, w.tiles_cap,
+                                  w.status, st);
+    if (rc) return rc;
     rc = launch_tc_grouped(D, ROLE_FWD1, P, x_perm, nullptr, au_saved, h_saved, counts,
-                           aligned_offsets, 0, w.tile_count, w.tiles, w.tiles_cap, w.status, st);
+                           aligned_offsets, 0, w.tile_count, w.tiles, w.tiles_cap, w.status, st, true);
     if (rc) return rc;
     return launch_tc_grouped(D, ROLE_FWD2, P, h_saved, nullptr, y_perm, nullptr, counts,
-                             aligned_offsets, 0, w.tile_count, w.tiles, w.tiles_cap, w.status, st);
+                             aligned_offsets, 0, w.tile_count + 64, w.tiles + w.tiles_cap,
+                             w.tiles_cap, w.status, st, true);
   }
   rc = launch_build_tiles(D, ROLE_FWD1, 64, 64, counts, aligned_offsets, w.tile_count, w.tiles,
                           w.tiles_cap, w.status, st);
@@ -336,6 +342,11 @@ static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy
   if (D.bf16 && !force_simt()) {
     MOHGE_CHECK_ARG(D.align == 128, "the BF16 tensor-core path needs row_align = 128");
     const int roles[4] = {ROLE_DGRAD_DOWN, ROLE_WGRAD_DOWN, ROLE_DGRAD_13, ROLE_WGRAD_13};
+    TilePlan plans[4];
+    for (int r = 0; r < 4; ++r) plans[r] = tc_tile_plan(D, roles[r]);
+    rc = launch_build_tiles_multi(plans, 4, aligned_offsets, w.tile_count, w.tiles, w.tiles_cap,
+                                  w.status, st);
+    if (rc) return rc;
     for (int r = 0; r < 4; ++r) {
       const void* A = nullptr; const void* B = nullptr; void* C = nullptr; void* C2 = nullptr;
       switch (roles[r]) {
@@ -345,7 +356,8 @@ static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy
         default: A = dau; B = x_perm; break;
       }
       rc = launch_tc_grouped(D, roles[r], P, A, B, C, C2, counts, aligned_offsets, accumulate,
-                             w.tile_count, w.tiles, w.tiles_cap, w.status, st);
+                             w.tile_count + 64 * r, w.tiles + w.tiles_cap * r, w.tiles_cap, w.status,
+                             st, true);
       if (rc) return rc;
     }
     return MOHGE_OK;

@@ -166,7 +166,14 @@ int32_t launch_simt_plain(int M, int N, int K, const void* A, int a_f32, int64_t
 int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
                           const void* B, void* C, void* C2, const int32_t* counts,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
-                          int64_t tiles_cap, int32_t* status, cudaStream_t st);
+                          int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt = false);
+TilePlan tc_tile_plan(const Dims& D, int role);
+// builds up to four tile lists with one launch; list i goes to tile_count + 64 * i (ints) and
+// tiles + i * tiles_cap
+constexpr int kMaxLists = 4;
+int32_t launch_build_tiles_multi(const TilePlan* plans, int nplans, const int32_t* aligned,
+                                 int32_t* tile_count, Tile* tiles, int64_t tiles_cap,
+                                 int32_t* status, cudaStream_t st);
 
 int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
                         void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st);

@@ -8,6 +8,8 @@
 // persistent CTAs walk the list with a fixed stride, so every CTA receives an interleaved sample
 // of the sorted costs and the totals differ by at most about one tile.
 
+#include <string.h>
+
 #include "common.cuh"
 
 namespace mohge {
@@ -19,9 +21,9 @@ namespace {
 #endif
 constexpr int kBandTiles = MOHGE_BAND_TILES;
 
-__global__ void __launch_bounds__(256)
-build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
-                   Tile* __restrict__ tiles, long long cap, int32_t* status) {
+__device__ __forceinline__ void
+build_tiles_body(const TilePlan& p, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
+                 Tile* __restrict__ tiles, long long cap, int32_t* status) {
   __shared__ int s_nt[256], s_mt[256], s_order[256], s_start[257];
   __shared__ long long s_cost[256];
   const int e = threadIdx.x;
@@ -119,6 +121,24 @@ build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __r
     }
     tiles[i] = t;
   }
+}
+
+__global__ void __launch_bounds__(256)
+build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
+                   Tile* __restrict__ tiles, long long cap, int32_t* status) {
+  build_tiles_body(p, aligned, tile_count, tiles, cap, status);
+}
+
+// Several lists with one launch: blockIdx.y picks the plan; list i keeps its count at
+// tile_count + 64 * i and its entries at tiles + i * cap.
+struct MultiPlan {
+  TilePlan p[kMaxLists];
+};
+__global__ void __launch_bounds__(256)
+build_tiles_multi_kernel(MultiPlan mp, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
+                         Tile* __restrict__ tiles, long long cap, int32_t* status) {
+  const int i = blockIdx.y;
+  build_tiles_body(mp.p[i], aligned, tile_count + 64 * i, tiles + (size_t)cap * i, cap, status);
 }
 
 // ---------------------------------------------------------------- FFMA tile core
@@ -342,6 +362,18 @@ GroupShape make_group_shape(const Dims& D) {
   for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) gs.W[g] = g < D.Ng ? D.W[g] : 0;
   gs.Ng = D.Ng; gs.N = D.N; gs.d = D.d; gs.Wmax = D.Wmax;
   return gs;
+}
+
+int32_t launch_build_tiles_multi(const TilePlan* plans, int nplans, const int32_t* aligned,
+                                 int32_t* tile_count, Tile* tiles, int64_t tiles_cap,
+                                 int32_t* status, cudaStream_t st) {
+  MultiPlan mp;
+  memset(&mp, 0, sizeof(mp));
+  for (int i = 0; i < nplans && i < kMaxLists; ++i) mp.p[i] = plans[i];
+  build_tiles_multi_kernel<<<dim3(32, nplans), 256, 0, st>>>(mp, aligned, tile_count, tiles,
+                                                           (long long)tiles_cap, status);
+  MOHGE_LAUNCH_CHECK("build_tiles_multi_kernel");
+  return MOHGE_OK;
 }
 
 int32_t launch_build_tiles_plan(const TilePlan& p, const int32_t* aligned, int32_t* tile_count,

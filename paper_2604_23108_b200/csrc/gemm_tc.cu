@@ -1195,10 +1195,31 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
 //   DGRAD_13    A = dau                  C = dx_perm
 //   WGRAD_DOWN  A = dy_perm, B = h_saved     -> dw2
 //   WGRAD_13    A = dau,     B = x_perm      -> dw13
+// Tile list plan of a grouped role (tile widths per group, pair rows, double-width flag): the same
+// choices launch_tc_grouped makes, so that the lists of several roles can be built by one launch
+// before the GEMMs run.
+TilePlan tc_tile_plan(const Dims& D, int role) {
+  const int CG = cta_group_size();
+  const int cand_n[2] = {256, 128};
+  const int cand_h[2] = {128, 64};
+  int bn_plan[MOHGE_MAX_GROUPS];
+  for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) bn_plan[g] = 128;
+  for (int g = 0; g < D.Ng; ++g) {
+    switch (role) {
+      case ROLE_FWD1: bn_plan[g] = pick_bn(D.W[g], cand_h, CG == 2 ? 1 : 2); break;
+      case ROLE_FWD2: case ROLE_DGRAD_13: case ROLE_WGRAD_13: bn_plan[g] = pick_bn(D.d, cand_n, 2); break;
+      default: bn_plan[g] = pick_bn(D.W[g], cand_n, 2); break;     // DGRAD_DOWN, WGRAD_DOWN
+    }
+  }
+  TilePlan plan = make_plan(D, role, BM * CG, bn_plan, role == ROLE_FWD1);
+  plan.wide = (CG == 2 && wide_tiles(D, role)) ? 1 : 0;
+  return plan;
+}
+
 int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
                           const void* B, void* C, void* C2, const int32_t* /*counts*/,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
-                          int64_t tiles_cap, int32_t* status, cudaStream_t st) {
+                          int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt) {
   static int sm_count = 0;
   if (!sm_count) {
     int dev = 0;
@@ -1305,11 +1326,12 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
     }
   }
   if (rc) return rc;
-  TilePlan plan = make_plan(D, role, BM * CG, bn_plan, role == ROLE_FWD1);
-  const bool wide = CG == 2 && wide_tiles(D, role);
-  plan.wide = wide ? 1 : 0;
-  rc = launch_build_tiles_plan(plan, aligned, tile_count, tiles, tiles_cap, status, st);
-  if (rc) return rc;
+  const TilePlan plan = tc_tile_plan(D, role);
+  const bool wide = plan.wide != 0;
+  if (!list_prebuilt) {
+    rc = launch_build_tiles_plan(plan, aligned, tile_count, tiles, tiles_cap, status, st);
+    if (rc) return rc;
+  }
   if (CG == 2 && wide) {
     switch (role) {
       case ROLE_FWD1: return launch_role<ROLE_FWD1, 2, 1>(p, sm_count, st);

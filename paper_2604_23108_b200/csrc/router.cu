@@ -259,12 +259,18 @@ __global__ void aux_finalize_kernel(RouterShape s, LossParams lp, int nblocks,
                                     const int32_t* __restrict__ cnt_lit, float* __restrict__ group_psum,
                                     float* __restrict__ expert_psum, float* __restrict__ loss_out) {
   __shared__ double s_tot[256 + MOHGE_MAX_GROUPS];
-  for (int c = threadIdx.x; c < s.NL; c += blockDim.x) {
+  // one warp per column: lane l adds the partial rows l, l + 32, ... in that order, then a
+  // butterfly adds the 32 lane sums; the order is fixed, so the result is run-to-run identical
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  for (int c = warp; c < s.NL; c += nwarps) {
     double v = 0.0;
-    for (int b = 0; b < nblocks; ++b) v += partials[(size_t)b * s.NL + c];
-    s_tot[c] = v;
-    if (c < s.Ne) expert_psum[c] = (float)v;
-    else group_psum[c - s.Ne] = (float)v;
+    for (int b = lane; b < nblocks; b += 32) v += partials[(size_t)b * s.NL + c];
+    for (int m = 16; m > 0; m >>= 1) v += __shfl_xor_sync(kFull, v, m);
+    if (lane == 0) {
+      s_tot[c] = v;
+      if (c < s.Ne) expert_psum[c] = (float)v;
+      else group_psum[c - s.Ne] = (float)v;
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -451,7 +457,7 @@ int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs
     lp.w_over_wmax[g] = g < D.Ng ? (float)D.W[g] / (float)D.Wmax : 0.0f;
   RouterShape s1 = s;
   if (s1.T == 0) s1.T = 1;   // empty batch: sums are zero, avoid 0/0 in the loss
-  aux_finalize_kernel<<<1, 320, 0, st>>>(s1, lp, blocks, partials, group_count, cnt_routed, cnt_lit,
+  aux_finalize_kernel<<<1, 1024, 0, st>>>(s1, lp, blocks, partials, group_count, cnt_routed, cnt_lit,
                                          group_psum, expert_psum, loss_out);
   MOHGE_LAUNCH_CHECK("aux_finalize_kernel");
   return MOHGE_OK;
