@@ -198,12 +198,30 @@ __device__ __forceinline__ Vec16 pack(const float (&f)[8], float) {
   return a;
 }
 
+// Zeroes a quarter (`part` of 4) of the padding rows [aligned[e] + counts[e], aligned[e+1]) of a
+// permuted buffer.  The row movers run 4 * N_e extra blocks that do this, so no launch of its own.
+__device__ __forceinline__ void zero_pad_part(const int32_t* __restrict__ counts,
+                                              const int32_t* __restrict__ aligned, int e, int part,
+                                              int row_vecs, Vec16* __restrict__ buf) {
+  const int r0 = aligned[e] + counts[e], r1 = aligned[e + 1];
+  const Vec16 z = {{0, 0, 0, 0}};
+  const size_t n = (size_t)(r1 - r0) * row_vecs;
+  Vec16* p = buf + (size_t)r0 * row_vecs;
+  for (size_t i = (size_t)part * blockDim.x + threadIdx.x; i < n; i += (size_t)4 * blockDim.x) p[i] = z;
+}
+
 // x_perm[prow_of[t,k], :] = x[t, :]   (row_vecs 16-byte vectors per row)
 __global__ void __launch_bounds__(256)
 permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ prow_of, int T, int Ke,
-                    int row_vecs, int rows_cap, Vec16* __restrict__ x_perm) {
+                    int row_vecs, int rows_cap, Vec16* __restrict__ x_perm, int nb_tok,
+                    const int32_t* __restrict__ counts, const int32_t* __restrict__ aligned) {
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
-  for (int t = blockIdx.x; t < T; t += gridDim.x) {
+  if ((int)blockIdx.x >= nb_tok) {      // padding rows (launched only when segments are aligned)
+    const int j = blockIdx.x - nb_tok;
+    zero_pad_part(counts, aligned, j >> 2, j & 3, row_vecs, x_perm);
+    return;
+  }
+  for (int t = blockIdx.x; t < T; t += nb_tok) {
     __syncthreads();
     if (threadIdx.x < Ke) s_row[threadIdx.x] = prow_of[(size_t)t * Ke + threadIdx.x];
     __syncthreads();
@@ -270,12 +288,18 @@ __global__ void __launch_bounds__(256)
 combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_perm,
                    const int32_t* __restrict__ prow_of, const float* __restrict__ gate_w, int Tn,
                    int Ke, int row_vecs, int rows_cap, Vec16* __restrict__ dy_perm,
-                   float* __restrict__ dgate_w) {
+                   float* __restrict__ dgate_w, int nb_tok, const int32_t* __restrict__ counts,
+                   const int32_t* __restrict__ aligned) {
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_red[MOHGE_MAX_K_EXPERTS][8];
+  if ((int)blockIdx.x >= nb_tok) {      // padding rows of dy_perm
+    const int j = blockIdx.x - nb_tok;
+    zero_pad_part(counts, aligned, j >> 2, j & 3, row_vecs, dy_perm);
+    return;
+  }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  for (int t = blockIdx.x; t < Tn; t += gridDim.x) {
+  for (int t = blockIdx.x; t < Tn; t += nb_tok) {
     __syncthreads();
     if (threadIdx.x < Ke) {
       s_row[threadIdx.x] = prow_of[(size_t)t * Ke + threadIdx.x];
@@ -340,13 +364,10 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
   MOHGE_LAUNCH_CHECK("dispatch_scatter_kernel");
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
-  permute_rows_kernel<<<blocks, block_for(row_vecs), 0, st>>>(
-      (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)x_perm);
+  const int pad_blocks = D.align > 1 ? 4 * D.Ne : 0;
+  permute_rows_kernel<<<blocks + pad_blocks, block_for(row_vecs), 0, st>>>(
+      (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)x_perm, blocks, counts, aligned);
   MOHGE_LAUNCH_CHECK("permute_rows_kernel");
-  if (D.align > 1) {
-    zero_pad_rows_kernel<<<dim3(D.Ne, 4), 256, 0, st>>>(counts, aligned, row_vecs, (Vec16*)x_perm);
-    MOHGE_LAUNCH_CHECK("zero_pad_rows_kernel");
-  }
   return MOHGE_OK;
 }
 
@@ -378,19 +399,20 @@ int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
                            const int32_t* aligned, void* dy_perm, float* dgate_w, cudaStream_t st) {
   const int T = (int)D.T;
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
+  const int pad_blocks = D.align > 1 ? 4 * D.Ne : 0;
   if (T > 0) {
     const int blocks = T < 148 * 16 ? T : 148 * 16;
     if (D.bf16)
-      combine_bwd_kernel<__nv_bfloat16><<<blocks, block_for(row_vecs), 0, st>>>(
+      combine_bwd_kernel<__nv_bfloat16><<<blocks + pad_blocks, block_for(row_vecs), 0, st>>>(
           (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
-          (Vec16*)dy_perm, dgate_w);
+          (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
     else
-      combine_bwd_kernel<float><<<blocks, block_for(row_vecs), 0, st>>>(
+      combine_bwd_kernel<float><<<blocks + pad_blocks, block_for(row_vecs), 0, st>>>(
           (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
-          (Vec16*)dy_perm, dgate_w);
+          (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
     MOHGE_LAUNCH_CHECK("combine_bwd_kernel");
   }
-  if (D.align > 1) {
+  if (D.align > 1 && T == 0) {
     zero_pad_rows_kernel<<<dim3(D.Ne, 4), 256, 0, st>>>(counts, aligned, row_vecs, (Vec16*)dy_perm);
     MOHGE_LAUNCH_CHECK("zero_pad_rows_kernel");
   }

@@ -164,6 +164,17 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
   }
 }
 
+// the three count arrays start at zero (one launch instead of three memsets)
+__global__ void zero_counts_kernel(int32_t* group_count, int Ng, int32_t* cnt_routed, int32_t* cnt_lit,
+                                   int Ne) {
+  for (int i = threadIdx.x; i < Ne; i += blockDim.x) {
+    cnt_routed[i] = 0;
+    cnt_lit[i] = 0;
+    if (i < Ng) group_count[i] = 0;
+  }
+  for (int i = Ne + threadIdx.x; i < Ng; i += blockDim.x) group_count[i] = 0;
+}
+
 // ---------------------------------------------------------------- statistics (Eq. 7-14)
 constexpr int kStatsThreads = 256;
 constexpr int kStatsWarps = kStatsThreads / 32;
@@ -438,9 +449,8 @@ int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs
                          float* group_psum, int32_t* cnt_routed, int32_t* cnt_lit,
                          float* expert_psum, float* loss_out, double* partials, cudaStream_t st) {
   const RouterShape s = make_shape(D);
-  MOHGE_CUDA(cudaMemsetAsync(group_count, 0, sizeof(int32_t) * D.Ng, st));
-  MOHGE_CUDA(cudaMemsetAsync(cnt_routed, 0, sizeof(int32_t) * D.Ne, st));
-  MOHGE_CUDA(cudaMemsetAsync(cnt_lit, 0, sizeof(int32_t) * D.Ne, st));
+  zero_counts_kernel<<<1, 256, 0, st>>>(group_count, D.Ng, cnt_routed, cnt_lit, D.Ne);
+  MOHGE_LAUNCH_CHECK("zero_counts_kernel");
   int blocks = ceil_div(D.T, kStatsWarps);
   if (blocks > kStatsBlocks) blocks = kStatsBlocks;
   if (blocks > 0) {
