@@ -329,6 +329,23 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes,
 // division sequence would cost more than the tile's MMAs.  exp overflow gives 1/inf = 0.
 __device__ __forceinline__ float sigmoid_fast(float a) { return __fdividef(1.0f, 1.0f + __expf(-a)); }
 __device__ __forceinline__ float silu_fast(float a) { return __fdividef(a, 1.0f + __expf(-a)); }
+// Two elements at a time with the packed FP32 instructions of sm_100 (one issue slot for both
+// lanes of a multiply, add or fused multiply-add); exp2 and reciprocal stay scalar.
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float2 sigmoid2_fast(float2 a) {
+  const float2 t = __fmul2_rn(a, make_float2(-1.4426950408889634f, -1.4426950408889634f));
+  const float2 den = __fadd2_rn(make_float2(ex2_approx(t.x), ex2_approx(t.y)), make_float2(1.0f, 1.0f));
+  return make_float2(rcp_approx(den.x), rcp_approx(den.y));
+}
 
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
   const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -729,8 +746,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               for (int e2 = 0; e2 < 4; ++e2) {
                 const float a0 = __uint_as_float(ra[j4 * 8 + 2 * e2]), a1 = __uint_as_float(ra[j4 * 8 + 2 * e2 + 1]);
                 const float u0 = __uint_as_float(ru[j4 * 8 + 2 * e2]), u1 = __uint_as_float(ru[j4 * 8 + 2 * e2 + 1]);
-                const float h0 = silu_fast(a0) * u0, h1 = silu_fast(a1) * u1;
-                pa[e2] = pack2(a0, a1); pu[e2] = pack2(u0, u1); ph[e2] = pack2(h0, h1);
+                const float2 a2 = make_float2(a0, a1), u2 = make_float2(u0, u1);
+                const float2 h2 = __fmul2_rn(__fmul2_rn(a2, sigmoid2_fast(a2)), u2);   // silu(a) * u
+                pa[e2] = pack2(a0, a1); pu[e2] = pack2(u0, u1); ph[e2] = pack2(h2.x, h2.y);
               }
               st_shared_v4(stg_addr(bA, lane, hh * 4 + j4), pa[0], pa[1], pa[2], pa[3]);
               st_shared_v4(stg_addr(bU, lane, hh * 4 + j4), pu[0], pu[1], pu[2], pu[3]);
@@ -804,9 +822,16 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               for (int e2 = 0; e2 < 4; ++e2) {
                 const float a0 = bf_lo(wa[e2]), a1 = bf_hi(wa[e2]), u0 = bf_lo(wu[e2]), u1 = bf_hi(wu[e2]);
                 const float dh0 = __uint_as_float(r[j4 * 8 + 2 * e2]), dh1 = __uint_as_float(r[j4 * 8 + 2 * e2 + 1]);
-                const float s0 = sigmoid_fast(a0), s1 = sigmoid_fast(a1);
-                oa[e2] = pack2(dh0 * u0 * s0 * (1.0f + a0 * (1.0f - s0)), dh1 * u1 * s1 * (1.0f + a1 * (1.0f - s1)));
-                ou[e2] = pack2(dh0 * a0 * s0, dh1 * a1 * s1);
+                const float2 a2 = make_float2(a0, a1), u2 = make_float2(u0, u1), dh2 = make_float2(dh0, dh1);
+                const float2 one = make_float2(1.0f, 1.0f);
+                const float2 s2 = sigmoid2_fast(a2);
+                const float2 oms = __ffma2_rn(s2, make_float2(-1.0f, -1.0f), one);      // 1 - s
+                const float2 t2 = __ffma2_rn(a2, oms, one);                             // 1 + a (1 - s)
+                const float2 dhs = __fmul2_rn(dh2, s2);
+                const float2 du2 = __fmul2_rn(dhs, a2);                                 // dh * silu(a)
+                const float2 da2 = __fmul2_rn(__fmul2_rn(dhs, u2), t2);                 // dh * u * silu'(a)
+                oa[e2] = pack2(da2.x, da2.y);
+                ou[e2] = pack2(du2.x, du2.y);
               }
               st_shared_v4(aa, oa[0], oa[1], oa[2], oa[3]);
               st_shared_v4(ua, ou[0], ou[1], ou[2], ou[3]);
