@@ -739,20 +739,23 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             tmem_ld32(taddr + c + 32 * hh, ra);
             tmem_ld32(taddr + half + c + 32 * hh, ru);
             tmem_ld_wait();
+            uint32_t pa[4][4], pu[4][4], ph[4][4];       // arithmetic first, then the stores
 #pragma unroll
             for (int j4 = 0; j4 < 4; ++j4) {
-              uint32_t pa[4], pu[4], ph[4];
 #pragma unroll
               for (int e2 = 0; e2 < 4; ++e2) {
                 const float a0 = __uint_as_float(ra[j4 * 8 + 2 * e2]), a1 = __uint_as_float(ra[j4 * 8 + 2 * e2 + 1]);
                 const float u0 = __uint_as_float(ru[j4 * 8 + 2 * e2]), u1 = __uint_as_float(ru[j4 * 8 + 2 * e2 + 1]);
                 const float2 a2 = make_float2(a0, a1), u2 = make_float2(u0, u1);
                 const float2 h2 = __fmul2_rn(__fmul2_rn(a2, sigmoid2_fast(a2)), u2);   // silu(a) * u
-                pa[e2] = pack2(a0, a1); pu[e2] = pack2(u0, u1); ph[e2] = pack2(h2.x, h2.y);
+                pa[j4][e2] = pack2(a0, a1); pu[j4][e2] = pack2(u0, u1); ph[j4][e2] = pack2(h2.x, h2.y);
               }
-              st_shared_v4(stg_addr(bA, lane, hh * 4 + j4), pa[0], pa[1], pa[2], pa[3]);
-              st_shared_v4(stg_addr(bU, lane, hh * 4 + j4), pu[0], pu[1], pu[2], pu[3]);
-              st_shared_v4(stg_addr(bH, lane, hh * 4 + j4), ph[0], ph[1], ph[2], ph[3]);
+            }
+#pragma unroll
+            for (int j4 = 0; j4 < 4; ++j4) {
+              st_shared_v4(stg_addr(bA, lane, hh * 4 + j4), pa[j4][0], pa[j4][1], pa[j4][2], pa[j4][3]);
+              st_shared_v4(stg_addr(bU, lane, hh * 4 + j4), pu[j4][0], pu[j4][1], pu[j4][2], pu[j4][3]);
+              st_shared_v4(stg_addr(bH, lane, hh * 4 + j4), ph[j4][0], ph[j4][1], ph[j4][2], ph[j4][3]);
             }
           }
           fence_async_smem();
@@ -807,22 +810,31 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           const bool in_ok = mbar_wait(ein_bar(quad, set), (n_chunk >> 1) & 1u, abort_flag, p.status, 5);
           if (!__all_sync(0xffffffffu, in_ok)) { alive = false; break; }
           const uint32_t bA = stg + set * 2 * kStgBufBytes, bU = bA + kStgBufBytes;
+          // both halves of the chunk leave tensor memory while the shared-memory reads are issued;
+          // loads, arithmetic and stores are grouped so that the single warp has independent work
+          uint32_t r[2][32];
+          tmem_ld32(taddr + c, r[0]);
+          tmem_ld32(taddr + c + 32, r[1]);
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            uint32_t r[32];
-            tmem_ld32(taddr + c + 32 * hh, r);
-            tmem_ld_wait();
+            uint4 va[4], vu[4];
 #pragma unroll
             for (int j4 = 0; j4 < 4; ++j4) {
-              const uint32_t aa = stg_addr(bA, lane, hh * 4 + j4), ua = stg_addr(bU, lane, hh * 4 + j4);
-              const uint4 va = ld_shared_v4(aa), vu = ld_shared_v4(ua);
-              const uint32_t wa[4] = {va.x, va.y, va.z, va.w}, wu[4] = {vu.x, vu.y, vu.z, vu.w};
-              uint32_t oa[4], ou[4];
+              va[j4] = ld_shared_v4(stg_addr(bA, lane, hh * 4 + j4));
+              vu[j4] = ld_shared_v4(stg_addr(bU, lane, hh * 4 + j4));
+            }
+            if (hh == 0) tmem_ld_wait();
+            uint32_t oa[4][4], ou[4][4];
+#pragma unroll
+            for (int j4 = 0; j4 < 4; ++j4) {
+              const uint32_t wa[4] = {va[j4].x, va[j4].y, va[j4].z, va[j4].w};
+              const uint32_t wu[4] = {vu[j4].x, vu[j4].y, vu[j4].z, vu[j4].w};
 #pragma unroll
               for (int e2 = 0; e2 < 4; ++e2) {
-                const float a0 = bf_lo(wa[e2]), a1 = bf_hi(wa[e2]), u0 = bf_lo(wu[e2]), u1 = bf_hi(wu[e2]);
-                const float dh0 = __uint_as_float(r[j4 * 8 + 2 * e2]), dh1 = __uint_as_float(r[j4 * 8 + 2 * e2 + 1]);
-                const float2 a2 = make_float2(a0, a1), u2 = make_float2(u0, u1), dh2 = make_float2(dh0, dh1);
+                const float2 a2 = make_float2(bf_lo(wa[e2]), bf_hi(wa[e2]));
+                const float2 u2 = make_float2(bf_lo(wu[e2]), bf_hi(wu[e2]));
+                const float2 dh2 = make_float2(__uint_as_float(r[hh][j4 * 8 + 2 * e2]),
+                                               __uint_as_float(r[hh][j4 * 8 + 2 * e2 + 1]));
                 const float2 one = make_float2(1.0f, 1.0f);
                 const float2 s2 = sigmoid2_fast(a2);
                 const float2 oms = __ffma2_rn(s2, make_float2(-1.0f, -1.0f), one);      // 1 - s
@@ -830,11 +842,14 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
                 const float2 dhs = __fmul2_rn(dh2, s2);
                 const float2 du2 = __fmul2_rn(dhs, a2);                                 // dh * silu(a)
                 const float2 da2 = __fmul2_rn(__fmul2_rn(dhs, u2), t2);                 // dh * u * silu'(a)
-                oa[e2] = pack2(da2.x, da2.y);
-                ou[e2] = pack2(du2.x, du2.y);
+                oa[j4][e2] = pack2(da2.x, da2.y);
+                ou[j4][e2] = pack2(du2.x, du2.y);
               }
-              st_shared_v4(aa, oa[0], oa[1], oa[2], oa[3]);
-              st_shared_v4(ua, ou[0], ou[1], ou[2], ou[3]);
+            }
+#pragma unroll
+            for (int j4 = 0; j4 < 4; ++j4) {
+              st_shared_v4(stg_addr(bA, lane, hh * 4 + j4), oa[j4][0], oa[j4][1], oa[j4][2], oa[j4][3]);
+              st_shared_v4(stg_addr(bU, lane, hh * 4 + j4), ou[j4][0], ou[j4][1], ou[j4][2], ou[j4][3]);
             }
           }
           fence_async_smem();
