@@ -59,7 +59,7 @@ template <int CG, int WIDE = 0> struct Geo {
   static constexpr int kStages = (CG == 2 && !WIDE) ? 5 : 3;
   static constexpr int kBBytes = 256 / CG * BK * 2;          // one B tile per CTA: 32 KiB or 16 KiB
   static constexpr int kStageBytes = kABytes + kBBytes * (WIDE ? 2 : 1);
-  static constexpr int kSmemBytes = kStages * kStageBytes + kStgBytes + 1024 + 512;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kStgBytes + 1024 + 512 + 1088;   // + segment table
   static constexpr int kTileM = BM * CG;
 };
 
@@ -410,7 +410,7 @@ __device__ __forceinline__ Tile fetch_tile(const TcParams& p, int ti) {
 }
 
 template <int ROLE>
-__device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) {
+__device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t, const int32_t* seg) {
   TileGeom q;
   if (is_plain<ROLE>()) {
     q.e = t.e; q.g = 0; q.i = 0; q.W = 0; q.bn = p.BN[0]; q.m0 = t.m0; q.n0 = t.n0; q.wide = 0;
@@ -434,7 +434,7 @@ __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t) 
   else if (ROLE == ROLE_DGRAD_13) q.num_kb = (2 * q.W + BK - 1) / BK;
   else {
     q.num_kb = t.ext / BK;
-    q.r0 = p.aligned[t.e];
+    q.r0 = seg[t.e];          // first physical row of the expert (table staged in shared memory)
   }
   return q;
 }
@@ -462,6 +462,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   auto ein_bar = [&](int quad, int set) { return bar0 + 8u * (2 * kStages + 4 + quad * 2 + set); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 12);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // expert segment table (aligned_offsets) staged once, so that no role chases it through global
+  // memory between tiles
+  int32_t* s_seg = reinterpret_cast<int32_t*>(smem_gen + kStages * kStageBytes + kStgBytes + 512);
+  if (!is_plain<ROLE>()) {
+    const int ne = p.gs.Ng * p.gs.N;
+    for (int i = threadIdx.x; i <= ne; i += blockDim.x) s_seg[i] = p.aligned[i];
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -504,6 +511,16 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   const int rounds = (total + unit_stride - 1) / unit_stride;
   // loop variable: the round when zigzag, else the tile index itself
   const int it0 = zigzag ? 0 : unit, it_step = zigzag ? 1 : unit_stride, it_end = zigzag ? rounds : total;
+  // The list entry of the NEXT tile is requested while the current one is worked on: a tile of a
+  // short contraction lasts a few thousand clocks, and a dependent global load in front of each
+  // one kept the MMA issuer idle for a quarter of that.
+  auto prefetch_tile = [&](int it) -> Tile {
+    Tile z;
+    z.e = 0; z.m0 = 0; z.n0 = 0; z.ext = 0;
+    if (it >= it_end) return z;
+    const int ti = zigzag ? tile_of(it) : it;
+    return ti < 0 ? z : fetch_tile<ROLE>(p, ti);
+  };
 
   if (warp == 0) {
     // ================= TMA producer =================
@@ -511,11 +528,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
+      Tile t_pf = prefetch_tile(it0);
       for (int it = it0; it < it_end && alive; it += it_step) {
         const int ti = zigzag ? tile_of(it) : it;
+        const Tile t = t_pf;
+        t_pf = prefetch_tile(it + it_step);
         if (ti < 0) continue;
-        const Tile t = fetch_tile<ROLE>(p, ti);
-        const TileGeom q = tile_geom<ROLE>(p, t);
+        const TileGeom q = tile_geom<ROLE>(p, t, s_seg);
         const CUtensorMap* mA = &p.mapA[q.g];
         const CUtensorMap* mB = &p.mapB[q.g];
         const int nb = q.bn / CG;                          // B rows staged by this CTA per B tile
@@ -592,11 +611,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       };
       auto free_stage = [&](int st) { if (CG == 2) umma2_commit(empty_bar(st)); else umma_commit(empty_bar(st)); };
       auto acc_done = [&](int b) { if (CG == 2) umma2_commit(tfull_bar(b)); else umma_commit(tfull_bar(b)); };
+      Tile t_pf = prefetch_tile(it0);
       for (int it = it0; it < it_end && alive; it += it_step) {
         const int ti = zigzag ? tile_of(it) : it;
+        const Tile t = t_pf;
+        t_pf = prefetch_tile(it + it_step);
         if (ti < 0) continue;
-        const Tile t = fetch_tile<ROLE>(p, ti);
-        const TileGeom q = tile_geom<ROLE>(p, t);
+        const TileGeom q = tile_geom<ROLE>(p, t, s_seg);
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
                                ((uint32_t)RT::B_MN << 16) | ((uint32_t)(q.bn >> 3) << 17) |
                                ((uint32_t)(G::kTileM >> 4) << 24);
@@ -672,11 +693,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     int buf = 0;
     uint32_t acc_phase = 0;
     bool alive = true;
+    Tile t_pf = prefetch_tile(it0);
     for (int it = it0; it < it_end && alive; it += it_step) {
       const int ti = zigzag ? tile_of(it) : it;
+      const Tile t = t_pf;
+      t_pf = prefetch_tile(it + it_step);
       if (ti < 0) continue;
-      const Tile t = fetch_tile<ROLE>(p, ti);
-      TileGeom q = tile_geom<ROLE>(p, t);
+      TileGeom q = tile_geom<ROLE>(p, t, s_seg);
       // a double-width entry is drained as two pieces, one accumulator buffer each
       const int pieces = (WIDE && q.wide) ? 2 : 1;
       for (int pc = 0; pc < pieces && alive; ++pc) {
@@ -724,7 +747,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       int next_kb = 0;
       if ((RT::EPI == EPI_BF16 || RT::EPI == EPI_F32) && !(WIDE && q.wide) && it + it_step < it_end &&
           (zigzag ? tile_of(it + 1) : it + it_step) >= 0)
-        next_kb = tile_geom<ROLE>(p, fetch_tile<ROLE>(p, zigzag ? tile_of(it + 1) : it + it_step)).num_kb;
+        next_kb = tile_geom<ROLE>(p, t_pf, s_seg).num_kb;
       if (RT::EPI == EPI_SWIGLU_FWD) {
         const int half = q.bn >> 1;
         for (int c = 0; rows_ok && c < half && q.n0 + c < q.W; c += 64) {
@@ -1058,14 +1081,16 @@ int32_t encode_stage_map_f32(CUtensorMap* m, const void* base, uint64_t cols, ui
   return encode_map(m, base, 3, dims, str, box, true);
 }
 
-// Tile width per group: among the candidates the one that wastes the fewest padded columns
-// (ties go to the wider tile, which keeps the tensor pipe busier per shared-memory byte).
+// Tile width per group.  Candidates come widest first.  A narrower tile is taken only when it
+// cuts the padded extent by more than a fifth: a 128-wide tile needs half again as many operand
+// bytes per FLOP as a 256-wide one, which costs more than a few percent of padded columns
+// (measured: hidden width 1408 as 11 x 128 ran 27 % slower than as 6 x 256 with 8 % padding).
 int pick_bn(int extent, const int* cand, int ncand) {
   int best = cand[0];
-  long long best_pad = -1;
-  for (int c = 0; c < ncand; ++c) {
+  long long best_pad = (long long)((extent + cand[0] - 1) / cand[0]) * cand[0];
+  for (int c = 1; c < ncand; ++c) {
     const long long pad = (long long)((extent + cand[c] - 1) / cand[c]) * cand[c];
-    if (best_pad < 0 || pad < best_pad) {
+    if (pad * 5 < best_pad * 4) {
       best_pad = pad;
       best = cand[c];
     }
