@@ -1245,7 +1245,7 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
       const int32_t rc2 = launch_role<ROLE_ROUTER_DW, 1>(p, grid, st);
       if (rc2 || p.plain_splits == 1) return rc2;
       const size_t n = (size_t)D.NL * D.d;
-      sum_partials_kernel<<<(unsigned)((n + 1023) / 1024), 256, 0, st>>>(partials, p.plain_splits, n, (float*)C);
+      sum_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partials, p.plain_splits, n, (float*)C);
       MOHGE_LAUNCH_CHECK("sum_partials_kernel");
       return MOHGE_OK;
     }
