@@ -7,13 +7,14 @@
 //   warps 2..5  epilogue: tcgen05.ld -> registers -> fused element-wise math -> swizzled staging
 //               buffers in shared memory -> TMA stores (every global write of the expert roles is
 //               a full 128-byte row piece; the SwiGLU backward also reads A and U through TMA)
-// One persistent CTA per SM walks the device-built, cost-sorted tile list with stride gridDim.x.
+// One persistent CTA per SM (a CTA pair per two SMs for the expert roles) walks the device-built,
+// cost-sorted tile list with a fixed stride, in alternating directions when tile costs differ.
 //
 // Six roles share the kernel (C = A . B^T over a contraction index k):
 //   FWD1        [A | U] = Xp . W13^T, fused SwiGLU epilogue writes A, U and H = silu(A) * U.
-//               The gate tile and the up tile of the same hidden columns are two TMA boxes that
-//               land back to back in shared memory, so ONE 128 x (2*BNh) MMA covers both and no
-//               weight repacking is needed.
+//               The gate tile and the up tile of the same hidden columns are two TMA boxes (one
+//               per CTA of a pair) that form one B operand, so ONE MMA covers both and no weight
+//               repacking is needed.
 //   FWD2        Yp = H . W2^T
 //   DGRAD_DOWN  dH = dYp . W2         (B read MN-major), epilogue turns dH into dA, dU using A, U
 //   DGRAD_13    dXp = [dA | dU] . W13 (B read MN-major)
@@ -22,7 +23,7 @@
 // Expert segments start at multiples of 128 physical rows with zero padding rows, so a 128-row
 // tile never straddles two experts and padding contributes exact zeros to the weight gradients.
 // Hidden widths that are not multiples of the tile are handled by TMA's out-of-bounds zero fill
-// on loads and by column masks on stores.
+// on loads and by the clipping of TMA stores.
 //
 // Every wait is bounded: after about one second without progress the waiting thread records
 // (1 << 24 | site) in the status word, raises a CTA-wide abort flag and every role leaves its
@@ -43,7 +44,7 @@ constexpr int kAccCols = 256;                 // tensor-memory columns per accum
 
 // CG = CTAs per MMA (tcgen05 cta_group).  CG = 2 pairs the two CTAs of a cluster on one
 // 256 x N tile: each CTA stages its own 128 rows of A and HALF of B, so operand traffic per FLOP
-// drops by a third and the smaller stages allow a six-deep pipeline.
+// drops by a third and the smaller stages allow a five-deep pipeline.
 // Epilogue staging: each of the four epilogue warps owns a ring of four 4 KiB buffers
 // (32 rows x 128 bytes, 128-byte swizzle: the layout a TMA box of 32 rows expects).
 constexpr int kStgBufBytes = 4096;
