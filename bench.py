@@ -203,6 +203,10 @@ def main():
     ap.add_argument("--shared-width", type=int, default=0,
                     help="hidden width of the shared experts (N_s FFNs concatenated); 0 = none, "
                          "the benchmark configurations have none")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one step in a CUDA graph and time its replays (launch-bound small "
+                         "workloads); the GEMM share for the roofline object is then taken from a "
+                         "short eager loop before the timed region")
     args = ap.parse_args()
     if args.forward_only:          # the end-to-end and CPU arms describe the fwd+bwd step only
         args.no_e2e = args.no_cpu_baseline = True
@@ -295,16 +299,34 @@ def main():
         raise SystemExit("device status word = 0x%x after warm-up" % status)
     counts = buf.counts.cpu().tolist()
 
+    graph = None
+    if args.graph:
+        # every launch of the step depends on device data only through device memory, so one
+        # capture serves every later batch written into the same buffers
+        for _ in range(min(args.steps, 10)):
+            step(mark=True)
+        torch.cuda.synchronize()
+        l0 = B.mohge_launch_count()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step()
+        launches_per_replay = B.mohge_launch_count() - l0
+        for _ in range(3):
+            graph.replay()
+
     sampler = ClockSampler(local_rank) if rank == 0 else None
     l0 = B.mohge_launch_count()
     barrier()
     t_start, t_end = ev(), ev()
     t_start.record()
     for _ in range(args.steps):
-        step(mark=True)
+        if graph is not None:
+            graph.replay()
+        else:
+            step(mark=True)
     t_end.record()
     barrier()
-    launches = B.mohge_launch_count() - l0
+    launches = launches_per_replay * args.steps if graph is not None else B.mohge_launch_count() - l0
     clocks = sampler.stop() if sampler else None
     ms_total = t_start.elapsed_time(t_end)
     ms_total = max_over_ranks(ms_total, dist, dev)
@@ -429,7 +451,8 @@ def main():
                    "experts_per_group": wl.experts_per_group, "group_width": list(wl.group_width),
                    "k_groups": wl.k_groups, "k_experts": wl.k_experts, "shared_width": args.shared_width,
                    "pass": "forward only" if args.forward_only else "forward + backward",
-                   "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only"},
+                   "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only",
+                   "launch": "CUDA graph replay" if args.graph else "stream launches"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
         "roofline": roofline, "cpu_baseline": cpu_baseline,
     }
