@@ -1161,10 +1161,16 @@ bool wide_tiles(const Dims& D, int role) {
   return den > 0.0 && num / den >= kWideMinK;
 }
 
-// CTAs per MMA for the grouped roles (debugging switch MOHGE_TC_CG=1 keeps the single-CTA form)
-int cta_group_size() {
+// CTAs per MMA for the grouped roles.  CTA pairs (256-row tiles, each CTA fetching half of B)
+// serve batches whose experts fill such tiles.  When an expert receives 128 rows or fewer on
+// average the GEMMs are bound by reading the weights once: a pair would spend half of its MMAs
+// and A loads on rows of the next expert, so single CTAs with 128-row tiles run instead (measured
+// 5.6 against 4.9 TB/s of weight traffic at 16 rows per expert).  MOHGE_TC_CG=1|2 forces a form.
+int cta_group_size(const Dims& D) {
   const char* e = getenv("MOHGE_TC_CG");
-  return (e && e[0] == '1') ? 1 : 2;
+  if (e && e[0] == '1') return 1;
+  if (e && e[0] == '2') return 2;
+  return D.R <= 128 * (int64_t)D.Ne ? 1 : 2;
 }
 
 }  // namespace
@@ -1265,7 +1271,7 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
 // choices launch_tc_grouped makes, so that the lists of several roles can be built by one launch
 // before the GEMMs run.
 TilePlan tc_tile_plan(const Dims& D, int role) {
-  const int CG = cta_group_size();
+  const int CG = cta_group_size(D);
   const int cand_n[2] = {256, 128};
   const int cand_h[2] = {128, 64};
   int bn_plan[MOHGE_MAX_GROUPS];
@@ -1307,7 +1313,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   p.accumulate = accumulate; p.status = status;
 
   const uint64_t d = D.d, rows = D.Rcap, pitchAU = 2ull * D.Wmax * 2, pitchH = (uint64_t)D.Wmax * 2;
-  const int CG = cta_group_size();
+  const int CG = cta_group_size(D);
   // UMMA N candidates: multiples of 128 so that a CTA pair's half of an MN-major B stays a
   // multiple of the 64-element swizzle block and the epilogue's 64-column boxes tile the width.
   const int cand_n[2] = {256, 128};

@@ -113,14 +113,18 @@ def test_out_of_range_expert_index_sets_the_status_word_without_faulting():
     assert int(b.counts.sum()) == 127
 
 
-@pytest.mark.parametrize("switch", ["MOHGE_TC_WIDE=63", "MOHGE_TC_WIDE=0", "MOHGE_TC_CG=1"])
+@pytest.mark.parametrize("switch", ["MOHGE_TC_CG=2,MOHGE_TC_WIDE=63", "MOHGE_TC_CG=2,MOHGE_TC_WIDE=0",
+                                    "MOHGE_TC_CG=1"])
 def test_every_form_of_the_grouped_gemm_on_small_ragged_cases(switch, monkeypatch):
     """The double-width form is chosen by default only for long contractions (the large
-    workload); here it is forced on small ragged shapes, as are the single-width and the
-    single-CTA forms, so that every kernel form meets odd widths, ragged tails and empty experts."""
-    name, value = switch.split("=")
-    monkeypatch.setenv(name, value)
+    workload) and single CTAs only for batches with few rows per expert; here each form is forced
+    on small ragged shapes, so that every kernel form meets odd widths, ragged tails, empty experts
+    and both a few and a few hundred rows per expert."""
+    for kv in switch.split(","):
+        name, value = kv.split("=")
+        monkeypatch.setenv(name, value)
     for wl in (Workload("forms_a", "bf16", 1000, 256, 3, 4, (352, 176, 88), 2, 4, seed=1),
+               Workload("forms_few", "bf16", 90, 256, 3, 4, (352, 176, 88), 2, 4, seed=2),
                Workload("forms_b", "bf16", 1500, 256, 4, 8, (256, 192, 128, 64), 2, 6,
                         zipf_beta=3.0, seed=5)):
         inp = make_inputs(wl)
