@@ -111,9 +111,12 @@ dispatch_scatter_kernel(const int32_t* __restrict__ expert_idx, int T, int Ke, i
   __shared__ int s_wcnt[kChunkWarps][256];
   __shared__ int s_start[256];     // dense row of the chunk's first token for expert e
   __shared__ int s_pstart[256];    // same in physical numbering
+  __shared__ unsigned s_set[kChunkWarps][32][8];   // expert set of every token of the chunk
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = blockIdx.x * kDispatchChunk + threadIdx.x;
   const ExpertSet s = load_set(expert_idx, t, T, Ke, Ne, status);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) s_set[warp][lane][i] = s.w[i];
   warp_counts(s, Ne, lane, s_wcnt[warp]);
   __syncthreads();
   for (int e = threadIdx.x; e < Ne; e += blockDim.x) {
@@ -129,30 +132,20 @@ dispatch_scatter_kernel(const int32_t* __restrict__ expert_idx, int T, int Ke, i
     s_pstart[e] = aligned[e] + b;
   }
   __syncthreads();
-  const unsigned lt = (1u << lane) - 1u;
-  // Rank inside the warp: for slot k every lane holds one expert e; the lanes below it whose
-  // token is also routed to e (in any slot) come first.  The membership ballots are gathered
-  // once per distinct e of the warp; every lane takes part in every ballot (lanes past T hold
-  // empty sets and e = -1).
+  // Rank inside the warp: the lanes below this one whose token is also routed to e (in any
+  // slot) come first; their membership bits are read from the sets the warp left in shared
+  // memory (lanes past T left empty sets).
   for (int k = 0; k < Ke; ++k) {
     int e = t < T ? expert_idx[(size_t)t * Ke + k] : -1;
     if (e >= Ne) e = -1;
-    unsigned todo = __ballot_sync(kFull, e >= 0);
-    unsigned bal = 0;
-    while (todo) {
-      const int leader = __ffs(todo) - 1;
-      const int el = __shfl_sync(kFull, e, leader);
-      unsigned member = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i)
-        if ((el >> 5) == i) member = (s.w[i] >> (el & 31)) & 1u;
-      const unsigned b2 = __ballot_sync(kFull, member);
-      const unsigned same = __ballot_sync(kFull, e == el);
-      if (e == el) bal = b2;
-      todo &= ~same;
+    int below = 0;
+    if (e >= 0) {
+      const int wi = e >> 5, bi = e & 31;
+#pragma unroll 8
+      for (int l = 0; l < 31; ++l) below += l < lane ? (int)((s_set[warp][l][wi] >> bi) & 1u) : 0;
     }
     if (e >= 0) {
-      const int rank = s_wcnt[warp][e] + __popc(bal & lt);
+      const int rank = s_wcnt[warp][e] + below;
       const int row = s_start[e] + rank;
       row_of[(size_t)t * Ke + k] = row;
       prow_of[(size_t)t * Ke + k] = s_pstart[e] + rank;
