@@ -207,7 +207,7 @@ int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const voi
     REQ_PTR(x); REQ_PTR(w_router); REQ_PTR(logits_out); OPT_PTR(logit_bias);
     const int f32 = D.bf16 ? 0 : 1;
     if (D.bf16 && !force_simt())
-      rc = launch_tc_plain(D, ROLE_LOGITS, x, w_router, 0, logits_out, logit_bias, nullptr, carve(D, ws).status, st);
+      rc = launch_tc_plain(D, ROLE_LOGITS, x, w_router, 0, logits_out, logit_bias, carve(D, ws).rdw, carve(D, ws).status, st);
     else
       rc = launch_simt_plain((int)T, D.NL, D.d, x, f32, D.d, 1, w_router, f32, D.d, 1, logits_out, 1,
                              D.NL, logit_bias, 0, st);

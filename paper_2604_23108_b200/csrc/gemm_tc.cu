@@ -103,7 +103,7 @@ struct TcParams {
   int32_t* status;
   // plain roles: C[M, N] over contraction K; tile ti -> (ti / ntn, ti % ntn)
   int plain_total, plain_ntn, plain_M, plain_N, plain_K;
-  int plain_splits, plain_kchunk;   // split-K of ROUTER_DW: ranges of plain_kchunk k-blocks
+  int plain_splits, plain_kchunk;   // split-K of ROUTER_DW and LOGITS: ranges of plain_kchunk k-blocks
   float* Cf;                     // LOGITS: logits [T, NL]; ROUTER_DW: dw_router [NL, d]
   const float* bias;             // LOGITS: optional logit bias [NL]
 };
@@ -557,7 +557,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0);
             }
           } else {
-            tma_2d<CG>(sA, mA, fb, k0, am0);
+            tma_2d<CG>(sA, mA, fb, (is_plain<ROLE>() ? q.r0 : 0) + k0, am0);   // r0: split-K offset
           }
           for (int pc = 0; pc < pieces; ++pc) {
             const uint32_t sB = sA + kABytes + pc * G::kBBytes;
@@ -573,7 +573,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             } else {
               const int bn0 = q.n0 + pc * q.bn + nb * (int)cta_rank;   // this CTA's slice of the columns
               if (ROLE == ROLE_LOGITS) {
-                tma_2d<CG>(sB, mB, fb, k0, bn0);
+                tma_2d<CG>(sB, mB, fb, q.r0 + k0, bn0);
               } else if (ROLE == ROLE_FWD2) {
                 tma_3d<CG>(sB, mB, fb, k0, bn0, q.i);
               } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
@@ -910,9 +910,11 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           }
         }
       } else if (RT::EPI == EPI_LOGITS) {
-        // logits[t, n] = acc + bias[n]; NL is arbitrary, so stores are scalar and masked
-        const long long row = q.m0 + row_in_tile;
+        // logits[t, n] = acc + bias[n]; NL is arbitrary, so stores are scalar and masked.  Under
+        // split-K every split writes its partial sum and the bias is added when they are summed.
+        const long long row = q.m0 + row_in_tile + (long long)q.e * p.plain_M;
         const bool row_ok = row_in_tile < t.ext;
+        const float* bias = p.plain_splits == 1 ? p.bias : nullptr;
         for (int c = 0; c < q.bn; c += 32) {
           uint32_t r[32];
           tmem_ld32(taddr + c, r);
@@ -922,7 +924,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int n = q.n0 + c + j;
-              if (n < p.plain_N) po[n] = __uint_as_float(r[j]) + (p.bias ? p.bias[n] : 0.0f);
+              if (n < p.plain_N) po[n] = __uint_as_float(r[j]) + (bias ? bias[n] : 0.0f);
             }
           }
         }
@@ -1189,6 +1191,32 @@ sum_partials_kernel(const float* __restrict__ part, int splits, size_t n, float*
     out[i] = acc;
   }
 }
+// the same for [rows][n_cols] partials of the router logits, plus the bias of the column
+__global__ void __launch_bounds__(256)
+sum_partials_bias_kernel(const float* __restrict__ part, int splits, size_t n, int n_cols,
+                         const float* __restrict__ bias, float* __restrict__ out) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    float acc = part[i];
+    for (int s = 1; s < splits; ++s) acc += part[(size_t)s * n + i];
+    out[i] = bias ? acc + bias[i % n_cols] : acc;
+  }
+}
+
+// Split-K factor of the router-logits GEMM: a batch of a few hundred tokens has one or two row
+// tiles, so two CTAs would walk the whole contraction alone; the contraction is cut so that about
+// one CTA per SM works, as far as the partial-sum buffer (sized for the router weight gradient)
+// holds [splits][T][NL] floats.  1 = no split (every batch of a few thousand tokens or more).
+int router_logits_splits(const Dims& D, int n_tiles) {
+  const int64_t tiles = (int64_t)((D.T + BM - 1) / BM) * n_tiles;
+  const int64_t k_blocks = (D.d + BK - 1) / BK;
+  int64_t s = 148 / tiles;
+  const int64_t fit = (int64_t)router_dw_splits(D) * D.d / D.T;
+  if (s > fit) s = fit;
+  if (s > k_blocks) s = k_blocks;
+  if (s < 4) return 1;                                   // little to win, one more launch to pay
+  const int64_t chunk = (k_blocks + s - 1) / s;
+  return (int)((k_blocks + chunk - 1) / chunk);          // no split is empty
+}
 }  // namespace
 
 int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
@@ -1244,10 +1272,23 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
     p.plain_kchunk = (total_kb + p.plain_splits - 1) / p.plain_splits;
     if (p.plain_splits > 1) p.Cf = partials;
   }
+  if (role == ROLE_LOGITS && partials != nullptr) {
+    p.plain_splits = router_logits_splits(D, p.plain_ntn);
+    p.plain_kchunk = (total_kb + p.plain_splits - 1) / p.plain_splits;
+    if (p.plain_splits > 1) p.Cf = partials;
+  }
   p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn * p.plain_splits;
   const int grid = p.plain_total < sm_count ? p.plain_total : sm_count;
   switch (role) {
-    case ROLE_LOGITS: return launch_role<ROLE_LOGITS, 1>(p, grid, st);
+    case ROLE_LOGITS: {
+      const int32_t rc2 = launch_role<ROLE_LOGITS, 1>(p, grid, st);
+      if (rc2 || p.plain_splits == 1) return rc2;
+      const size_t n = (size_t)D.T * D.NL;
+      sum_partials_bias_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partials, p.plain_splits, n, D.NL,
+                                                                           bias, (float*)C);
+      MOHGE_LAUNCH_CHECK("sum_partials_bias_kernel");
+      return MOHGE_OK;
+    }
     case ROLE_ROUTER_DW: {
       const int32_t rc2 = launch_role<ROLE_ROUTER_DW, 1>(p, grid, st);
       if (rc2 || p.plain_splits == 1) return rc2;

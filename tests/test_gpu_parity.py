@@ -26,6 +26,9 @@ CASES = {
     "bf16_paper_shape": Workload("bf16_paper_shape", "bf16", 600, 256, 8, 4,
                                  (64, 80, 96, 128, 160, 192, 208, 224), 3, 6, seed=4),
     "bf16_odd_d": Workload("bf16_odd_d", "bf16", 500, 200, 2, 4, (72, 40), 1, 3, seed=6),
+    # few tokens: split-K router logits (3 row tiles, 8 k-blocks) and, at 100 rows per expert,
+    # the single-CTA form of the grouped GEMMs
+    "bf16_few_tokens": Workload("bf16_few_tokens", "bf16", 300, 512, 3, 4, (256, 128, 64), 2, 4, seed=7),
     "bf16_skew": Workload("bf16_skew", "bf16", 1500, 256, 4, 8, (256, 192, 128, 64), 2, 6,
                           zipf_beta=3.0, seed=5),
 }
