@@ -1187,6 +1187,7 @@ __global__ void __launch_bounds__(256)
 sum_partials_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     float acc = part[i];
+#pragma unroll 8
     for (int s = 1; s < splits; ++s) acc += part[(size_t)s * n + i];
     out[i] = acc;
   }
@@ -1197,6 +1198,7 @@ sum_partials_bias_kernel(const float* __restrict__ part, int splits, size_t n, i
                          const float* __restrict__ bias, float* __restrict__ out) {
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     float acc = part[i];
+#pragma unroll 8
     for (int s = 1; s < splits; ++s) acc += part[(size_t)s * n + i];
     out[i] = bias ? acc + bias[i % n_cols] : acc;
   }
@@ -1212,6 +1214,7 @@ int router_logits_splits(const Dims& D, int n_tiles) {
   int64_t s = 148 / tiles;
   const int64_t fit = (int64_t)router_dw_splits(D) * D.d / D.T;
   if (s > fit) s = fit;
+  if (s > 16) s = 16;                                    // the sum of the partials costs too
   if (s > k_blocks) s = k_blocks;
   if (s < 4) return 1;                                   // little to win, one more launch to pay
   const int64_t chunk = (k_blocks + s - 1) / s;
