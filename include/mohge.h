@@ -19,6 +19,12 @@
  *     allocates no caller-visible memory, frees nothing, and never synchronises the device:
  *     work is enqueued on `stream` (a cudaStream_t passed as void*) and the call returns.
  *   - Arguments are validated before anything is launched; an invalid call launches nothing.
+ *   - Stream capture: launch shapes depend on the config and T only; everything that depends on
+ *     the batch (counts, offsets, tile lists, statistics) stays in device memory.  A sequence of
+ *     calls captured into a CUDA graph therefore serves every later batch of the same T held in
+ *     the same buffers.  The first call of a process does one-time host set-up (driver entry
+ *     point, kernel attributes): make one call outside capture first.  mohge_get_device_status
+ *     synchronises and must stay outside capture.
  *   - `ws` is a caller-provided workspace of mohge_workspace_bytes() bytes.  It holds the
  *     device status word, tile lists and partial sums.  Calls that share a workspace must be
  *     ordered on one stream.
