@@ -130,3 +130,26 @@ def test_every_form_of_the_grouped_gemm_on_small_ragged_cases(switch, monkeypatc
         inp = make_inputs(wl)
         _, _, logits32 = oracle_layer(wl, inp)
         _compare(wl, inp, logits32)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_single_expert_layer_is_a_plain_ffn(dtype):
+    """N_g = N = K_g = K_e = 1: the gate is 1 for every token, so y is the expert's FFN of x and
+    the router receives no gradient beyond float32 cancellation noise (the exact value is of the
+    order of eps, far below anything a relative bar could be applied to)."""
+    wl = Workload("one_expert", dtype, 257, 64, 1, 1, (344,), 1, 1, seed=9)
+    inp = make_inputs(wl)
+    fwd, bwd, logits32 = oracle_layer(wl, inp)
+    b, dev = gpu_layer(wl, inp, logits32=logits32)
+    tol = tol_for(dtype)
+    assert (b.gate_w.cpu().numpy() == 1.0).all() and (b.expert_idx.cpu().numpy() == 0).all()
+    A, U, H, Y = O.swiglu_ffn(to_np64(inp["x"]), to_np64(inp["w13"][0][0]), to_np64(inp["w2"][0][0]))
+    assert max_rel(to_np64(b.y), Y) <= tol and max_rel(fwd["y"], Y) <= 1e-12
+    assert max_rel(to_np64(b.dx), bwd["dx"]) <= tol
+    assert max_rel(to_np64(b.dw13[0]), bwd["dw13"][0]) <= tol
+    assert max_rel(to_np64(b.dw2[0]), bwd["dw2"][0]) <= tol
+    assert max_rel(to_np64(b.dgate), bwd["dgate"]) <= tol
+    scale = float(np.abs(bwd["dgate"]).max())
+    assert np.abs(bwd["dlogits"]).max() <= 1e-12 * scale
+    assert float(b.dlogits.abs().max()) <= 1e-6 * scale
+    assert float(b.dw_router.abs().max()) <= 1e-6 * scale * wl.T
