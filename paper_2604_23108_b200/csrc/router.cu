@@ -55,38 +55,47 @@ __device__ __forceinline__ float sig_s(float z) {
   return z >= 0.0f ? __fdiv_rn(1.0f, den) : __fdiv_rn(e, den);
 }
 
+// Order-preserving map float -> unsigned (a < b  <=>  ord_key(a) < ord_key(b), no NaNs here) and
+// its inverse, so that one integer warp reduction finds the largest key.
+__device__ __forceinline__ unsigned ord_key(float k) {
+  const unsigned b = __float_as_uint(k);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float ord_key_inv(unsigned u) {
+  return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+
 // K rounds of warp arg-max over (key descending, index ascending).  key[j] belongs to expert
 // eid[j] (ascending in j inside a lane).  Winner of round k is left in lane k (win_e, win_key).
+// A round is one max-reduction over the ordered keys and one min-reduction over the indices of
+// the lanes that hold the maximum; taken experts drop to the key -3.
 template <int J>
 __device__ __forceinline__ void warp_topk(float (&key)[J], const int (&eid)[J], int K, int lane,
                                           int& win_e, float& win_key) {
   win_e = -1;
   win_key = 0.0f;
+  unsigned uk[J];
+#pragma unroll
+  for (int j = 0; j < J; ++j) uk[j] = ord_key(key[j]);
+  const unsigned taken = ord_key(-3.0f);
   for (int k = 0; k < K; ++k) {
-    float bk = -4.0f;
+    unsigned bu = 0;                     // below every ordered key
     int be = 0x7fffffff;
 #pragma unroll
     for (int j = 0; j < J; ++j) {
-      if (key[j] > bk) {
-        bk = key[j];
+      if (uk[j] > bu) {
+        bu = uk[j];
         be = eid[j];
       }
     }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ok = __shfl_xor_sync(kFull, bk, off);
-      const int oe = __shfl_xor_sync(kFull, be, off);
-      if (ok > bk || (ok == bk && oe < be)) {
-        bk = ok;
-        be = oe;
-      }
-    }
+    const unsigned m = __reduce_max_sync(kFull, bu);
+    const int we = __reduce_min_sync(kFull, bu == m ? be : 0x7fffffff);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (eid[j] == be) key[j] = -3.0f;
+      if (eid[j] == we) uk[j] = taken;
     if (lane == k) {
-      win_e = be;
-      win_key = bk;
+      win_e = we;
+      win_key = ord_key_inv(m);
     }
   }
 }
@@ -122,7 +131,8 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
       gmask |= 1u << best;
       if (lane == 0) group_idx[(size_t)t * s.Kg + k] = best;
     }
-    if (lane < s.Ng) gs_saved[(size_t)t * s.Ng + lane] = sig_s(L[lane]);
+    const float gsv = lane < s.Ng ? sig_s(L[lane]) : 0.0f;      // GS of group `lane`
+    if (lane < s.Ng) gs_saved[(size_t)t * s.Ng + lane] = gsv;
     // ---- Eq. 3, 4: keys of the lane's slots ----
     float key[J];
     int eid[J];
@@ -140,11 +150,11 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
       float S = p;
       for (int mask = 1; mask < s.P; mask <<= 1) S = __fadd_rn(S, __shfl_xor_sync(kFull, S, mask));
       const bool sel = valid && ((gmask >> g) & 1u);
-      const float gl = valid ? L[g] : 0.0f;
+      const float sg = __shfl_sync(kFull, gsv, g & 31);           // GS of this slot's group
       float kv = valid ? -1.0f : -2.0f;
       float ev = 0.0f;
       if (sel) {
-        kv = __fmul_rn(p, __fdiv_rn(sig_s(gl), S));
+        kv = __fmul_rn(p, __fdiv_rn(sg, S));
         ev = __fdiv_rn(p, S);
       }
       key[j] = kv;
@@ -176,7 +186,7 @@ __global__ void zero_counts_kernel(int32_t* group_count, int Ng, int32_t* cnt_ro
 }
 
 // ---------------------------------------------------------------- statistics (Eq. 7-14)
-constexpr int kStatsThreads = 256;
+constexpr int kStatsThreads = 512;
 constexpr int kStatsWarps = kStatsThreads / 32;
 
 template <int J>
