@@ -466,10 +466,11 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   // expert segment table (aligned_offsets) staged once, so that no role chases it through global
   // memory between tiles
   int32_t* s_seg = reinterpret_cast<int32_t*>(smem_gen + kStages * kStageBytes + kStgBytes + 512);
-  if (!is_plain<ROLE>()) {
-    const int ne = p.gs.Ng * p.gs.N;
-    for (int i = threadIdx.x; i <= ne; i += blockDim.x) s_seg[i] = p.aligned[i];
-  }
+  // Programmatic dependent launch (when the host asked for it): the next kernel of the stream may
+  // be scheduled onto SMs as the CTAs of this one leave, and this kernel may itself have been
+  // scheduled while its predecessor was draining.  Nothing before griddep_wait() below touches
+  // global memory; without the launch attribute both instructions do nothing.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -500,6 +501,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   if (CG == 2) cluster_sync_all();     // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // barriers and TMEM are set up; from here on the predecessor's results are read
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!is_plain<ROLE>()) {
+    const int ne = p.gs.Ng * p.gs.N;
+    for (int i = threadIdx.x; i <= ne; i += blockDim.x) s_seg[i] = p.aligned[i];
+    __syncthreads();
+  }
   const int total = is_plain<ROLE>() ? p.plain_total : *p.tile_count;
   // Tile of this CTA (pair) in round i.  The list is sorted by cost, heaviest first.  When the
   // costs differ (zigzag), rounds alternate direction (0..n-1, then n-1..0), so no CTA always gets
@@ -1101,6 +1109,14 @@ int pick_bn(int extent, const int* cand, int ncand) {
   return best;
 }
 
+// Programmatic dependent launch of the GEMM kernels (see the kernel's prologue): on unless
+// MOHGE_PDL=0.  Measured 1.5-2.5 % of the step at the 8k- and 16k-token workloads (launch and
+// prologue of each GEMM hidden behind the tail of its predecessor), nothing at the large one.
+static bool dependent_launch() {
+  const char* e = getenv("MOHGE_PDL");
+  return !(e && e[0] == '0');
+}
+
 template <int ROLE, int CG, int WIDE = 0>
 int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
@@ -1115,11 +1131,13 @@ int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = Geo<CG, WIDE>::kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = CG;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (CG == 2) {
@@ -1135,6 +1153,7 @@ int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
     const int want = grid / CG < max_clusters ? grid / CG : max_clusters;
     cfg.gridDim = dim3(want * CG);
   }
+  cfg.numAttrs = dependent_launch() ? 2 : 1;
   MOHGE_CUDA(cudaLaunchKernelEx(&cfg, tc_grouped_kernel<ROLE, CG, WIDE>, p));
   MOHGE_LAUNCH_CHECK("tc_grouped_kernel");
   return MOHGE_OK;
