@@ -37,6 +37,36 @@ extern unsigned long long g_launches;   // kernels launched by this library (hos
     ++::mohge::g_launches;                                         \
   } while (0)
 
+// ---------------------------------------------------------------- dependent launches
+// Every kernel of the library is launched with the programmatic-stream-serialization attribute
+// (unless MOHGE_PDL=0) and starts with pdl_enter(): the block lets the next kernel of the stream
+// be scheduled as soon as SM resources allow, then waits until the previous kernel has completed
+// and its writes are visible.  The wait is the first thing a block does, so the order of all
+// memory effects is that of ordinary stream launches; what overlaps is launch latency and block
+// scheduling.  (The tensor-core GEMM kernel places the wait after its own set-up instead.)
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
+bool dependent_launch();   // false when MOHGE_PDL=0
+
+template <typename... KArgs, typename... Args>
+inline void launch_dep(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = dependent_launch() ? 1 : 0;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // error read by MOHGE_LAUNCH_CHECK
+}
+
 // ---------------------------------------------------------------- derived sizes
 struct Dims {
   int d, Ng, N, P, Ne, NL, Kg, Ke, Wmax, align;

@@ -59,6 +59,7 @@ __device__ __forceinline__ void warp_counts(const ExpertSet& s, int Ne, int lane
 __global__ void __launch_bounds__(kDispatchChunk)
 dispatch_hist_kernel(const int32_t* __restrict__ expert_idx, int T, int Ke, int Ne,
                      int32_t* __restrict__ hist, int32_t* status) {
+  pdl_enter();
   __shared__ int s_wcnt[kChunkWarps][256];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = blockIdx.x * kDispatchChunk + threadIdx.x;
@@ -77,6 +78,7 @@ __global__ void __launch_bounds__(256)
 dispatch_scan_kernel(int chunks, int Ne, int align, const int32_t* __restrict__ hist,
                      int32_t* __restrict__ base, int32_t* __restrict__ counts,
                      int32_t* __restrict__ offsets, int32_t* __restrict__ aligned) {
+  pdl_enter();
   __shared__ int s_cnt[256];
   const int e = threadIdx.x;
   if (e < Ne) {
@@ -108,6 +110,7 @@ dispatch_scatter_kernel(const int32_t* __restrict__ expert_idx, int T, int Ke, i
                         const int32_t* __restrict__ aligned, int32_t* __restrict__ row_of,
                         int32_t* __restrict__ prow_of, int32_t* __restrict__ src_of,
                         int32_t* status) {
+  pdl_enter();
   __shared__ int s_wcnt[kChunkWarps][256];
   __shared__ int s_start[256];     // dense row of the chunk's first token for expert e
   __shared__ int s_pstart[256];    // same in physical numbering
@@ -208,6 +211,7 @@ __global__ void __launch_bounds__(256)
 permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ prow_of, int T, int Ke,
                     int row_vecs, int rows_cap, Vec16* __restrict__ x_perm, int nb_tok,
                     const int32_t* __restrict__ counts, const int32_t* __restrict__ aligned) {
+  pdl_enter();
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   if ((int)blockIdx.x >= nb_tok) {      // padding rows (launched only when segments are aligned)
     const int j = blockIdx.x - nb_tok;
@@ -230,6 +234,7 @@ permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ pro
 __global__ void __launch_bounds__(256)
 zero_pad_rows_kernel(const int32_t* __restrict__ counts, const int32_t* __restrict__ aligned,
                      int row_vecs, Vec16* __restrict__ buf) {
+  pdl_enter();
   const int e = blockIdx.x;
   const int r0 = aligned[e] + counts[e], r1 = aligned[e + 1];
   const Vec16 z = {{0, 0, 0, 0}};
@@ -246,6 +251,7 @@ __global__ void __launch_bounds__(256)
 combine_kernel(const Vec16* __restrict__ y_perm, const int32_t* __restrict__ prow_of,
                const float* __restrict__ gate_w, const Vec16* __restrict__ add, int Tn, int Ke,
                int row_vecs, int rows_cap, Vec16* __restrict__ y) {
+  pdl_enter();
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
   for (int t = blockIdx.x; t < Tn; t += gridDim.x) {
@@ -283,6 +289,7 @@ combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_per
                    int Ke, int row_vecs, int rows_cap, Vec16* __restrict__ dy_perm,
                    float* __restrict__ dgate_w, int nb_tok, const int32_t* __restrict__ counts,
                    const int32_t* __restrict__ aligned) {
+  pdl_enter();
   __shared__ int s_row[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_g[MOHGE_MAX_K_EXPERTS];
   __shared__ float s_red[MOHGE_MAX_K_EXPERTS][8];
@@ -346,19 +353,19 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
   const int chunks = ceil_div(D.T, kDispatchChunk);
   const int T = (int)D.T;
   if (chunks > 0) {
-    dispatch_hist_kernel<<<chunks, kDispatchChunk, 0, st>>>(expert_idx, T, D.Ke, D.Ne, hist, status);
+    launch_dep(dispatch_hist_kernel, dim3(chunks), dim3(kDispatchChunk), st, expert_idx, T, D.Ke, D.Ne, hist, status);
     MOHGE_LAUNCH_CHECK("dispatch_hist_kernel");
   }
-  dispatch_scan_kernel<<<1, 256, 0, st>>>(chunks, D.Ne, D.align, hist, base, counts, offsets, aligned);
+  launch_dep(dispatch_scan_kernel, dim3(1), dim3(256), st, chunks, D.Ne, D.align, hist, base, counts, offsets, aligned);
   MOHGE_LAUNCH_CHECK("dispatch_scan_kernel");
   if (chunks == 0) return MOHGE_OK;
-  dispatch_scatter_kernel<<<chunks, kDispatchChunk, 0, st>>>(expert_idx, T, D.Ke, D.Ne, base, offsets,
+  launch_dep(dispatch_scatter_kernel, dim3(chunks), dim3(kDispatchChunk), st, expert_idx, T, D.Ke, D.Ne, base, offsets,
                                                             aligned, row_of, prow_of, src_of, status);
   MOHGE_LAUNCH_CHECK("dispatch_scatter_kernel");
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   const int pad_blocks = D.align > 1 ? 4 * D.Ne : 0;
-  permute_rows_kernel<<<blocks + pad_blocks, block_for(row_vecs), 0, st>>>(
+  launch_dep(permute_rows_kernel, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st, 
       (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)x_perm, blocks, counts, aligned);
   MOHGE_LAUNCH_CHECK("permute_rows_kernel");
   return MOHGE_OK;
@@ -371,11 +378,11 @@ int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   if (D.bf16)
-    combine_kernel<__nv_bfloat16><<<blocks, block_for(row_vecs), 0, st>>>(
+    launch_dep(combine_kernel<__nv_bfloat16>, dim3(blocks), dim3(block_for(row_vecs)), st, 
         (const Vec16*)y_perm, prow_of, gate_w, (const Vec16*)add, T, D.Ke, row_vecs, (int)D.Rcap,
         (Vec16*)y);
   else
-    combine_kernel<float><<<blocks, block_for(row_vecs), 0, st>>>(
+    launch_dep(combine_kernel<float>, dim3(blocks), dim3(block_for(row_vecs)), st, 
         (const Vec16*)y_perm, prow_of, gate_w, (const Vec16*)add, T, D.Ke, row_vecs, (int)D.Rcap,
         (Vec16*)y);
   MOHGE_LAUNCH_CHECK("combine_kernel");
@@ -396,17 +403,17 @@ int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
   if (T > 0) {
     const int blocks = T < 148 * 16 ? T : 148 * 16;
     if (D.bf16)
-      combine_bwd_kernel<__nv_bfloat16><<<blocks + pad_blocks, block_for(row_vecs), 0, st>>>(
+      launch_dep(combine_bwd_kernel<__nv_bfloat16>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st, 
           (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
           (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
     else
-      combine_bwd_kernel<float><<<blocks + pad_blocks, block_for(row_vecs), 0, st>>>(
+      launch_dep(combine_bwd_kernel<float>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st, 
           (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
           (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
     MOHGE_LAUNCH_CHECK("combine_bwd_kernel");
   }
   if (D.align > 1 && T == 0) {
-    zero_pad_rows_kernel<<<dim3(D.Ne, 4), 256, 0, st>>>(counts, aligned, row_vecs, (Vec16*)dy_perm);
+    launch_dep(zero_pad_rows_kernel, dim3(dim3(D.Ne, 4)), dim3(256), st, counts, aligned, row_vecs, (Vec16*)dy_perm);
     MOHGE_LAUNCH_CHECK("zero_pad_rows_kernel");
   }
   return MOHGE_OK;

@@ -126,6 +126,7 @@ build_tiles_body(const TilePlan& p, const int32_t* __restrict__ aligned, int32_t
 __global__ void __launch_bounds__(256)
 build_tiles_kernel(TilePlan p, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
                    Tile* __restrict__ tiles, long long cap, int32_t* status) {
+  pdl_enter();
   build_tiles_body(p, aligned, tile_count, tiles, cap, status);
 }
 
@@ -137,6 +138,7 @@ struct MultiPlan {
 __global__ void __launch_bounds__(256)
 build_tiles_multi_kernel(MultiPlan mp, const int32_t* __restrict__ aligned, int32_t* __restrict__ tile_count,
                          Tile* __restrict__ tiles, long long cap, int32_t* status) {
+  pdl_enter();
   const int i = blockIdx.y;
   build_tiles_body(mp.p[i], aligned, tile_count + 64 * i, tiles + (size_t)cap * i, cap, status);
 }
@@ -206,6 +208,7 @@ struct SimtArgs {
 __global__ void __launch_bounds__(256)
 simt_grouped_kernel(SimtArgs a, const int32_t* __restrict__ aligned,
                     const int32_t* __restrict__ tile_count, const Tile* __restrict__ tiles) {
+  pdl_enter();
   const int total = *tile_count;
   const bool f32 = a.f32;
   const long long d = a.gs.d, pitchAU = 2LL * a.gs.Wmax, pitchH = a.gs.Wmax;
@@ -278,6 +281,7 @@ __global__ void __launch_bounds__(256)
 simt_plain_kernel(int M, int N, int K, const void* A, int a32, long long sAm, long long sAk,
                   const void* B, int b32, long long sBn, long long sBk, void* C, int c32,
                   long long sCm, const float* __restrict__ bias, int accumulate) {
+  pdl_enter();
   const int m0 = blockIdx.y * SBM, n0 = blockIdx.x * SBN;
   const size_t ea = a32 ? 4 : 2, eb = b32 ? 4 : 2;
   float acc[4][4];
@@ -314,6 +318,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 swiglu_fwd_kernel(GroupShape gs, const int32_t* __restrict__ aligned, const T* __restrict__ au,
                   T* __restrict__ h) {
+  pdl_enter();
   const int e = blockIdx.x, W = gs.W[e / gs.N];
   const long long r0 = aligned[e], n = (long long)(aligned[e + 1] - aligned[e]) * W;
   for (long long i = (long long)blockIdx.y * blockDim.x + threadIdx.x; i < n;
@@ -329,6 +334,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 swiglu_bwd_kernel(GroupShape gs, const int32_t* __restrict__ aligned, const T* __restrict__ au,
                   T* __restrict__ dau) {
+  pdl_enter();
   const int e = blockIdx.x, W = gs.W[e / gs.N];
   const long long r0 = aligned[e], n = (long long)(aligned[e + 1] - aligned[e]) * W;
   for (long long i = (long long)blockIdx.y * blockDim.x + threadIdx.x; i < n;
@@ -345,6 +351,7 @@ swiglu_bwd_kernel(GroupShape gs, const int32_t* __restrict__ aligned, const T* _
 // experts without tokens: their weight gradients are exactly zero
 __global__ void __launch_bounds__(256)
 zero_empty_wgrad_kernel(GroupShape gs, GroupPtrs gp, const int32_t* __restrict__ counts) {
+  pdl_enter();
   const int e = blockIdx.x;
   if (counts[e] != 0) return;
   const int g = e / gs.N, i = e % gs.N;
@@ -370,7 +377,7 @@ int32_t launch_build_tiles_multi(const TilePlan* plans, int nplans, const int32_
   MultiPlan mp;
   memset(&mp, 0, sizeof(mp));
   for (int i = 0; i < nplans && i < kMaxLists; ++i) mp.p[i] = plans[i];
-  build_tiles_multi_kernel<<<dim3(32, nplans), 256, 0, st>>>(mp, aligned, tile_count, tiles,
+  launch_dep(build_tiles_multi_kernel, dim3(dim3(32, nplans)), dim3(256), st, mp, aligned, tile_count, tiles,
                                                            (long long)tiles_cap, status);
   MOHGE_LAUNCH_CHECK("build_tiles_multi_kernel");
   return MOHGE_OK;
@@ -378,7 +385,7 @@ int32_t launch_build_tiles_multi(const TilePlan* plans, int nplans, const int32_
 
 int32_t launch_build_tiles_plan(const TilePlan& p, const int32_t* aligned, int32_t* tile_count,
                                 Tile* tiles, int64_t tiles_cap, int32_t* status, cudaStream_t st) {
-  build_tiles_kernel<<<32, 256, 0, st>>>(p, aligned, tile_count, tiles, (long long)tiles_cap, status);
+  launch_dep(build_tiles_kernel, dim3(32), dim3(256), st, p, aligned, tile_count, tiles, (long long)tiles_cap, status);
   MOHGE_LAUNCH_CHECK("build_tiles_kernel");
   return MOHGE_OK;
 }
@@ -423,7 +430,7 @@ int32_t launch_simt_grouped(const Dims& D, int role, const GroupPtrs& P, const v
   SimtArgs a;
   a.role = role; a.f32 = D.bf16 ? 0 : 1; a.accumulate = accumulate;
   a.gs = make_group_shape(D); a.gp = P; a.A = A; a.B = B; a.C = C;
-  simt_grouped_kernel<<<148 * 4, 256, 0, st>>>(a, aligned, tile_count, tiles);
+  launch_dep(simt_grouped_kernel, dim3(148 * 4), dim3(256), st, a, aligned, tile_count, tiles);
   MOHGE_LAUNCH_CHECK("simt_grouped_kernel");
   return MOHGE_OK;
 }
@@ -431,9 +438,9 @@ int32_t launch_simt_grouped(const Dims& D, int role, const GroupPtrs& P, const v
 int32_t launch_swiglu_fwd(const Dims& D, const int32_t* aligned, void* au, void* h, cudaStream_t st) {
   const GroupShape gs = make_group_shape(D);
   if (D.bf16)
-    swiglu_fwd_kernel<__nv_bfloat16><<<dim3(D.Ne, 32), 256, 0, st>>>(gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)h);
+    launch_dep(swiglu_fwd_kernel<__nv_bfloat16>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)h);
   else
-    swiglu_fwd_kernel<float><<<dim3(D.Ne, 32), 256, 0, st>>>(gs, aligned, (const float*)au, (float*)h);
+    launch_dep(swiglu_fwd_kernel<float>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const float*)au, (float*)h);
   MOHGE_LAUNCH_CHECK("swiglu_fwd_kernel");
   return MOHGE_OK;
 }
@@ -441,15 +448,15 @@ int32_t launch_swiglu_fwd(const Dims& D, const int32_t* aligned, void* au, void*
 int32_t launch_swiglu_bwd(const Dims& D, const int32_t* aligned, const void* au, void* dau, cudaStream_t st) {
   const GroupShape gs = make_group_shape(D);
   if (D.bf16)
-    swiglu_bwd_kernel<__nv_bfloat16><<<dim3(D.Ne, 32), 256, 0, st>>>(gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)dau);
+    launch_dep(swiglu_bwd_kernel<__nv_bfloat16>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)dau);
   else
-    swiglu_bwd_kernel<float><<<dim3(D.Ne, 32), 256, 0, st>>>(gs, aligned, (const float*)au, (float*)dau);
+    launch_dep(swiglu_bwd_kernel<float>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const float*)au, (float*)dau);
   MOHGE_LAUNCH_CHECK("swiglu_bwd_kernel");
   return MOHGE_OK;
 }
 
 int32_t launch_zero_empty_wgrad(const Dims& D, const GroupPtrs& P, const int32_t* counts, cudaStream_t st) {
-  zero_empty_wgrad_kernel<<<dim3(D.Ne, 16), 256, 0, st>>>(make_group_shape(D), P, counts);
+  launch_dep(zero_empty_wgrad_kernel, dim3(dim3(D.Ne, 16)), dim3(256), st, make_group_shape(D), P, counts);
   MOHGE_LAUNCH_CHECK("zero_empty_wgrad_kernel");
   return MOHGE_OK;
 }
@@ -459,7 +466,7 @@ int32_t launch_simt_plain(int M, int N, int K, const void* A, int a_f32, int64_t
                           int64_t sCm, const float* bias, int accumulate, cudaStream_t st) {
   if (M == 0 || N == 0) return MOHGE_OK;
   dim3 grid((N + SBN - 1) / SBN, (M + SBM - 1) / SBM);
-  simt_plain_kernel<<<grid, 256, 0, st>>>(M, N, K, A, a_f32, sAm, sAk, B, b_f32, sBn, sBk, C, c_f32,
+  launch_dep(simt_plain_kernel, dim3(grid), dim3(256), st, M, N, K, A, a_f32, sAm, sAk, B, b_f32, sBn, sBk, C, c_f32,
                                           sCm, bias, accumulate);
   MOHGE_LAUNCH_CHECK("simt_plain_kernel");
   return MOHGE_OK;

@@ -1109,14 +1109,6 @@ int pick_bn(int extent, const int* cand, int ncand) {
   return best;
 }
 
-// Programmatic dependent launch of the GEMM kernels (see the kernel's prologue): on unless
-// MOHGE_PDL=0.  Measured 1.5-2.5 % of the step at the 8k- and 16k-token workloads (launch and
-// prologue of each GEMM hidden behind the tail of its predecessor), nothing at the large one.
-static bool dependent_launch() {
-  const char* e = getenv("MOHGE_PDL");
-  return !(e && e[0] == '0');
-}
-
 template <int ROLE, int CG, int WIDE = 0>
 int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
@@ -1204,6 +1196,7 @@ namespace {
 // out[i] = part[0][i] + part[1][i] + ... in this fixed order (run-to-run identical bits)
 __global__ void __launch_bounds__(256)
 sum_partials_kernel(const float* __restrict__ part, int splits, size_t n, float* __restrict__ out) {
+  pdl_enter();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     float acc = part[i];
 #pragma unroll 8
@@ -1215,6 +1208,7 @@ sum_partials_kernel(const float* __restrict__ part, int splits, size_t n, float*
 __global__ void __launch_bounds__(256)
 sum_partials_bias_kernel(const float* __restrict__ part, int splits, size_t n, int n_cols,
                          const float* __restrict__ bias, float* __restrict__ out) {
+  pdl_enter();
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     float acc = part[i];
 #pragma unroll 8
@@ -1306,7 +1300,7 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
       const int32_t rc2 = launch_role<ROLE_LOGITS, 1>(p, grid, st);
       if (rc2 || p.plain_splits == 1) return rc2;
       const size_t n = (size_t)D.T * D.NL;
-      sum_partials_bias_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partials, p.plain_splits, n, D.NL,
+      launch_dep(sum_partials_bias_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), st, partials, p.plain_splits, n, D.NL,
                                                                            bias, (float*)C);
       MOHGE_LAUNCH_CHECK("sum_partials_bias_kernel");
       return MOHGE_OK;
@@ -1315,7 +1309,7 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
       const int32_t rc2 = launch_role<ROLE_ROUTER_DW, 1>(p, grid, st);
       if (rc2 || p.plain_splits == 1) return rc2;
       const size_t n = (size_t)D.NL * D.d;
-      sum_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(partials, p.plain_splits, n, (float*)C);
+      launch_dep(sum_partials_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), st, partials, p.plain_splits, n, (float*)C);
       MOHGE_LAUNCH_CHECK("sum_partials_kernel");
       return MOHGE_OK;
     }

@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(256)
 router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* __restrict__ group_idx,
                      int32_t* __restrict__ expert_idx, float* __restrict__ gate_w,
                      float* __restrict__ gs_saved, float* __restrict__ esp_saved) {
+  pdl_enter();
   const int lane = threadIdx.x & 31;
   const int warps_total = (gridDim.x * blockDim.x) >> 5;
   for (int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < s.T; t += warps_total) {
@@ -177,6 +178,7 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
 // the three count arrays start at zero (one launch instead of three memsets)
 __global__ void zero_counts_kernel(int32_t* group_count, int Ng, int32_t* cnt_routed, int32_t* cnt_lit,
                                    int Ne) {
+  pdl_enter();
   for (int i = threadIdx.x; i < Ne; i += blockDim.x) {
     cnt_routed[i] = 0;
     cnt_lit[i] = 0;
@@ -195,6 +197,7 @@ aux_stats_kernel(RouterShape s, float eps, const float* __restrict__ gs, const f
                  const int32_t* __restrict__ group_idx, const int32_t* __restrict__ expert_idx,
                  int32_t* __restrict__ group_count, int32_t* __restrict__ cnt_routed,
                  int32_t* __restrict__ cnt_lit, double* __restrict__ partials) {
+  pdl_enter();
   __shared__ int s_cg[MOHGE_MAX_GROUPS];
   __shared__ int s_cr[256];
   __shared__ int s_cl[256];
@@ -279,6 +282,7 @@ __global__ void aux_finalize_kernel(RouterShape s, LossParams lp, int nblocks,
                                     const int32_t* __restrict__ cnt_routed,
                                     const int32_t* __restrict__ cnt_lit, float* __restrict__ group_psum,
                                     float* __restrict__ expert_psum, float* __restrict__ loss_out) {
+  pdl_enter();
   __shared__ double s_tot[256 + MOHGE_MAX_GROUPS];
   // one warp per column: lane l adds the partial rows l, l + 32, ... in that order, then a
   // butterfly adds the 32 lane sums; the order is fixed, so the result is run-to-run identical
@@ -328,6 +332,7 @@ router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
                   const int32_t* __restrict__ group_idx, const int32_t* __restrict__ expert_idx,
                   const int32_t* __restrict__ group_count, const int32_t* __restrict__ expert_count,
                   float* __restrict__ dlogits, __nv_bfloat16* __restrict__ dl16, int dl16_pitch) {
+  pdl_enter();
   __shared__ float s_dkey[kBwdWarps][256];
   __shared__ float s_dgs[kBwdWarps][MOHGE_MAX_GROUPS];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -448,7 +453,7 @@ int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_
   if (D.T == 0) return MOHGE_OK;
   const RouterShape s = make_shape(D);
   const int blocks = (int)((D.T + 7) / 8) < 148 * 8 ? (int)((D.T + 7) / 8) : 148 * 8;
-  MOHGE_DISPATCH_J(slots_per_lane(D), (router_select_kernel<JJ><<<blocks, 256, 0, st>>>(
+  MOHGE_DISPATCH_J(slots_per_lane(D), (launch_dep(router_select_kernel<JJ>, dim3(blocks), dim3(256), st, 
                                           s, logits, group_idx, expert_idx, gate_w, gs, esp)));
   MOHGE_LAUNCH_CHECK("router_select_kernel");
   return MOHGE_OK;
@@ -459,13 +464,13 @@ int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs
                          float* group_psum, int32_t* cnt_routed, int32_t* cnt_lit,
                          float* expert_psum, float* loss_out, double* partials, cudaStream_t st) {
   const RouterShape s = make_shape(D);
-  zero_counts_kernel<<<1, 256, 0, st>>>(group_count, D.Ng, cnt_routed, cnt_lit, D.Ne);
+  launch_dep(zero_counts_kernel, dim3(1), dim3(256), st, group_count, D.Ng, cnt_routed, cnt_lit, D.Ne);
   MOHGE_LAUNCH_CHECK("zero_counts_kernel");
   int blocks = ceil_div(D.T, kStatsWarps);
   if (blocks > kStatsBlocks) blocks = kStatsBlocks;
   if (blocks > 0) {
     MOHGE_DISPATCH_J(slots_per_lane(D),
-                     (aux_stats_kernel<JJ><<<blocks, kStatsThreads, 0, st>>>(
+                     (launch_dep(aux_stats_kernel<JJ>, dim3(blocks), dim3(kStatsThreads), st, 
                          s, cfg.eps, gs, esp, group_idx, expert_idx, group_count, cnt_routed,
                          cnt_lit, partials)));
     MOHGE_LAUNCH_CHECK("aux_stats_kernel");
@@ -477,7 +482,7 @@ int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs
     lp.w_over_wmax[g] = g < D.Ng ? (float)D.W[g] / (float)D.Wmax : 0.0f;
   RouterShape s1 = s;
   if (s1.T == 0) s1.T = 1;   // empty batch: sums are zero, avoid 0/0 in the loss
-  aux_finalize_kernel<<<1, 1024, 0, st>>>(s1, lp, blocks, partials, group_count, cnt_routed, cnt_lit,
+  launch_dep(aux_finalize_kernel, dim3(1), dim3(1024), st, s1, lp, blocks, partials, group_count, cnt_routed, cnt_lit,
                                          group_psum, expert_psum, loss_out);
   MOHGE_LAUNCH_CHECK("aux_finalize_kernel");
   return MOHGE_OK;
@@ -500,7 +505,7 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
   int blocks = ceil_div(D.T, kBwdWarps);
   if (blocks > 148 * 8) blocks = 148 * 8;
   MOHGE_DISPATCH_J(slots_per_lane(D),
-                   (router_bwd_kernel<JJ><<<blocks, kBwdWarps * 32, 0, st>>>(
+                   (launch_dep(router_bwd_kernel<JJ>, dim3(blocks), dim3(kBwdWarps * 32), st, 
                        s, bp, dgate, gs, esp, group_idx, expert_idx, group_count, expert_count,
                        dlogits, dl16, dl16_pitch)));
   MOHGE_LAUNCH_CHECK("router_bwd_kernel");
