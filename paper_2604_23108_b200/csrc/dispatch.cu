@@ -365,7 +365,7 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   const int pad_blocks = D.align > 1 ? 4 * D.Ne : 0;
-  launch_dep(permute_rows_kernel, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st, 
+  launch_dep(permute_rows_kernel, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st,
       (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)x_perm, blocks, counts, aligned);
   MOHGE_LAUNCH_CHECK("permute_rows_kernel");
   return MOHGE_OK;
@@ -378,11 +378,11 @@ int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   if (D.bf16)
-    launch_dep(combine_kernel<__nv_bfloat16>, dim3(blocks), dim3(block_for(row_vecs)), st, 
+    launch_dep(combine_kernel<__nv_bfloat16>, dim3(blocks), dim3(block_for(row_vecs)), st,
         (const Vec16*)y_perm, prow_of, gate_w, (const Vec16*)add, T, D.Ke, row_vecs, (int)D.Rcap,
         (Vec16*)y);
   else
-    launch_dep(combine_kernel<float>, dim3(blocks), dim3(block_for(row_vecs)), st, 
+    launch_dep(combine_kernel<float>, dim3(blocks), dim3(block_for(row_vecs)), st,
         (const Vec16*)y_perm, prow_of, gate_w, (const Vec16*)add, T, D.Ke, row_vecs, (int)D.Rcap,
         (Vec16*)y);
   MOHGE_LAUNCH_CHECK("combine_kernel");
@@ -403,17 +403,17 @@ int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
   if (T > 0) {
     const int blocks = T < 148 * 16 ? T : 148 * 16;
     if (D.bf16)
-      launch_dep(combine_bwd_kernel<__nv_bfloat16>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st, 
+      launch_dep(combine_bwd_kernel<__nv_bfloat16>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st,
           (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
           (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
     else
-      launch_dep(combine_bwd_kernel<float>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st, 
+      launch_dep(combine_bwd_kernel<float>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st,
           (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
           (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
     MOHGE_LAUNCH_CHECK("combine_bwd_kernel");
   }
   if (D.align > 1 && T == 0) {
-    launch_dep(zero_pad_rows_kernel, dim3(dim3(D.Ne, 4)), dim3(256), st, counts, aligned, row_vecs, (Vec16*)dy_perm);
+    launch_dep(zero_pad_rows_kernel, dim3(D.Ne, 4), dim3(256), st, counts, aligned, row_vecs, (Vec16*)dy_perm);
     MOHGE_LAUNCH_CHECK("zero_pad_rows_kernel");
   }
   return MOHGE_OK;

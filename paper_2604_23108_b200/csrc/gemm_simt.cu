@@ -377,7 +377,7 @@ int32_t launch_build_tiles_multi(const TilePlan* plans, int nplans, const int32_
   MultiPlan mp;
   memset(&mp, 0, sizeof(mp));
   for (int i = 0; i < nplans && i < kMaxLists; ++i) mp.p[i] = plans[i];
-  launch_dep(build_tiles_multi_kernel, dim3(dim3(32, nplans)), dim3(256), st, mp, aligned, tile_count, tiles,
+  launch_dep(build_tiles_multi_kernel, dim3(32, nplans), dim3(256), st, mp, aligned, tile_count, tiles,
                                                            (long long)tiles_cap, status);
   MOHGE_LAUNCH_CHECK("build_tiles_multi_kernel");
   return MOHGE_OK;
@@ -438,9 +438,9 @@ int32_t launch_simt_grouped(const Dims& D, int role, const GroupPtrs& P, const v
 int32_t launch_swiglu_fwd(const Dims& D, const int32_t* aligned, void* au, void* h, cudaStream_t st) {
   const GroupShape gs = make_group_shape(D);
   if (D.bf16)
-    launch_dep(swiglu_fwd_kernel<__nv_bfloat16>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)h);
+    launch_dep(swiglu_fwd_kernel<__nv_bfloat16>, dim3(D.Ne, 32), dim3(256), st, gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)h);
   else
-    launch_dep(swiglu_fwd_kernel<float>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const float*)au, (float*)h);
+    launch_dep(swiglu_fwd_kernel<float>, dim3(D.Ne, 32), dim3(256), st, gs, aligned, (const float*)au, (float*)h);
   MOHGE_LAUNCH_CHECK("swiglu_fwd_kernel");
   return MOHGE_OK;
 }
@@ -448,15 +448,15 @@ int32_t launch_swiglu_fwd(const Dims& D, const int32_t* aligned, void* au, void*
 int32_t launch_swiglu_bwd(const Dims& D, const int32_t* aligned, const void* au, void* dau, cudaStream_t st) {
   const GroupShape gs = make_group_shape(D);
   if (D.bf16)
-    launch_dep(swiglu_bwd_kernel<__nv_bfloat16>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)dau);
+    launch_dep(swiglu_bwd_kernel<__nv_bfloat16>, dim3(D.Ne, 32), dim3(256), st, gs, aligned, (const __nv_bfloat16*)au, (__nv_bfloat16*)dau);
   else
-    launch_dep(swiglu_bwd_kernel<float>, dim3(dim3(D.Ne, 32)), dim3(256), st, gs, aligned, (const float*)au, (float*)dau);
+    launch_dep(swiglu_bwd_kernel<float>, dim3(D.Ne, 32), dim3(256), st, gs, aligned, (const float*)au, (float*)dau);
   MOHGE_LAUNCH_CHECK("swiglu_bwd_kernel");
   return MOHGE_OK;
 }
 
 int32_t launch_zero_empty_wgrad(const Dims& D, const GroupPtrs& P, const int32_t* counts, cudaStream_t st) {
-  launch_dep(zero_empty_wgrad_kernel, dim3(dim3(D.Ne, 16)), dim3(256), st, make_group_shape(D), P, counts);
+  launch_dep(zero_empty_wgrad_kernel, dim3(D.Ne, 16), dim3(256), st, make_group_shape(D), P, counts);
   MOHGE_LAUNCH_CHECK("zero_empty_wgrad_kernel");
   return MOHGE_OK;
 }

@@ -453,7 +453,7 @@ int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_
   if (D.T == 0) return MOHGE_OK;
   const RouterShape s = make_shape(D);
   const int blocks = (int)((D.T + 7) / 8) < 148 * 8 ? (int)((D.T + 7) / 8) : 148 * 8;
-  MOHGE_DISPATCH_J(slots_per_lane(D), (launch_dep(router_select_kernel<JJ>, dim3(blocks), dim3(256), st, 
+  MOHGE_DISPATCH_J(slots_per_lane(D), (launch_dep(router_select_kernel<JJ>, dim3(blocks), dim3(256), st,
                                           s, logits, group_idx, expert_idx, gate_w, gs, esp)));
   MOHGE_LAUNCH_CHECK("router_select_kernel");
   return MOHGE_OK;
@@ -470,7 +470,7 @@ int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs
   if (blocks > kStatsBlocks) blocks = kStatsBlocks;
   if (blocks > 0) {
     MOHGE_DISPATCH_J(slots_per_lane(D),
-                     (launch_dep(aux_stats_kernel<JJ>, dim3(blocks), dim3(kStatsThreads), st, 
+                     (launch_dep(aux_stats_kernel<JJ>, dim3(blocks), dim3(kStatsThreads), st,
                          s, cfg.eps, gs, esp, group_idx, expert_idx, group_count, cnt_routed,
                          cnt_lit, partials)));
     MOHGE_LAUNCH_CHECK("aux_stats_kernel");
@@ -505,7 +505,7 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
   int blocks = ceil_div(D.T, kBwdWarps);
   if (blocks > 148 * 8) blocks = 148 * 8;
   MOHGE_DISPATCH_J(slots_per_lane(D),
-                   (launch_dep(router_bwd_kernel<JJ>, dim3(blocks), dim3(kBwdWarps * 32), st, 
+                   (launch_dep(router_bwd_kernel<JJ>, dim3(blocks), dim3(kBwdWarps * 32), st,
                        s, bp, dgate, gs, esp, group_idx, expert_idx, group_count, expert_count,
                        dlogits, dl16, dl16_pitch)));
   MOHGE_LAUNCH_CHECK("router_bwd_kernel");
