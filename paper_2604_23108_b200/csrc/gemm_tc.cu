@@ -7,8 +7,11 @@
 //   warps 2..5  epilogue: tcgen05.ld -> registers -> fused element-wise math -> swizzled staging
 //               buffers in shared memory -> TMA stores (every global write of the expert roles is
 //               a full 128-byte row piece; the SwiGLU backward also reads A and U through TMA)
-// One persistent CTA per SM (a CTA pair per two SMs for the expert roles) walks the device-built,
-// cost-sorted tile list with a fixed stride, in alternating directions when tile costs differ.
+// One persistent CTA per SM (a CTA pair per two SMs for the expert roles; single CTAs when the
+// batch brings 128 rows per expert or fewer) walks the device-built, cost-sorted tile list with a
+// fixed stride, in alternating directions when tile costs differ.  The kernel is launched as a
+// programmatic dependent of its predecessor: barriers and tensor memory are set up before
+// griddepcontrol.wait, every global access comes after it.
 //
 // Six roles share the kernel (C = A . B^T over a contraction index k):
 //   FWD1        [A | U] = Xp . W13^T, fused SwiGLU epilogue writes A, U and H = silu(A) * U.
