@@ -298,21 +298,28 @@ __global__ void aux_finalize_kernel(RouterShape s, LossParams lp, int nblocks,
     }
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (warp == 0) {
+    // losses: lane l adds the terms l, l + 32, ... in that order, then a butterfly (fixed order)
     const double T = (double)s.T;
     const double fn = lp.f_norm_by_T ? 1.0 / T : 1.0;
     double LG = 0.0, LE = 0.0;
-    for (int g = 0; g < s.Ng; ++g) {
-      const double f = (double)s.Ng / s.Kg * group_count[g] * fn;     // Eq. 8
-      LG += lp.w_over_wmax[g] * f * (s_tot[s.Ne + g] / T);             // Eq. 7, 9
+    if (lane < s.Ng) {
+      const double f = (double)s.Ng / s.Kg * group_count[lane] * fn;   // Eq. 8
+      LG = lp.w_over_wmax[lane] * f * (s_tot[s.Ne + lane] / T);        // Eq. 7, 9
     }
     const int32_t* ce = lp.fe_mode == 0 ? cnt_lit : cnt_routed;
-    for (int e = 0; e < s.Ne; ++e) {
+    for (int e = lane; e < s.Ne; e += 32) {
       const double f = (double)s.N / s.Ke * ce[e] * fn;                // Eq. 12
       LE += f * (s_tot[e] / T);                                        // Eq. 11, 13
     }
-    loss_out[0] = (float)(lp.alpha_g * LG);
-    loss_out[1] = (float)(lp.alpha_e * LE);
+    for (int m = 16; m > 0; m >>= 1) {
+      LG += __shfl_xor_sync(kFull, LG, m);
+      LE += __shfl_xor_sync(kFull, LE, m);
+    }
+    if (lane == 0) {
+      loss_out[0] = (float)(lp.alpha_g * LG);
+      loss_out[1] = (float)(lp.alpha_e * LE);
+    }
   }
 }
 
