@@ -141,12 +141,8 @@ static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 #define OPT_PTR(p) MOHGE_CHECK_ARG(aligned16(p), #p " must be 16-byte aligned")
 
 static bool force_simt() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("MOHGE_FORCE_SIMT");
-    v = (e && e[0] == '1') ? 1 : 0;
-  }
-  return v == 1;
+  const char* e = getenv("MOHGE_FORCE_SIMT");
+  return e && e[0] == '1';
 }
 
 static int32_t group_ptrs(const Dims& D, const void* const* w13, const void* const* w2,

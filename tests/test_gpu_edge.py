@@ -114,7 +114,7 @@ def test_out_of_range_expert_index_sets_the_status_word_without_faulting():
 
 
 @pytest.mark.parametrize("switch", ["MOHGE_TC_CG=2,MOHGE_TC_WIDE=63", "MOHGE_TC_CG=2,MOHGE_TC_WIDE=0",
-                                    "MOHGE_TC_CG=1", "MOHGE_PDL=0"])
+                                    "MOHGE_TC_CG=1", "MOHGE_PDL=0", "MOHGE_FORCE_SIMT=1"])
 def test_every_form_of_the_grouped_gemm_on_small_ragged_cases(switch, monkeypatch):
     """The double-width form is chosen by default only for long contractions (the large
     workload) and single CTAs only for batches with few rows per expert, and the GEMM kernels are

@@ -158,7 +158,14 @@ def test_deterministic_rerun(case):
         assert torch.equal(b.dw13[g], b2.dw13[g]) and torch.equal(b.dw2[g], b2.dw2[g])
 
 
-def test_accumulate_adds_into_weight_gradients():
+@pytest.mark.parametrize("switch", ["", "MOHGE_TC_CG=1", "MOHGE_TC_CG=2,MOHGE_TC_WIDE=63",
+                                    "MOHGE_FORCE_SIMT=1"])
+def test_accumulate_adds_into_weight_gradients(switch, monkeypatch):
+    """accumulate = 1 adds the weight gradients into dw13 / dw2 (TMA reduce-add in the tensor-core
+    forms, read-modify-write in the FFMA kernel); checked in every form of the grouped GEMM."""
+    for kv in filter(None, switch.split(",")):
+        name, value = kv.split("=")
+        monkeypatch.setenv(name, value)
     wl = CASES["bf16_small"]
     inp = make_inputs(wl)
     _, _, logits32 = oracle_layer(wl, inp)
