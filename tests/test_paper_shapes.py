@@ -17,6 +17,9 @@ def _rows():
         if line.startswith("#") or not line.strip():
             continue
         f = line.split()
+        if f[0] == "alpha":
+            out["alpha"] = {f[1]: float(f[2]), f[3]: float(f[4])}
+            continue
         out[f[0]] = dict(d=int(f[1]), N_g=int(f[2]), K_g=int(f[3]), N_e=int(f[4]), K_e=int(f[5]),
                          N_s=int(f[6]), widths=tuple(int(v) for v in f[7:]))
     return out
@@ -53,3 +56,12 @@ def test_oracle_accepts_the_printed_architectures(scale):
                          k_groups=row["K_g"], k_experts=row["K_e"], group_width=list(row["widths"]))
     assert cfg.n_experts == row["N_e"]
     assert row["K_e"] <= row["K_g"] * (row["N_e"] // row["N_g"])     # Eq. 5 can always pick K_e experts
+
+
+def test_default_loss_coefficients_are_the_papers_best_row():
+    a = _rows()["alpha"]
+    from paper_2604_23108_b200 import binding as B
+    ocfg = O.OracleConfig(d_model=8, n_groups=1, experts_per_group=1, k_groups=1, k_experts=1, group_width=[8])
+    gcfg = B.Config(d_model=8, n_groups=1, experts_per_group=1, k_groups=1, k_experts=1, group_width=[8])
+    assert (ocfg.alpha_e, ocfg.alpha_g) == (a["alpha_E"], a["alpha_G"])
+    assert (gcfg.alpha_e, gcfg.alpha_g) == (a["alpha_E"], a["alpha_G"])
