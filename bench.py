@@ -34,7 +34,7 @@ from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs
 # capture summarised in profiles/launch_list_layer_step_cfg5.md (the L2 hit rate of these launches
 # differs between the GPUs of the pool: captures of the same build range over tens of GB); workloads without a
 # capture of the current kernels report null.
-NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 72.9e9}
+NCU_DRAM_TRAFFIC_PER_STEP = {}
 
 METRIC = "MoHGE layer fwd+bwd tokens/s"
 METRIC_FWD = "MoHGE layer fwd tokens/s"
@@ -268,12 +268,15 @@ def main():
             if mark:
                 gemm_marks.append((e0, e1, e1, e1))
             return
-        B.mohge_combine_bwd(gcfg, T, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.counts,
-                            buf.aligned, buf.dy_perm, buf.dgate)
+        # the gate gradient comes out of the experts' backward, so combine_bwd reads no y_perm
+        B.mohge_combine_bwd(gcfg, T, inp["dy"], None, buf.prow_of, buf.gate_w, buf.counts,
+                            buf.aligned, buf.dy_perm, None)
         if mark:
             e2.record()
-        B.mohge_expert_bwd(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts, buf.aligned,
-                           inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13, buf.dw2, 0, buf.ws)
+        B.mohge_expert_bwd_dgate(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts,
+                                 buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13,
+                                 buf.dw2, 0, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate,
+                                 buf.ws)
         if shared is not None:
             B.mohge_shared_bwd(gcfg, T, args.shared_width, inp["dy"], inp["x"], buf.au_sh, buf.h_sh,
                                shared[0], shared[1], buf.dau_sh, buf.dx_sh, buf.dw13_sh, buf.dw2_sh,

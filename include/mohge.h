@@ -205,6 +205,8 @@ int32_t mohge_combine(const mohge_config* cfg, int64_t T, const void* y_perm,
 /*
  * Backward of the combine:  dgate_w[t,k] = <dy[t], y_perm[prow_of[t,k]]>,
  * dy_perm[prow_of[t,k], :] = gate_w[t,k] * dy[t, :]; padding rows of dy_perm are zeroed.
+ *   y_perm and dgate_w may both be NULL: only dy_perm is written and y_perm is not read (half
+ *   of this call's memory traffic); the gate gradient then comes from mohge_expert_bwd_dgate.
  */
 int32_t mohge_combine_bwd(const mohge_config* cfg, int64_t T, const void* dy, const void* y_perm,
                           const int32_t* prow_of, const float* gate_w, const int32_t* counts,
@@ -224,6 +226,27 @@ int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm
                          const void* const* w13, const void* const* w2, void* dau, void* dx_perm,
                          float* const* dw13, float* const* dw2, int32_t accumulate, void* ws,
                          void* stream);
+
+/*
+ * mohge_expert_bwd that also returns the gate gradient of the combine (derivative of Eq. 15 with
+ * respect to the gate of Eq. 6), so that mohge_combine_bwd need not read y_perm.  With
+ * dy_perm = gate * dy (what mohge_combine_bwd writes), dH = dy_perm . W_down carries the gate,
+ * and sum_j dH_j H_j = gate * <dy, Y>: the SwiGLU-backward epilogue adds dH_j H_j over the
+ * columns of its tile per row (H recomputed from the saved A and U), a small kernel adds the
+ * tiles of a row in ascending order and divides by the gate.  A pair whose gate is exactly zero
+ * takes the definition <dy[t], y_perm[prow_of[t,k]]>.  The FP32 layer computes the definition
+ * for every pair.
+ *   dy [T, d] dtype, y_perm [rows, d] dtype, prow_of [T, K_e], gate_w [T, K_e] (inputs)
+ *   dgate_w [T, K_e] float32 (output); everything else as in mohge_expert_bwd.
+ */
+int32_t mohge_expert_bwd_dgate(const mohge_config* cfg, int64_t T, const void* dy_perm,
+                               const void* x_perm, const void* au_saved, const void* h_saved,
+                               const int32_t* counts, const int32_t* aligned_offsets,
+                               const void* const* w13, const void* const* w2, void* dau,
+                               void* dx_perm, float* const* dw13, float* const* dw2,
+                               int32_t accumulate, const void* dy, const void* y_perm,
+                               const int32_t* prow_of, const float* gate_w, float* dgate_w, void* ws,
+                               void* stream);
 
 /*
  * Backward of the permutation: dx[t, :] = sum_k dx_perm[prow_of[t,k], :] (+ dx_add[t, :]).

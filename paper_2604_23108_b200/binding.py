@@ -51,6 +51,8 @@ _SIGS = {
     "mohge_combine_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 9),
     "mohge_expert_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12
                          + [C.c_int32, _P, _P]),
+    "mohge_expert_bwd_dgate": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12
+                               + [C.c_int32] + [_P] * 7),
     "mohge_dispatch_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 5),
     "mohge_shared_fwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 8),
     "mohge_shared_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 10
@@ -234,6 +236,17 @@ def mohge_expert_bwd(cfg, T, dy_perm, x_perm, au_saved, h_saved, counts, aligned
                                   _stream()), "mohge_expert_bwd")
 
 
+def mohge_expert_bwd_dgate(cfg, T, dy_perm, x_perm, au_saved, h_saved, counts, aligned_offsets, w13, w2,
+                           dau, dx_perm, dw13, dw2, accumulate, dy, y_perm, prow_of, gate_w, dgate_w, ws):
+    a13, a2, d13, d2 = _ptr_array(w13), _ptr_array(w2), _ptr_array(dw13), _ptr_array(dw2)
+    _check(lib().mohge_expert_bwd_dgate(C.byref(cfg.c()), T, _ptr(dy_perm), _ptr(x_perm), _ptr(au_saved),
+                                        _ptr(h_saved), _ptr(counts), _ptr(aligned_offsets),
+                                        C.cast(a13, _P), C.cast(a2, _P), _ptr(dau), _ptr(dx_perm),
+                                        C.cast(d13, _P), C.cast(d2, _P), int(accumulate), _ptr(dy),
+                                        _ptr(y_perm), _ptr(prow_of), _ptr(gate_w), _ptr(dgate_w),
+                                        _ptr(ws), _stream()), "mohge_expert_bwd_dgate")
+
+
 def mohge_dispatch_bwd(cfg, T, dx_perm, prow_of, dx, dx_add=None):
     _check(lib().mohge_dispatch_bwd(C.byref(cfg.c()), T, _ptr(dx_perm), _ptr(prow_of),
                                     _ptr(dx_add), _ptr(dx), _stream()), "mohge_dispatch_bwd")
@@ -323,12 +336,21 @@ def layer_forward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, logit_bias
 
 
 def layer_backward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, dy, aux=True, accumulate=False,
-                   shared=None):
-    """combine_bwd -> expert_bwd (-> shared_bwd) -> dispatch_bwd -> route_bwd; results stay in `b`."""
+                   shared=None, fused_dgate=True):
+    """combine_bwd -> expert_bwd (-> shared_bwd) -> dispatch_bwd -> route_bwd; results stay in `b`.
+    fused_dgate: the gate gradient comes out of the experts' backward (mohge_expert_bwd_dgate) and
+    combine_bwd does not read y_perm; otherwise combine_bwd computes it from y_perm."""
     T = b.T
-    mohge_combine_bwd(cfg, T, dy, b.y_perm, b.prow_of, b.gate_w, b.counts, b.aligned, b.dy_perm, b.dgate)
-    mohge_expert_bwd(cfg, T, b.dy_perm, b.x_perm, b.au, b.h, b.counts, b.aligned, w13, w2, b.dau,
-                     b.dx_perm, b.dw13, b.dw2, accumulate, b.ws)
+    if fused_dgate:
+        mohge_combine_bwd(cfg, T, dy, None, b.prow_of, b.gate_w, b.counts, b.aligned, b.dy_perm, None)
+        mohge_expert_bwd_dgate(cfg, T, b.dy_perm, b.x_perm, b.au, b.h, b.counts, b.aligned, w13, w2,
+                               b.dau, b.dx_perm, b.dw13, b.dw2, accumulate, dy, b.y_perm, b.prow_of,
+                               b.gate_w, b.dgate, b.ws)
+    else:
+        mohge_combine_bwd(cfg, T, dy, b.y_perm, b.prow_of, b.gate_w, b.counts, b.aligned, b.dy_perm,
+                          b.dgate)
+        mohge_expert_bwd(cfg, T, b.dy_perm, b.x_perm, b.au, b.h, b.counts, b.aligned, w13, w2, b.dau,
+                         b.dx_perm, b.dw13, b.dw2, accumulate, b.ws)
     if shared is not None:
         mohge_shared_bwd(cfg, T, b.shared_width, dy, x, b.au_sh, b.h_sh, shared[0], shared[1],
                          b.dau_sh, b.dx_sh, b.dw13_sh, b.dw2_sh, accumulate, b.ws)

@@ -103,7 +103,11 @@ WsLayout ws_layout(const Dims& D) {
   const int64_t row_tiled = mt * ((wide + 63) / 64);
   const int64_t wgrad = (int64_t)D.Ne * ((2 * D.Wmax + 63) / 64) * ((D.d + 63) / 64);
   L.tiles_cap = row_tiled > wgrad ? row_tiled : wgrad;
-  L.total = L.tiles_off + 1024 + (int64_t)kMaxLists * up256(L.tiles_cap * (int64_t)sizeof(Tile));
+  L.dgp_off = L.tiles_off + 1024 + (int64_t)kMaxLists * up256(L.tiles_cap * (int64_t)sizeof(Tile));
+  // gate-gradient partial sums of the experts' backward: one float per physical row and
+  // 128-column slot of the hidden axis
+  L.dgate_slots = (D.Wmax + 127) / 128;
+  L.total = L.dgp_off + up256(D.Rcap * (int64_t)L.dgate_slots * 4);
   return L;
 }
 
@@ -117,6 +121,8 @@ struct Ws {
   int32_t* tile_count;
   Tile* tiles;
   int64_t tiles_cap;
+  float* dgp;
+  int dgate_slots;
 };
 
 static Ws carve(const Dims& D, void* ws) {
@@ -132,6 +138,8 @@ static Ws carve(const Dims& D, void* ws) {
   w.tile_count = (int32_t*)(p + L.tiles_off);
   w.tiles = (Tile*)(p + L.tiles_off + 1024);   // kMaxLists lists, tiles_cap entries apart
   w.tiles_cap = L.tiles_cap;
+  w.dgp = (float*)(p + L.dgp_off);
+  w.dgate_slots = L.dgate_slots;
   return w;
 }
 
@@ -326,17 +334,30 @@ int32_t mohge_combine_bwd(const mohge_config* cfg, int64_t T, const void* dy, co
   Dims D;
   int32_t rc = make_dims(cfg, T, &D);
   if (rc) return rc;
-  REQ_PTR(dy); REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(counts);
-  REQ_PTR(aligned_offsets); REQ_PTR(dy_perm); REQ_PTR(dgate_w);
-  return launch_combine_bwd(D, dy, y_perm, prow_of, gate_w, counts, aligned_offsets, dy_perm,
-                            dgate_w, (cudaStream_t)stream);
+  REQ_PTR(dy); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(counts);
+  REQ_PTR(aligned_offsets); REQ_PTR(dy_perm);
+  MOHGE_CHECK_ARG((y_perm == nullptr) == (dgate_w == nullptr),
+                  "y_perm and dgate_w must both be given, or both be NULL (scaled rows only)");
+  if (y_perm) { REQ_PTR(y_perm); REQ_PTR(dgate_w); }
+  return launch_combine_bwd(D, y_perm ? 0 : 1, dy, y_perm, prow_of, gate_w, counts, aligned_offsets,
+                            dy_perm, dgate_w, (cudaStream_t)stream);
 }
 
 // Backward of the grouped SwiGLU experts for already validated arguments (see expert_fwd_impl).
+// Optional by-product of the experts' backward: the gate gradient (see mohge_expert_bwd_dgate).
+struct DgateArgs {
+  const void* dy;
+  const void* y_perm;
+  const int32_t* prow_of;
+  const float* gate_w;
+  float* dgate_w;
+};
+
 static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy_perm,
                                const void* x_perm, const void* au_saved, const void* h_saved,
                                const int32_t* counts, const int32_t* aligned_offsets, void* dau,
-                               void* dx_perm, int32_t accumulate, const Ws& w, cudaStream_t st) {
+                               void* dx_perm, int32_t accumulate, const Ws& w, cudaStream_t st,
+                               const DgateArgs* dg = nullptr) {
   int32_t rc;
   if (!accumulate) {
     rc = launch_zero_empty_wgrad(D, P, counts, st);
@@ -360,10 +381,23 @@ static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy
       }
       rc = launch_tc_grouped(D, roles[r], P, A, B, C, C2, counts, aligned_offsets, accumulate,
                              w.tile_count + 64 * r, w.tiles + w.tiles_cap * r, w.tiles_cap, w.status,
-                             st, true);
+                             st, true, dg ? w.dgp : nullptr, w.dgate_slots);
       if (rc) return rc;
+      if (dg && roles[r] == ROLE_DGRAD_DOWN) {
+        int bn[MOHGE_MAX_GROUPS];
+        for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) bn[g] = g < D.Ng ? tc_dgrad_down_bn(D, g) : 128;
+        rc = launch_dgate_reduce(D, bn, w.dgp, w.dgate_slots, dg->prow_of, dg->gate_w, aligned_offsets,
+                                 dg->dy, dg->y_perm, dg->dgate_w, st);
+        if (rc) return rc;
+      }
     }
     return MOHGE_OK;
+  }
+  if (dg) {
+    // FP32 / FFMA path: the definition, <dy[t], y_perm[row]>
+    rc = launch_combine_bwd(D, 2, dg->dy, dg->y_perm, dg->prow_of, dg->gate_w, counts, aligned_offsets,
+                            nullptr, dg->dgate_w, st);
+    if (rc) return rc;
   }
   struct Step { int role; const void* A; const void* B; void* C; };
   const Step steps[4] = {{ROLE_DGRAD_DOWN, dy_perm, nullptr, dau},
@@ -403,6 +437,29 @@ int32_t mohge_expert_bwd(const mohge_config* cfg, int64_t T, const void* dy_perm
   if (rc) return rc;
   return expert_bwd_impl(D, P, dy_perm, x_perm, au_saved, h_saved, counts, aligned_offsets, dau,
                          dx_perm, accumulate, carve(D, ws), (cudaStream_t)stream);
+}
+
+int32_t mohge_expert_bwd_dgate(const mohge_config* cfg, int64_t T, const void* dy_perm,
+                               const void* x_perm, const void* au_saved, const void* h_saved,
+                               const int32_t* counts, const int32_t* aligned_offsets,
+                               const void* const* w13, const void* const* w2, void* dau,
+                               void* dx_perm, float* const* dw13, float* const* dw2,
+                               int32_t accumulate, const void* dy, const void* y_perm,
+                               const int32_t* prow_of, const float* gate_w, float* dgate_w, void* ws,
+                               void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(dy_perm); REQ_PTR(x_perm); REQ_PTR(au_saved); REQ_PTR(h_saved); REQ_PTR(counts);
+  REQ_PTR(aligned_offsets); REQ_PTR(dau); REQ_PTR(dx_perm); REQ_PTR(ws);
+  REQ_PTR(dy); REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(dgate_w);
+  MOHGE_CHECK_ARG(w13 && w2 && dw13 && dw2, "w13, w2, dw13, dw2 must be host arrays of n_groups device pointers");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, dw13, dw2, &P);
+  if (rc) return rc;
+  const DgateArgs dg = {dy, y_perm, prow_of, gate_w, dgate_w};
+  return expert_bwd_impl(D, P, dy_perm, x_perm, au_saved, h_saved, counts, aligned_offsets, dau,
+                         dx_perm, accumulate, carve(D, ws), (cudaStream_t)stream, &dg);
 }
 
 int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,

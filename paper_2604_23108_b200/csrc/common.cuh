@@ -90,7 +90,8 @@ constexpr int kStatsBlocks = 296;
 constexpr int kDispatchChunk = 256;  // tokens per dispatch block
 
 struct WsLayout {
-  int64_t status_off, stats_off, hist_off, base_off, dl16_off, rdw_off, tiles_off, total;
+  int64_t status_off, stats_off, hist_off, base_off, dl16_off, rdw_off, tiles_off, dgp_off, total;
+  int dgate_slots;       // 128-column slots per row of the gate-gradient partial sums
   int64_t tiles_cap;
   int chunks;
 };
@@ -168,9 +169,12 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
                         int32_t* status, cudaStream_t st);
 int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of,
                        const float* gate_w, const void* add, void* y, cudaStream_t st);
-int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
+int32_t launch_combine_bwd(const Dims& D, int mode, const void* dy, const void* y_perm,
                            const int32_t* prow_of, const float* gate_w, const int32_t* counts,
                            const int32_t* aligned, void* dy_perm, float* dgate_w, cudaStream_t st);
+int32_t launch_dgate_reduce(const Dims& D, const int* bn, const float* part, int slots,
+                            const int32_t* prow_of, const float* gate_w, const int32_t* aligned,
+                            const void* dy, const void* y_perm, float* dgate_w, cudaStream_t st);
 int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* prow_of,
                              const void* add, void* dx, cudaStream_t st);
 
@@ -196,7 +200,10 @@ int32_t launch_simt_plain(int M, int N, int K, const void* A, int a_f32, int64_t
 int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
                           const void* B, void* C, void* C2, const int32_t* counts,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
-                          int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt = false);
+                          int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt = false,
+                          float* dgate_part = nullptr, int dgate_slots = 0);
+// UMMA N of a group in ROLE_DGRAD_DOWN (128 or 256): which 128-column slots of dgate_part are written
+int tc_dgrad_down_bn(const Dims& D, int g);
 TilePlan tc_tile_plan(const Dims& D, int role);
 // builds up to four tile lists with one launch; list i goes to tile_count + 64 * i (ints) and
 // tiles + i * tiles_cap

@@ -282,7 +282,9 @@ combine_kernel(const Vec16* __restrict__ y_perm, const int32_t* __restrict__ pro
 }
 
 // dgate[t,k] = <dy[t], y_perm[prow[t,k]]>,  dy_perm[prow[t,k]] = gate[t,k] * dy[t]
-template <typename T>
+// MODE 0: both; MODE 1: only the scaled rows (the gate gradient then comes out of the experts'
+// backward, and y_perm is not read); MODE 2: only the gate gradient.
+template <typename T, int MODE>
 __global__ void __launch_bounds__(256)
 combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_perm,
                    const int32_t* __restrict__ prow_of, const float* __restrict__ gate_w, int Tn,
@@ -295,7 +297,7 @@ combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_per
   __shared__ float s_red[MOHGE_MAX_K_EXPERTS][8];
   if ((int)blockIdx.x >= nb_tok) {      // padding rows of dy_perm
     const int j = blockIdx.x - nb_tok;
-    zero_pad_part(counts, aligned, j >> 2, j & 3, row_vecs, dy_perm);
+    if (MODE != 2) zero_pad_part(counts, aligned, j >> 2, j & 3, row_vecs, dy_perm);
     return;
   }
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -306,6 +308,21 @@ combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_per
       s_g[threadIdx.x] = gate_w[(size_t)t * Ke + threadIdx.x];
     }
     __syncthreads();
+    if (MODE == 1) {
+      // one read of dy[t], K_e scaled copies
+      for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
+        float a[8], o[8];
+        unpack(dy[(size_t)t * row_vecs + c], a, T());
+        for (int k = 0; k < Ke; ++k) {
+          if ((unsigned)s_row[k] >= (unsigned)rows_cap) continue;
+          const float g = s_g[k];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) o[i] = g * a[i];
+          dy_perm[(size_t)s_row[k] * row_vecs + c] = pack(o, T());
+        }
+      }
+      continue;
+    }
     for (int k = 0; k < Ke; ++k) {
       float part = 0.0f;
       const float g = s_g[k];
@@ -322,7 +339,7 @@ combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_per
           part = fmaf(a[i], b[i], part);
           o[i] = g * a[i];
         }
-        dy_perm[rbase + c] = pack(o, T());
+        if (MODE == 0) dy_perm[rbase + c] = pack(o, T());
       }
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) part += __shfl_xor_sync(kFull, part, off);
@@ -334,6 +351,59 @@ combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_per
       for (int w = 0; w < nwarps; ++w) v += s_red[threadIdx.x][w];
       dgate_w[(size_t)t * Ke + threadIdx.x] = v;
     }
+  }
+}
+
+// Gate gradient from the partial sums the SwiGLU-backward epilogue leaves per physical row and
+// 128-column slot: sum_j dH_j h_j with dH = (gate * dy) W2, i.e. gate * <dy, Y>; the slots are
+// added in ascending order (fixed) and the sum is divided by the gate.  A gate that is exactly
+// zero left a zero row in dy_perm; such a pair takes the definition <dy[t], y_perm[row]> instead.
+struct DgateShape {
+  int N, Ne, Ke, slots, d;
+  int W[MOHGE_MAX_GROUPS];
+  int step[MOHGE_MAX_GROUPS];      // tile width of the group / 128: every step-th slot is written
+};
+
+template <typename T>
+__device__ __forceinline__ float as_float(T v);
+template <>
+__device__ __forceinline__ float as_float<float>(float v) { return v; }
+template <>
+__device__ __forceinline__ float as_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+dgate_reduce_kernel(DgateShape s, int n, const float* __restrict__ part,
+                    const int32_t* __restrict__ prow_of, const float* __restrict__ gate_w,
+                    const int32_t* __restrict__ aligned, const T* __restrict__ dy,
+                    const T* __restrict__ y_perm, int rows_cap, float* __restrict__ dgate_w) {
+  pdl_enter();
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < n; idx += gridDim.x * blockDim.x) {
+    const int r = prow_of[idx];
+    float v = 0.0f;
+    if ((unsigned)r < (unsigned)rows_cap) {
+      const float gate = gate_w[idx];
+      if (gate != 0.0f) {
+        int lo = 0, hi = s.Ne;           // aligned[lo] <= r < aligned[hi]: lo ends at the row's expert
+        while (hi - lo > 1) {
+          const int mid = (lo + hi) >> 1;
+          if (aligned[mid] <= r) lo = mid; else hi = mid;
+        }
+        const int g = lo / s.N;
+        const float* pr = part + (size_t)r * s.slots;
+        const int ns = (s.W[g] + 127) >> 7;
+        float acc = 0.0f;
+        for (int j = 0; j < ns; j += s.step[g]) acc += pr[j];
+        v = acc / gate;
+      } else {
+        const size_t t = (size_t)(idx / s.Ke);
+        float acc = 0.0f;
+        for (int c = 0; c < s.d; ++c)
+          acc = fmaf(as_float<T>(dy[t * s.d + c]), as_float<T>(y_perm[(size_t)r * s.d + c]), acc);
+        v = acc;
+      }
+    }
+    dgate_w[idx] = v;
   }
 }
 
@@ -394,25 +464,58 @@ int32_t launch_unpermute_sum(const Dims& D, const void* dx_perm, const int32_t* 
   return launch_combine(D, dx_perm, prow_of, nullptr, add, dx, st);
 }
 
-int32_t launch_combine_bwd(const Dims& D, const void* dy, const void* y_perm,
+int32_t launch_dgate_reduce(const Dims& D, const int* bn, const float* part, int slots,
+                            const int32_t* prow_of, const float* gate_w, const int32_t* aligned,
+                            const void* dy, const void* y_perm, float* dgate_w, cudaStream_t st) {
+  if (D.T == 0) return MOHGE_OK;
+  DgateShape s;
+  s.N = D.N; s.Ne = D.Ne; s.Ke = D.Ke; s.slots = slots; s.d = D.d;
+  for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) {
+    s.W[g] = g < D.Ng ? D.W[g] : 0;
+    s.step[g] = g < D.Ng ? bn[g] / 128 : 1;
+  }
+  const int n = (int)(D.T * D.Ke);
+  const int blocks = (n + 255) / 256 < 148 * 8 ? (n + 255) / 256 : 148 * 8;
+  if (D.bf16)
+    launch_dep(dgate_reduce_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), st, s, n, part, prow_of, gate_w,
+               aligned, (const __nv_bfloat16*)dy, (const __nv_bfloat16*)y_perm, (int)D.Rcap, dgate_w);
+  else
+    launch_dep(dgate_reduce_kernel<float>, dim3(blocks), dim3(256), st, s, n, part, prow_of, gate_w, aligned,
+               (const float*)dy, (const float*)y_perm, (int)D.Rcap, dgate_w);
+  MOHGE_LAUNCH_CHECK("dgate_reduce_kernel");
+  return MOHGE_OK;
+}
+
+template <typename T, int MODE>
+static void launch_combine_bwd_mode(const Dims& D, int blocks, int pad_blocks, int row_vecs, const void* dy,
+                                    const void* y_perm, const int32_t* prow_of, const float* gate_w,
+                                    const int32_t* counts, const int32_t* aligned, void* dy_perm,
+                                    float* dgate_w, cudaStream_t st) {
+  launch_dep(combine_bwd_kernel<T, MODE>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st,
+             (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, (int)D.T, D.Ke, row_vecs, (int)D.Rcap,
+             (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
+}
+
+// mode 0: dy_perm and dgate_w; 1: dy_perm only (y_perm, dgate_w unused); 2: dgate_w only
+int32_t launch_combine_bwd(const Dims& D, int mode, const void* dy, const void* y_perm,
                            const int32_t* prow_of, const float* gate_w, const int32_t* counts,
                            const int32_t* aligned, void* dy_perm, float* dgate_w, cudaStream_t st) {
   const int T = (int)D.T;
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
-  const int pad_blocks = D.align > 1 ? 4 * D.Ne : 0;
+  const int pad_blocks = (D.align > 1 && mode != 2) ? 4 * D.Ne : 0;
   if (T > 0) {
     const int blocks = T < 148 * 16 ? T : 148 * 16;
-    if (D.bf16)
-      launch_dep(combine_bwd_kernel<__nv_bfloat16>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st,
-          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
-          (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
-    else
-      launch_dep(combine_bwd_kernel<float>, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st,
-          (const Vec16*)dy, (const Vec16*)y_perm, prow_of, gate_w, T, D.Ke, row_vecs, (int)D.Rcap,
-          (Vec16*)dy_perm, dgate_w, blocks, counts, aligned);
+#define MOHGE_CB(TT, MM) launch_combine_bwd_mode<TT, MM>(D, blocks, pad_blocks, row_vecs, dy, y_perm, prow_of, \
+                                                        gate_w, counts, aligned, dy_perm, dgate_w, st)
+    if (D.bf16) {
+      if (mode == 0) MOHGE_CB(__nv_bfloat16, 0); else if (mode == 1) MOHGE_CB(__nv_bfloat16, 1); else MOHGE_CB(__nv_bfloat16, 2);
+    } else {
+      if (mode == 0) MOHGE_CB(float, 0); else if (mode == 1) MOHGE_CB(float, 1); else MOHGE_CB(float, 2);
+    }
+#undef MOHGE_CB
     MOHGE_LAUNCH_CHECK("combine_bwd_kernel");
   }
-  if (D.align > 1 && T == 0) {
+  if (D.align > 1 && T == 0 && mode != 2) {
     launch_dep(zero_pad_rows_kernel, dim3(D.Ne, 4), dim3(256), st, counts, aligned, row_vecs, (Vec16*)dy_perm);
     MOHGE_LAUNCH_CHECK("zero_pad_rows_kernel");
   }

@@ -109,6 +109,10 @@ struct TcParams {
   int plain_splits, plain_kchunk;   // split-K of ROUTER_DW and LOGITS: ranges of plain_kchunk k-blocks
   float* Cf;                     // LOGITS: logits [T, NL]; ROUTER_DW: dw_router [NL, d]
   const float* bias;             // LOGITS: optional logit bias [NL]
+  // DGRAD_DOWN, optional: per physical row and 128-column slot of the hidden axis, the sum over
+  // the tile's columns of dH_j * h_j (the gate gradient times the gate, see dgate_reduce_kernel)
+  float* dgate_part;
+  int dgate_slots;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -832,6 +836,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       } else if (RT::EPI == EPI_SWIGLU_BWD) {
         // per 64-column chunk: A and U arrive by TMA in one of two buffer pairs, dA and dU are
         // written over them in place and leave by TMA; the next chunk's loads fly meanwhile
+        float2 dg2 = make_float2(0.0f, 0.0f);          // sum over this tile's columns of dH * h
         for (int ci = 0; ci < nch_in; ++ci, ++n_chunk) {
           const int c = ci * 64;
           const uint32_t set = n_chunk & 1u;
@@ -877,6 +882,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
                 const float2 dhs = __fmul2_rn(dh2, s2);
                 const float2 du2 = __fmul2_rn(dhs, a2);                                 // dh * silu(a)
                 const float2 da2 = __fmul2_rn(__fmul2_rn(dhs, u2), t2);                 // dh * u * silu'(a)
+                dg2 = __ffma2_rn(du2, u2, dg2);                                         // dh * h
                 oa[j4][e2] = pack2(da2.x, da2.y);
                 ou[j4][e2] = pack2(du2.x, du2.y);
               }
@@ -896,6 +902,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           }
         }
         if (!alive) break;
+        // nch_in > 0 only for CTAs whose rows lie inside the expert's segment (padding rows give 0)
+        if (p.dgate_part != nullptr && nch_in > 0)
+          p.dgate_part[(size_t)(row0 + lane) * p.dgate_slots + (q.n0 >> 7)] = dg2.x + dg2.y;
       } else if (RT::EPI == EPI_F32) {
         // weight gradients: FP32 boxes of 32 rows x 32 columns into [expert, rows, columns]
         const int Mext = ROLE == ROLE_WGRAD_DOWN ? (int)d : 2 * q.W;
@@ -1330,6 +1339,11 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
 // Tile list plan of a grouped role (tile widths per group, pair rows, double-width flag): the same
 // choices launch_tc_grouped makes, so that the lists of several roles can be built by one launch
 // before the GEMMs run.
+int tc_dgrad_down_bn(const Dims& D, int g) {
+  const int cand_n[2] = {256, 128};
+  return pick_bn(D.W[g], cand_n, 2);
+}
+
 TilePlan tc_tile_plan(const Dims& D, int role) {
   const int CG = cta_group_size(D);
   const int cand_n[2] = {256, 128};
@@ -1351,7 +1365,8 @@ TilePlan tc_tile_plan(const Dims& D, int role) {
 int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
                           const void* B, void* C, void* C2, const int32_t* /*counts*/,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
-                          int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt) {
+                          int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt,
+                          float* dgate_part, int dgate_slots) {
   static int sm_count = 0;
   if (!sm_count) {
     int dev = 0;
@@ -1371,6 +1386,8 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   p.aligned = aligned; p.tile_count = tile_count; p.tiles = tiles;
   p.C = (__nv_bfloat16*)C; p.C2 = (__nv_bfloat16*)C2; p.E = nullptr;
   p.accumulate = accumulate; p.status = status;
+  p.dgate_part = role == ROLE_DGRAD_DOWN ? dgate_part : nullptr;
+  p.dgate_slots = dgate_slots;
 
   const uint64_t d = D.d, rows = D.Rcap, pitchAU = 2ull * D.Wmax * 2, pitchH = (uint64_t)D.Wmax * 2;
   const int CG = cta_group_size(D);

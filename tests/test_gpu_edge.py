@@ -154,3 +154,21 @@ def test_single_expert_layer_is_a_plain_ffn(dtype):
     assert np.abs(bwd["dlogits"]).max() <= 1e-12 * scale
     assert float(b.dlogits.abs().max()) <= 1e-6 * scale
     assert float(b.dw_router.abs().max()) <= 1e-6 * scale * wl.T
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gate_that_is_exactly_zero_still_gets_its_gradient(dtype):
+    """One of the two selected experts has a score that underflows to 0 in the float32 contract,
+    so its gate is exactly 0 and its row of dy_perm is zero; its gate gradient <dy, Y> is not."""
+    wl = Workload("zero_gate", dtype, 200, 64, 1, 2, (96,), 1, 2, seed=11)
+    inp = make_inputs(wl)
+    logits = np.zeros((wl.T, wl.n_logits), np.float32)
+    logits[:, 2] = -200.0                      # second expert: exp_s(-200) = 0
+    fwd, bwd, _ = oracle_layer(wl, inp, logits32=logits)
+    b, dev = gpu_layer(wl, inp, logits32=logits)
+    g = b.gate_w.cpu().numpy()
+    assert (g[:, 0] == 1.0).all() and (g[:, 1] == 0.0).all()
+    assert (b.expert_idx.cpu().numpy() == fwd["expert_idx"]).all()
+    assert np.abs(bwd["dgate"][:, 1]).max() > 0
+    assert max_rel(to_np64(b.dgate), bwd["dgate"]) <= tol_for(dtype)
+    assert max_rel(to_np64(b.y), fwd["y"]) <= tol_for(dtype)

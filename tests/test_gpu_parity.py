@@ -179,3 +179,30 @@ def test_accumulate_adds_into_weight_gradients(switch, monkeypatch):
     for g in range(wl.n_groups):
         assert max_rel(to_np64(b.dw13[g]), 2 * to_np64(ref13[g])) <= 1e-6
         assert max_rel(to_np64(b.dw2[g]), 2 * to_np64(ref2[g])) <= 1e-6
+
+
+def test_gate_gradient_from_the_experts_backward_and_from_y_perm(case):
+    """The layer's default backward takes the gate gradient out of the SwiGLU-backward epilogue;
+    the other route computes <dy, y_perm> in combine_bwd.  Both meet the oracle, and nothing else
+    in the backward depends on which one ran."""
+    wl, inp, fwd, bwd, logits32, b, dev = case
+    tol = tol_for(wl.dtype)
+    assert max_rel(to_np64(b.dgate), bwd["dgate"]) <= tol
+    fused = {k: getattr(b, k).clone() for k in ("dgate", "dx", "dlogits", "dw_router", "dy_perm", "dau")}
+    fused_dw = [t.clone() for t in b.dw13] + [t.clone() for t in b.dw2]
+    B.layer_backward(gpu_cfg(wl), b, dev["x"], dev["w_router"], dev["w13"], dev["w2"], dev["dy"],
+                     aux=True, fused_dgate=False)
+    torch.cuda.synchronize()
+    assert B.mohge_get_device_status(b.ws) == 0
+    assert max_rel(to_np64(b.dgate), bwd["dgate"]) <= tol
+    assert max_rel(to_np64(b.dgate), to_np64(fused["dgate"])) <= tol
+    # same bits either way (compared as integers: columns past a narrow group's width are never
+    # written and may hold NaN patterns)
+    bits = lambda t: t.view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32)
+    for k in ("dy_perm", "dau"):
+        assert torch.equal(bits(getattr(b, k)), bits(fused[k])), k
+    for t_new, t_old in zip(list(b.dw13) + list(b.dw2), fused_dw):
+        assert torch.equal(t_new, t_old)
+    # dx, dlogits, dw_router take dgate as an input: equal within the tolerance
+    for k in ("dx", "dlogits", "dw_router"):
+        assert max_rel(to_np64(getattr(b, k)), to_np64(fused[k])) <= tol, k
