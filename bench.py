@@ -417,6 +417,10 @@ def main():
                "overlap": "uploads and downloads on their own streams, double-buffered",
                "checked": "last download equals a device-only step bit for bit"}
 
+    status = B.mohge_get_device_status(buf.ws)
+    if status != 0:
+        raise SystemExit("device status word = 0x%x after the timed region" % status)
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -466,7 +470,7 @@ def main():
                    "pass": "forward only" if args.forward_only else "forward + backward",
                    "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only",
                    "launch": "CUDA graph replay" if args.graph else "stream launches"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "device_status": status,
         "roofline": roofline, "cpu_baseline": cpu_baseline,
     }
     print(json.dumps(line), flush=True)
