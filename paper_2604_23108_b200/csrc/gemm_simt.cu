@@ -55,30 +55,49 @@ build_tiles_body(const TilePlan& p, const int32_t* __restrict__ aligned, int32_t
     s_order[rank] = e;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x < 32) {
+    // first tile of every rank (exclusive prefix sum over the sorted experts) and the range of
+    // the costs per tile, by one warp: 32 ranks per round, a shuffle scan inside the round
+    const int lane = threadIdx.x;
     int run = 0;
-    for (int r = 0; r < p.Ne; ++r) {
-      s_start[r] = run;
-      run += s_nt[s_order[r]];
-    }
-    s_start[p.Ne] = run;
-    if (run > cap) {
-      if (blockIdx.x == 0) atomicCAS(status, 0, (2 << 24) | 2);
-      s_start[p.Ne] = 0;
-    }
-    if (blockIdx.x == 0) {
-      tile_count[0] = s_start[p.Ne];
-      // tile_count[1]: 1 when the costs per tile differ by more than a quarter between experts
-      // (skewed routing, or groups of different contraction length): the persistent CTAs then
-      // walk the sorted list in alternating directions
-      long long lo = -1, hi = -1;
-      for (int r = 0; r < p.Ne; ++r) {
-        const long long c = s_cost[r];
-        if (c <= 0) continue;
+    long long lo = -1, hi = -1;
+    for (int base = 0; base < p.Ne; base += 32) {
+      const int r = base + lane;
+      const int v = r < p.Ne ? s_nt[s_order[r]] : 0;
+      int inc = v;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, inc, off);
+        if (lane >= off) inc += up;
+      }
+      if (r < p.Ne) s_start[r] = run + inc - v;
+      run += __shfl_sync(0xffffffffu, inc, 31);
+      const long long c = r < p.Ne ? s_cost[r] : -1;
+      if (c > 0) {
         if (lo < 0 || c < lo) lo = c;
         if (c > hi) hi = c;
       }
-      tile_count[1] = (lo > 0 && hi * 4 > lo * 5) ? 1 : 0;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const long long olo = __shfl_xor_sync(0xffffffffu, lo, off);
+      const long long ohi = __shfl_xor_sync(0xffffffffu, hi, off);
+      if (olo > 0 && (lo < 0 || olo < lo)) lo = olo;
+      if (ohi > hi) hi = ohi;
+    }
+    if (lane == 0) {
+      s_start[p.Ne] = run;
+      if (run > cap) {
+        if (blockIdx.x == 0) atomicCAS(status, 0, (2 << 24) | 2);
+        s_start[p.Ne] = 0;
+      }
+      if (blockIdx.x == 0) {
+        tile_count[0] = s_start[p.Ne];
+        // tile_count[1]: 1 when the costs per tile differ by more than a quarter between experts
+        // (skewed routing, or groups of different contraction length): the persistent CTAs then
+        // walk the sorted list in alternating directions
+        tile_count[1] = (lo > 0 && hi * 4 > lo * 5) ? 1 : 0;
+      }
     }
   }
   __syncthreads();
