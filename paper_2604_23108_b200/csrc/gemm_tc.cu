@@ -59,10 +59,13 @@ constexpr int kStgBytes = 4 * kStgBufs * kStgBufBytes;       // 64 KiB per CTA
 // and the pair's halves of both B tiles (48 KiB per CTA, three stages), which cuts the operand
 // bytes per FLOP by a quarter; the price is that the epilogue of an entry no longer overlaps
 // the MMAs of the next one.  It pays where the contraction is long (see launch_tc_grouped).
+// WIDE = 2 (single CTAs, router logits with at most 160 outputs): a B tile of 20 KiB instead of
+// 32, so the same shared memory holds four stages instead of three.  That GEMM streams x once and
+// is bound by the bytes it keeps in flight against the memory latency.
 template <int CG, int WIDE = 0> struct Geo {
-  static constexpr int kStages = (CG == 2 && !WIDE) ? 5 : 3;
-  static constexpr int kBBytes = 256 / CG * BK * 2;          // one B tile per CTA: 32 KiB or 16 KiB
-  static constexpr int kStageBytes = kABytes + kBBytes * (WIDE ? 2 : 1);
+  static constexpr int kStages = WIDE == 2 ? 4 : (CG == 2 && !WIDE) ? 5 : 3;
+  static constexpr int kBBytes = WIDE == 2 ? 160 * BK * 2 : 256 / CG * BK * 2;   // one B tile per CTA: 32 KiB or 16 KiB
+  static constexpr int kStageBytes = kABytes + kBBytes * (WIDE == 1 ? 2 : 1);
   static constexpr int kSmemBytes = kStages * kStageBytes + kStgBytes + 1024 + 512 + 1088;   // + segment table
   static constexpr int kTileM = BM * CG;
 };
@@ -1309,7 +1312,8 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
   const int grid = p.plain_total < sm_count ? p.plain_total : sm_count;
   switch (role) {
     case ROLE_LOGITS: {
-      const int32_t rc2 = launch_role<ROLE_LOGITS, 1>(p, grid, st);
+      const int32_t rc2 = p.BN[0] <= 160 ? launch_role<ROLE_LOGITS, 1, 2>(p, grid, st)
+                                          : launch_role<ROLE_LOGITS, 1>(p, grid, st);
       if (rc2 || p.plain_splits == 1) return rc2;
       const size_t n = (size_t)D.T * D.NL;
       launch_dep(sum_partials_bias_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), st, partials, p.plain_splits, n, D.NL,
