@@ -61,3 +61,20 @@ def test_sizes_and_validation_without_a_device():
                              None, C.c_void_p(16), None) == -1
     assert b"16-byte" in lib.mohge_last_error()
     assert lib.mohge_route(C.byref(good), -5, *([None] * 12)) == -1
+
+
+def test_combine_bwd_takes_y_perm_and_dgate_together_or_not_at_all():
+    """mohge_combine_bwd computes the gate gradient from y_perm, or neither reads the one nor
+    writes the other (the gradient then comes from mohge_expert_bwd_dgate); a call that gives only
+    one of the two is refused before any launch."""
+    lib = B.lib()
+    good = B.Config(1024, 3, 8, 2, 4, [1408, 704, 352]).c()
+    p = C.c_void_p(256)                    # never dereferenced: the call is refused first
+    args = lambda y_perm, dgate: (C.byref(good), 128, p, y_perm, p, p, p, p, p, dgate, None)
+    assert lib.mohge_combine_bwd(*args(p, None)) == -1
+    assert b"both" in lib.mohge_last_error()
+    assert lib.mohge_combine_bwd(*args(None, p)) == -1
+    # the fused backward wants every pointer of its gate-gradient part
+    rc = lib.mohge_expert_bwd_dgate(C.byref(good), 128, *([p] * 6), None, None, p, p, None, None, 0,
+                                    p, None, p, p, p, p, None)
+    assert rc == -1 and b"y_perm" in lib.mohge_last_error()
