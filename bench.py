@@ -243,7 +243,7 @@ def main():
     ev = lambda: torch.cuda.Event(enable_timing=True)
     gemm_marks = []
 
-    def step(mark=False, y=None, dx=None):
+    def step(mark=False, y=None, dx=None, after_fwd=None, before_bwd=None):
         y = buf.y if y is None else y
         dx = buf.dx if dx is None else dx
         B.mohge_route(gcfg, T, inp["x"], inp["w_router"], inp["logit_bias"], None, buf.logits,
@@ -264,10 +264,14 @@ def main():
             e1.record()
         B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, y,
                         y_add=buf.y_sh if shared is not None else None)
+        if after_fwd is not None:
+            after_fwd()                     # y is final here (the end-to-end arm starts its download)
         if args.forward_only:
             if mark:
                 gemm_marks.append((e0, e1, e1, e1))
             return
+        if before_bwd is not None:
+            before_bwd()                    # dy is first read below (the end-to-end arm waits for its upload)
         # the gate gradient comes out of the experts' backward, so combine_bwd reads no y_perm
         B.mohge_combine_bwd(gcfg, T, inp["dy"], None, buf.prow_of, buf.gate_w, buf.counts,
                             buf.aligned, buf.dy_perm, None)
@@ -358,8 +362,10 @@ def main():
         ddx_out = [torch.empty_like(buf.dx) for _ in range(2)]
         dloss_out = [torch.empty_like(buf.loss) for _ in range(2)]
         s_up, s_down, s_main = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
-        up_done = [torch.cuda.Event() for _ in range(2)]
+        x_done = [torch.cuda.Event() for _ in range(2)]
+        dy_done = [torch.cuda.Event() for _ in range(2)]
         in_free = [torch.cuda.Event() for _ in range(2)]
+        y_ready = [torch.cuda.Event() for _ in range(2)]
         out_ready = [torch.cuda.Event() for _ in range(2)]
         out_free = [torch.cuda.Event() for _ in range(2)]
         for e_ in in_free + out_free:
@@ -370,18 +376,26 @@ def main():
             with torch.cuda.stream(s_up):
                 s_up.wait_event(in_free[k])
                 dx_in[k].copy_(hx, non_blocking=True)
+                x_done[k].record(s_up)                         # the forward needs x only
                 ddy_in[k].copy_(hdy, non_blocking=True)
-                up_done[k].record(s_up)
-            s_main.wait_event(up_done[k])
+                dy_done[k].record(s_up)
+            s_main.wait_event(x_done[k])
             inp["x"], inp["dy"] = dx_in[k], ddy_in[k]
             s_main.wait_event(out_free[k])
-            step(y=dy_out[k], dx=ddx_out[k])                   # y and dx go to this step's own set,
-            in_free[k].record(s_main)                          # so the next step need not wait for
-            dloss_out[k].copy_(buf.loss, non_blocking=True)    # their download
+
+            def after_fwd():                                   # y goes home while the backward runs
+                y_ready[k].record(s_main)
+                with torch.cuda.stream(s_down):
+                    s_down.wait_event(y_ready[k])
+                    hy[k].copy_(dy_out[k], non_blocking=True)
+
+            step(y=dy_out[k], dx=ddx_out[k], after_fwd=after_fwd,      # y and dx go to this step's
+                 before_bwd=lambda: s_main.wait_event(dy_done[k]))     # own set of buffers
+            in_free[k].record(s_main)
+            dloss_out[k].copy_(buf.loss, non_blocking=True)
             out_ready[k].record(s_main)
             with torch.cuda.stream(s_down):
                 s_down.wait_event(out_ready[k])
-                hy[k].copy_(dy_out[k], non_blocking=True)
                 hdx[k].copy_(ddx_out[k], non_blocking=True)
                 hloss[k].copy_(dloss_out[k], non_blocking=True)
                 out_free[k].record(s_down)
@@ -414,7 +428,8 @@ def main():
         e2e = {"value": world * T / (ms / n_e2e * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": 2 * hx.numel() * es,
                "d2h_bytes_per_step": 2 * hx.numel() * es + 16,
-               "overlap": "uploads and downloads on their own streams, double-buffered",
+               "overlap": "uploads and downloads on their own streams, double-buffered; the forward "
+                          "starts when x has arrived, y leaves while the backward runs",
                "checked": "last download equals a device-only step bit for bit"}
 
     status = B.mohge_get_device_status(buf.ws)
