@@ -34,7 +34,7 @@ from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs
 # capture summarised in profiles/launch_list_layer_step_cfg5.md (the L2 hit rate of these launches
 # differs between the GPUs of the pool: captures of the same build range over tens of GB); workloads without a
 # capture of the current kernels report null.
-NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 74.2e9}
+NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 74.3e9}
 
 METRIC = "MoHGE layer fwd+bwd tokens/s"
 METRIC_FWD = "MoHGE layer fwd tokens/s"
