@@ -78,3 +78,39 @@ def test_combine_bwd_takes_y_perm_and_dgate_together_or_not_at_all():
     rc = lib.mohge_expert_bwd_dgate(C.byref(good), 128, *([p] * 6), None, None, p, p, None, None, 0,
                                     p, None, p, p, p, p, None)
     assert rc == -1 and b"y_perm" in lib.mohge_last_error()
+
+
+def test_header_and_library_are_usable_from_plain_c(tmp_path):
+    """A C99 program includes mohge.h, links libmohge.so and asks for sizes (no device needed)."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    from paper_2604_23108_b200.build import build
+    build()
+    pkg = os.path.join(ROOT, "paper_2604_23108_b200")
+    src = tmp_path / "sizes.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include <string.h>
+#include "mohge.h"
+int main(void) {
+  mohge_config c;
+  memset(&c, 0, sizeof c);
+  c.d_model = 1024; c.n_groups = 3; c.experts_per_group = 8; c.k_groups = 2; c.k_experts = 4;
+  c.group_width[0] = 1408; c.group_width[1] = 704; c.group_width[2] = 352;
+  c.dtype = MOHGE_BF16; c.alpha_g = 1e-4f; c.alpha_e = 2.5e-3f; c.eps = 1e-20f;
+  c.f_norm_by_T = 1; c.fe_mode = 0; c.row_align = 128;
+  printf("%lld %lld\n", (long long)mohge_workspace_bytes(&c, 8192), (long long)mohge_perm_rows(&c, 8192));
+  c.k_experts = 17;                      /* more than K_g * N: refused */
+  printf("%lld %s\n", (long long)mohge_workspace_bytes(&c, 8192), mohge_last_error());
+  return 0;
+}
+''')
+    exe = tmp_path / "sizes"
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", str(src), "-I", os.path.join(ROOT, "include"),
+                    "-L", pkg, "-lmohge", "-Wl,-rpath," + pkg, "-o", str(exe)], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split("\n")
+    cfg = B.Config(1024, 3, 8, 2, 4, [1408, 704, 352])
+    assert out[0].split() == [str(B.mohge_workspace_bytes(cfg, 8192)), str(B.mohge_perm_rows(cfg, 8192))]
+    assert out[1].startswith("0 ") and "k_experts" in out[1]
