@@ -466,7 +466,7 @@ def main():
         roofline.update(bound="alu", peak=None, frac=None,
                         kernel="simt_grouped_kernel (FP32 FMA; correctness configuration)")
     cpu_baseline = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:      # timed at N = 1 only: the other GPUs would wait
         sample = min(wl.T, args.ref_sample)
         cpu_inp = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in inp.items()
                    if k not in ("w13", "w2")}
