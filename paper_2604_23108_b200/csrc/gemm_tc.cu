@@ -45,14 +45,30 @@ constexpr int kABytes = BM * BK * 2;          // 16 KiB: 128 rows of A per CTA a
 constexpr int kThreads = 192;
 constexpr int kAccCols = 256;                 // tensor-memory columns per accumulator buffer
 
+// Build-time option -DMOHGE_TC_COUNTERS: every CTA adds, per role, the clocks its MMA issuer spent
+// in its loop, waiting for operands (full barriers) and waiting for a free accumulator (the
+// exposed part of the epilogue), the clocks per k-block in the middle of long tiles (steady
+// state), the clocks its producer waited for a free stage, the clocks the first epilogue warp
+// waited for an accumulator, the tiles and k-blocks it processed and its lifetime in
+// nanoseconds.  mohge_debug_tc_counters() copies the table to the host.  This is how the balance
+// of the tile scheduler over the SMs and the cost of the tile boundaries are measured.  Off in
+// the normal build; with it MOHGE_TC_GRID=<n> also limits the persistent grid to n CTAs.
+#ifdef MOHGE_TC_COUNTERS
+constexpr int kCntRoles = 9, kCntCtas = 160, kCntSlots = 12;
+__device__ unsigned long long g_tc_counters[kCntRoles][kCntCtas][kCntSlots];
+#define TCC(...) __VA_ARGS__
+#else
+#define TCC(...)
+#endif
+
 // CG = CTAs per MMA (tcgen05 cta_group).  CG = 2 pairs the two CTAs of a cluster on one
 // 256 x N tile: each CTA stages its own 128 rows of A and HALF of B, so operand traffic per FLOP
 // drops by a third and the smaller stages allow a five-deep pipeline.
 // Epilogue staging: each of the four epilogue warps owns a ring of four 4 KiB buffers
 // (32 rows x 128 bytes, 128-byte swizzle: the layout a TMA box of 32 rows expects).
 constexpr int kStgBufBytes = 4096;
-constexpr int kStgBufs = 4;
-constexpr int kStgBytes = 4 * kStgBufs * kStgBufBytes;       // 64 KiB per CTA
+constexpr int kSlots = 4;
+constexpr int kStgBytes = 4 * kSlots * kStgBufBytes;         // 64 KiB per CTA
 
 // WIDE = 1 (CTA pairs only): the pair works on double-width entries, 256 x 512 outputs from ONE
 // pass over A, the two 256-column halves in the two accumulator buffers.  A stage then holds A
@@ -89,7 +105,8 @@ struct TcParams {
   CUtensorMap mapA[MOHGE_MAX_GROUPS];
   CUtensorMap mapB[MOHGE_MAX_GROUPS];
   // epilogue outputs, boxes of 32 rows x 128 bytes.  FWD1: A, U, H regions per group;
-  // FWD2 / DGRAD_13: [0][0]; DGRAD_DOWN: dA, dU regions per group; WGRAD: FP32 [N, rows, cols]
+  // FWD2 / DGRAD_13 / ROUTER_DX: [0][0]; DGRAD_DOWN: dA, dU regions per group; WGRAD: FP32
+  // [N, rows, cols]
   CUtensorMap mapO[3][MOHGE_MAX_GROUPS];
   CUtensorMap mapE[2][MOHGE_MAX_GROUPS];   // DGRAD_DOWN epilogue inputs: saved A and U regions
   GroupShape gs;
@@ -201,15 +218,15 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "l"(pol) : "memory");
 }
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t pol) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(pol) : "memory");
-}
 // element-wise FP32 add into global memory (each output element is touched by exactly one box)
 __device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
   asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void bulk_wait_read() {
@@ -483,6 +500,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  TCC(const uint64_t cnt_t0 = global_ns();
+      unsigned long long* const cnt = g_tc_counters[ROLE][blockIdx.x < kCntCtas ? blockIdx.x : kCntCtas - 1];)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -547,6 +566,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
+      TCC(long long c_empty = 0;)
       Tile t_pf = prefetch_tile(it0);
       for (int it = it0; it < it_end && alive; it += it_step) {
         const int ti = zigzag ? tile_of(it) : it;
@@ -561,7 +581,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         const uint32_t tx = kABytes + (uint32_t)pieces * nb * BK * 2;
         const int am0 = q.m0 + BM * (int)cta_rank;         // this CTA's 128 rows of the tile
         for (int kb = 0; kb < q.num_kb; ++kb) {
+          TCC(const long long w0 = clock64();)
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1)) { alive = false; break; }
+          TCC(c_empty += clock64() - w0;)
           const uint32_t sA = smem_base + stage * kStageBytes;
           // CG == 2: both CTAs report to the full barrier of the pair's leader (rank 0)
           const uint32_t fb = CG == 2 ? mapa_rank(full_bar(stage), 0) : full_bar(stage);
@@ -606,6 +628,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
+      TCC(atomicAdd(&cnt[4], (unsigned long long)c_empty);)
     }
   } else if (warp == 1) {
     // ================= MMA issuer =================
@@ -615,6 +638,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       int buf = 0;
       uint32_t acc_phase = 0;
       bool alive = true;
+      TCC(long long c_w0 = 0, c_full = 0, c_tempty = 0, c_tiles = 0, c_kb = 0, c_mid0 = 0, c_mid = 0, c_midn = 0; const long long c_start = clock64();)
       // MMAs of one k-block into accumulator column base d_tmem from the B tile at sB
       auto issue_kblock = [&](uint32_t d_tmem, uint32_t sA, uint32_t sB, uint32_t idesc, bool first) {
 #pragma unroll
@@ -637,15 +661,21 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         t_pf = prefetch_tile(it + it_step);
         if (ti < 0) continue;
         const TileGeom q = tile_geom<ROLE>(p, t, s_seg);
+        TCC(c_tiles += 1; c_kb += q.num_kb * ((WIDE && q.wide) ? 2 : 1);)
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
                                ((uint32_t)RT::B_MN << 16) | ((uint32_t)(q.bn >> 3) << 17) |
                                ((uint32_t)(G::kTileM >> 4) << 24);
         if (!WIDE || !q.wide) {
+          TCC(c_w0 = clock64();)
           if (!mbar_wait(tempty_bar(buf), acc_phase ^ 1u, abort_flag, p.status, 2)) { alive = false; break; }
+          TCC(c_tempty += clock64() - c_w0;)
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * kAccCols;
           for (int kb = 0; kb < q.num_kb; ++kb) {
+            TCC(c_w0 = clock64();)
             if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
+            TCC(c_full += clock64() - c_w0;
+                if (q.num_kb >= 32) { if (kb == 8) c_mid0 = clock64(); if (kb == 24) { c_mid += clock64() - c_mid0; c_midn += 16; } })
             tc_fence_after();
             const uint32_t sA = smem_base + stage * kStageBytes;
             issue_kblock(d_tmem, sA, sA + kABytes, idesc, kb == 0);
@@ -666,11 +696,15 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         const uint32_t d0 = tmem_base + b0 * kAccCols, d1 = tmem_base + b1 * kAccCols;
         constexpr int kDefer = 2;
         const int nd = q.num_kb < kDefer ? q.num_kb : kDefer;
+        TCC(c_w0 = clock64();)
         if (!mbar_wait(tempty_bar(b0), ph0 ^ 1u, abort_flag, p.status, 2)) { alive = false; break; }
+        TCC(c_tempty += clock64() - c_w0;)
         tc_fence_after();
         int st_d[kDefer];
         for (int kb = 0; kb < nd; ++kb) {
+          TCC(c_w0 = clock64();)
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
+          TCC(c_full += clock64() - c_w0;)
           tc_fence_after();
           const uint32_t sA = smem_base + stage * kStageBytes;
           issue_kblock(d0, sA, sA + kABytes, idesc, kb == 0);
@@ -678,15 +712,24 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!alive) break;
+        TCC(c_w0 = clock64();)
         if (!mbar_wait(tempty_bar(b1), ph1 ^ 1u, abort_flag, p.status, 6)) { alive = false; break; }
+        TCC(c_tempty += clock64() - c_w0;)
         tc_fence_after();
         for (int kb = 0; kb < nd; ++kb) {
           const uint32_t sA = smem_base + st_d[kb] * kStageBytes;
           issue_kblock(d1, sA, sA + kABytes + G::kBBytes, idesc, kb == 0);
           free_stage(st_d[kb]);
         }
-        for (int kb = nd; kb < q.num_kb; ++kb) {
+        // The last kLead k-blocks feed b0 first and b1 afterwards (from the same stages), so b0
+        // is complete, and its epilogue under way, while b1's last MMAs still run.
+        constexpr int kLead = 2;
+        const int nl = q.num_kb - nd >= kLead ? kLead : 0;
+        for (int kb = nd; kb < q.num_kb - nl; ++kb) {
+          TCC(c_w0 = clock64();)
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
+          TCC(c_full += clock64() - c_w0;
+              if (q.num_kb >= 32) { if (kb == 8) c_mid0 = clock64(); if (kb == 24) { c_mid += clock64() - c_mid0; c_midn += 32; } })
           tc_fence_after();
           const uint32_t sA = smem_base + stage * kStageBytes;
           issue_kblock(d0, sA, sA + kABytes, idesc, false);
@@ -695,23 +738,45 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!alive) break;
+        int st_l[kLead];
+        for (int j = 0; j < nl; ++j) {
+          TCC(c_w0 = clock64();)
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 3)) { alive = false; break; }
+          TCC(c_full += clock64() - c_w0;)
+          tc_fence_after();
+          const uint32_t sA = smem_base + stage * kStageBytes;
+          issue_kblock(d0, sA, sA + kABytes, idesc, false);
+          st_l[j] = stage;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!alive) break;
         acc_done(b0);
+        for (int j = 0; j < nl; ++j) {
+          const uint32_t sA = smem_base + st_l[j] * kStageBytes;
+          issue_kblock(d1, sA, sA + kABytes + G::kBBytes, idesc, false);
+          free_stage(st_l[j]);
+        }
         acc_done(b1);
         // two buffers used: the buffer index is unchanged, the phase of both advances
         if (b0 == 0) acc_phase ^= 1u; else { buf = 1; acc_phase ^= 1u; }
       }
+      TCC(atomicAdd(&cnt[0], 1ull); atomicAdd(&cnt[1], (unsigned long long)(clock64() - c_start));
+          atomicAdd(&cnt[2], (unsigned long long)c_full); atomicAdd(&cnt[3], (unsigned long long)c_tempty);
+          atomicAdd(&cnt[8], (unsigned long long)c_tiles); atomicAdd(&cnt[9], (unsigned long long)c_kb);
+          atomicAdd(&cnt[10], (unsigned long long)c_mid); atomicAdd(&cnt[11], (unsigned long long)c_midn);)
     }
   } else {
     // ================= epilogue warps =================
     const int quad = warp & 3;                 // tensor-memory lanes [32*quad, 32*quad + 32)
     const int row_in_tile = BM * (int)cta_rank + quad * 32 + lane;   // row of the (pair's) tile
-    const uint32_t stg = stg0 + (uint32_t)quad * (kStgBufs * kStgBufBytes);   // this warp's staging ring
+    const uint32_t stg = stg0 + (uint32_t)quad * (kSlots * kStgBufBytes);   // this warp's staging ring
     uint32_t n_store = 0;                      // stores issued so far: ring slot = n_store % 4
     uint32_t n_chunk = 0;                      // SwiGLU backward: input chunks consumed so far
     const uint64_t pol_stream = l2_policy_evict_first();
     int buf = 0;
     uint32_t acc_phase = 0;
     bool alive = true;
+    TCC(long long c_tfull = 0; const long long c_start = clock64();)
     Tile t_pf = prefetch_tile(it0);
     for (int it = it0; it < it_end && alive; it += it_step) {
       const int ti = zigzag ? tile_of(it) : it;
@@ -756,7 +821,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         }
       }
       // the whole warp must agree before the warp-collective tensor-memory loads
+      TCC(const long long c_w0 = clock64();)
       const bool got = mbar_wait(tfull_bar(buf), acc_phase, abort_flag, p.status, 4);
+      TCC(c_tfull += clock64() - c_w0;)
       if (!__all_sync(0xffffffffu, got)) { alive = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kAccCols;
@@ -767,20 +834,46 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       if ((RT::EPI == EPI_BF16 || RT::EPI == EPI_F32) && !(WIDE && q.wide) && it + it_step < it_end &&
           (zigzag ? tile_of(it + 1) : it + it_step) >= 0)
         next_kb = tile_geom<ROLE>(p, t_pf, s_seg).num_kb;
+      // The accumulator is handed back to the MMA issuer as soon as its last column has left
+      // tensor memory, before the arithmetic, the staging and the stores of that data: with
+      // double-width entries the next entry's MMAs wait for exactly this.
+      bool released = false;
+      auto release_acc = [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (CG == 2) mbar_arrive_cluster(mapa_rank(tempty_bar(buf), 0)); else mbar_arrive(tempty_bar(buf));
+        }
+        released = true;
+      };
+      // Staging ring of this warp: kSlots boxes of 4 KiB used in turn; store #n leaves from box
+      // n % kSlots.  Before a box is written again the store that last read it (kSlots stores
+      // back) must be done reading: with i stores of the current batch not yet issued, at most
+      // kSlots - 1 - i of the store groups committed so far may still be pending.
+      auto ring_slot = [&](int i) { return stg + ((n_store + (uint32_t)i) % kSlots) * kStgBufBytes; };
+      auto ring_wait = [&](int i) {
+        const int allowed = kSlots - 1 - i;
+        if (lane == 0) {
+          if (allowed <= 0) bulk_wait_read<0>();
+          else if (allowed == 1) bulk_wait_read<1>();
+          else if (allowed == 2) bulk_wait_read<2>();
+          else bulk_wait_read<3>();
+        }
+        __syncwarp();
+      };
       if (RT::EPI == EPI_SWIGLU_FWD) {
         const int half = q.bn >> 1;
         for (int c = 0; rows_ok && c < half && q.n0 + c < q.W; c += 64) {
-          if (lane == 0) bulk_wait_read<1>();          // three of the four ring slots are free
-          __syncwarp();
-          const uint32_t bA = stg + ((n_store & 3u) << 12), bU = stg + (((n_store + 1) & 3u) << 12),
-                         bH = stg + (((n_store + 2) & 3u) << 12);
-          n_store += 3;
+          const bool last_chunk = !(c + 64 < half && q.n0 + c + 64 < q.W);
+          ring_wait(2);                                // three boxes of the ring are free
+          const uint32_t bA = ring_slot(0), bU = ring_slot(1), bH = ring_slot(2);
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             uint32_t ra[32], ru[32];
             tmem_ld32(taddr + c + 32 * hh, ra);
             tmem_ld32(taddr + half + c + 32 * hh, ru);
             tmem_ld_wait();
+            if (last_chunk && hh == 1) release_acc();
             uint32_t pa[4][4], pu[4][4], ph[4][4];       // arithmetic first, then the stores
 #pragma unroll
             for (int j4 = 0; j4 < 4; ++j4) {
@@ -807,34 +900,49 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             tma_store_2d(&p.mapO[1][q.g], bU, q.n0 + c, row0, pol_stream); bulk_commit();
             tma_store_2d(&p.mapO[2][q.g], bH, q.n0 + c, row0, pol_stream); bulk_commit();
           }
+          n_store += 3;
         }
       } else if (RT::EPI == EPI_BF16) {
-        for (int c = 0; rows_ok && c < q.bn && q.n0 + c < (int)d; c += 64) {
-          pace(t_epi, c, q.bn, next_kb);
-          if (lane == 0) bulk_wait_read<3>();
-          __syncwarp();
-          const uint32_t bO = stg + ((n_store & 3u) << 12);
-          n_store += 1;
-          uint32_t r0[32], r1[32];
-          tmem_ld32(taddr + c, r0);
-          tmem_ld32(taddr + c + 32, r1);
-          tmem_ld_wait();
+        int nch = 0;                                   // 64-column chunks of this piece (at most 4)
+        if (rows_ok) { const int left = (int)d - q.n0; nch = ((left < q.bn ? left : q.bn) + 63) >> 6; }
+        // Chunks go out in batches of one fence: single chunks while the output is paced against
+        // the next tile's MMAs, else as many as the ring holds.
+        const int batch = next_kb ? 1 : kSlots;
+        for (int c0 = 0; c0 < nch; c0 += batch) {
+          const int nb = nch - c0 < batch ? nch - c0 : batch;
+          for (int i = 0; i < nb; ++i) {
+            const int ci = c0 + i;
+            pace(t_epi, ci * 64, q.bn, next_kb);
+            ring_wait(i);
+            const uint32_t bO = ring_slot(i);
+            uint32_t r0[32], r1[32];
+            tmem_ld32(taddr + ci * 64, r0);
+            tmem_ld32(taddr + ci * 64 + 32, r1);
+            tmem_ld_wait();
+            if (ci + 1 == nch) release_acc();
 #pragma unroll
-          for (int j4 = 0; j4 < 4; ++j4) {
-            st_shared_v4(stg_addr(bO, lane, j4),
-                         pack2(__uint_as_float(r0[j4 * 8 + 0]), __uint_as_float(r0[j4 * 8 + 1])),
-                         pack2(__uint_as_float(r0[j4 * 8 + 2]), __uint_as_float(r0[j4 * 8 + 3])),
-                         pack2(__uint_as_float(r0[j4 * 8 + 4]), __uint_as_float(r0[j4 * 8 + 5])),
-                         pack2(__uint_as_float(r0[j4 * 8 + 6]), __uint_as_float(r0[j4 * 8 + 7])));
-            st_shared_v4(stg_addr(bO, lane, 4 + j4),
-                         pack2(__uint_as_float(r1[j4 * 8 + 0]), __uint_as_float(r1[j4 * 8 + 1])),
-                         pack2(__uint_as_float(r1[j4 * 8 + 2]), __uint_as_float(r1[j4 * 8 + 3])),
-                         pack2(__uint_as_float(r1[j4 * 8 + 4]), __uint_as_float(r1[j4 * 8 + 5])),
-                         pack2(__uint_as_float(r1[j4 * 8 + 6]), __uint_as_float(r1[j4 * 8 + 7])));
+            for (int j4 = 0; j4 < 4; ++j4) {
+              st_shared_v4(stg_addr(bO, lane, j4),
+                           pack2(__uint_as_float(r0[j4 * 8 + 0]), __uint_as_float(r0[j4 * 8 + 1])),
+                           pack2(__uint_as_float(r0[j4 * 8 + 2]), __uint_as_float(r0[j4 * 8 + 3])),
+                           pack2(__uint_as_float(r0[j4 * 8 + 4]), __uint_as_float(r0[j4 * 8 + 5])),
+                           pack2(__uint_as_float(r0[j4 * 8 + 6]), __uint_as_float(r0[j4 * 8 + 7])));
+              st_shared_v4(stg_addr(bO, lane, 4 + j4),
+                           pack2(__uint_as_float(r1[j4 * 8 + 0]), __uint_as_float(r1[j4 * 8 + 1])),
+                           pack2(__uint_as_float(r1[j4 * 8 + 2]), __uint_as_float(r1[j4 * 8 + 3])),
+                           pack2(__uint_as_float(r1[j4 * 8 + 4]), __uint_as_float(r1[j4 * 8 + 5])),
+                           pack2(__uint_as_float(r1[j4 * 8 + 6]), __uint_as_float(r1[j4 * 8 + 7])));
+            }
           }
           fence_async_smem();
           __syncwarp();
-          if (lane == 0) { tma_store_2d(&p.mapO[0][0], bO, q.n0 + c, row0, pol_stream); bulk_commit(); }
+          if (lane == 0) {
+            for (int i = 0; i < nb; ++i) {
+              tma_store_2d(&p.mapO[0][0], ring_slot(i), q.n0 + (c0 + i) * 64, row0, pol_stream);
+              bulk_commit();
+            }
+          }
+          n_store += nb;
         }
       } else if (RT::EPI == EPI_SWIGLU_BWD) {
         // per 64-column chunk: A and U arrive by TMA in one of two buffer pairs, dA and dU are
@@ -866,7 +974,10 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               va[j4] = ld_shared_v4(stg_addr(bA, lane, hh * 4 + j4));
               vu[j4] = ld_shared_v4(stg_addr(bU, lane, hh * 4 + j4));
             }
-            if (hh == 0) tmem_ld_wait();
+            if (hh == 0) {
+              tmem_ld_wait();
+              if (ci + 1 == nch_in) release_acc();
+            }
             uint32_t oa[4][4], ou[4][4];
 #pragma unroll
             for (int j4 = 0; j4 < 4; ++j4) {
@@ -912,25 +1023,68 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         // weight gradients: FP32 boxes of 32 rows x 32 columns into [expert, rows, columns]
         const int Mext = ROLE == ROLE_WGRAD_DOWN ? (int)d : 2 * q.W;
         const int Next = ROLE == ROLE_WGRAD_DOWN ? q.W : (int)d;
-        for (int c = 0; row0 < Mext && c < q.bn && q.n0 + c < Next; c += 32) {
-          pace(t_epi, c, q.bn, next_kb);
-          if (lane == 0) bulk_wait_read<3>();
-          __syncwarp();
-          const uint32_t bO = stg + ((n_store & 3u) << 12);
-          n_store += 1;
-          uint32_t r[32];
-          tmem_ld32(taddr + c, r);
-          tmem_ld_wait();
-#pragma unroll
-          for (int j = 0; j < 8; ++j)
-            st_shared_v4(stg_addr(bO, lane, j), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        int nch = 0;                                   // 32-column chunks of this piece (at most 8)
+        if (row0 < Mext) { const int left = Next - q.n0; nch = ((left < q.bn ? left : q.bn) + 31) >> 5; }
+        auto send_batch = [&](int c0, int nb) {         // boxes ring_slot(0..nb-1) hold chunks c0..
           fence_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (p.accumulate) tma_reduce_add_3d(&p.mapO[0][q.g], bO, q.n0 + c, row0, q.i);
-            else tma_store_3d(&p.mapO[0][q.g], bO, q.n0 + c, row0, q.i, pol_stream);
-            bulk_commit();
+            for (int i = 0; i < nb; ++i) {
+              const int col = q.n0 + (c0 + i) * 32;
+              if (p.accumulate) tma_reduce_add_3d(&p.mapO[0][q.g], ring_slot(i), col, row0, q.i);
+              else tma_store_3d(&p.mapO[0][q.g], ring_slot(i), col, row0, q.i, pol_stream);
+              bulk_commit();
+            }
           }
+          n_store += nb;
+        };
+        auto stage_chunk = [&](uint32_t bO, const uint32_t (&r)[32]) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            st_shared_v4(stg_addr(bO, lane, j), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+        };
+        if (!next_kb && kSlots == 4 && nch > 4) {
+          // Nothing to pace against (double-width entries): four chunks go into the ring, the
+          // other (up to) four wait in registers, and the accumulator is released at once.
+          for (int i = 0; i < 4; ++i) {
+            ring_wait(i);
+            uint32_t r[32];
+            tmem_ld32(taddr + i * 32, r);
+            tmem_ld_wait();
+            stage_chunk(ring_slot(i), r);
+          }
+          uint32_t rr[4][32];
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            if (4 + j < nch) tmem_ld32(taddr + (4 + j) * 32, rr[j]);
+          tmem_ld_wait();
+          release_acc();
+          send_batch(0, 4);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (4 + j < nch) {
+              ring_wait(j);
+              stage_chunk(ring_slot(j), rr[j]);
+            }
+          }
+          send_batch(4, nch - 4);
+          nch = 0;                                       // done
+        }
+        const int batch = next_kb ? 1 : kSlots;
+        for (int c0 = 0; c0 < nch; c0 += batch) {
+          const int nb = nch - c0 < batch ? nch - c0 : batch;
+          for (int i = 0; i < nb; ++i) {
+            const int ci = c0 + i;
+            pace(t_epi, ci * 32, q.bn, next_kb);
+            ring_wait(i);
+            const uint32_t bO = ring_slot(i);
+            uint32_t r[32];
+            tmem_ld32(taddr + ci * 32, r);
+            tmem_ld_wait();
+            if (ci + 1 == nch) release_acc();
+            stage_chunk(bO, r);
+          }
+          send_batch(c0, nb);
         }
       } else if (RT::EPI == EPI_LOGITS) {
         // logits[t, n] = acc + bias[n]; NL is arbitrary, so stores are scalar and masked.  Under
@@ -1002,19 +1156,20 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           }
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if (CG == 2) mbar_arrive_cluster(mapa_rank(tempty_bar(buf), 0)); else mbar_arrive(tempty_bar(buf));
-      }
+      if (!released) release_acc();
       if (++buf == 2) { buf = 0; acc_phase ^= 1u; }
       }   // pieces
     }
     if (lane == 0) bulk_wait_all();            // staged stores have left before the CTA retires
+    TCC(if (warp == 2 && lane == 0) {
+          atomicAdd(&cnt[5], (unsigned long long)c_tfull);
+          atomicAdd(&cnt[6], (unsigned long long)(clock64() - c_start));
+        })
   }
 
   // ---- teardown ----
   __syncthreads();
+  TCC(if (threadIdx.x == 0) atomicAdd(&cnt[7], (unsigned long long)(global_ns() - cnt_t0));)
   if (*abort_flag) __nanosleep(200000);    // let copies in flight land before the CTA retires
   if (CG == 2) cluster_sync_all();         // the peer may still signal this CTA's barriers until here
   tc_fence_after();
@@ -1161,6 +1316,12 @@ int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
     cfg.gridDim = dim3(want * CG);
   }
   cfg.numAttrs = dependent_launch() ? 2 : 1;
+#ifdef MOHGE_TC_COUNTERS
+  if (const char* e = getenv("MOHGE_TC_GRID")) {        // measurements with fewer CTAs than SMs
+    const int g = atoi(e) / CG * CG;
+    if (g >= CG && g < (int)cfg.gridDim.x) cfg.gridDim = dim3(g);
+  }
+#endif
   MOHGE_CUDA(cudaLaunchKernelEx(&cfg, tc_grouped_kernel<ROLE, CG, WIDE>, p));
   MOHGE_LAUNCH_CHECK("tc_grouped_kernel");
   return MOHGE_OK;
@@ -1516,3 +1677,23 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
 }
 
 }  // namespace mohge
+
+#ifdef MOHGE_TC_COUNTERS
+// Copies the counter table [9 roles][160 CTAs][12 slots] (uint64) to `host_out` after a device
+// synchronisation; `reset` != 0 clears it afterwards.  Slots: 0 launches, 1 issuer loop clocks,
+// 2 issuer waiting for operands, 3 issuer waiting for an accumulator, 4 producer waiting for a
+// stage, 5 epilogue warp waiting for an accumulator, 6 epilogue loop clocks, 7 CTA lifetime ns,
+// 8 tiles, 9 k-blocks (a double-width entry counts twice), 10 clocks between the 8th and the 24th
+// k-block of tiles with 32 k-blocks or more, 11 the k-blocks those clocks cover.
+extern "C" int32_t mohge_debug_tc_counters(unsigned long long* host_out, int32_t reset) {
+  using namespace mohge;
+  MOHGE_CUDA(cudaDeviceSynchronize());
+  MOHGE_CUDA(cudaMemcpyFromSymbol(host_out, g_tc_counters, sizeof(g_tc_counters)));
+  if (reset) {
+    void* p = nullptr;
+    MOHGE_CUDA(cudaGetSymbolAddress(&p, g_tc_counters));
+    MOHGE_CUDA(cudaMemset(p, 0, sizeof(g_tc_counters)));
+  }
+  return MOHGE_OK;
+}
+#endif
