@@ -30,11 +30,13 @@ import torch  # noqa: E402
 
 from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs  # noqa: E402
 
-# DRAM bytes (read + written) of the six grouped-GEMM launches of one step, from the 1-pass ncu
-# capture summarised in profiles/launch_list_layer_step_cfg5.md (the L2 hit rate of these launches
-# differs between the GPUs of the pool: captures of the same build range over tens of GB); workloads without a
-# capture of the current kernels report null.
-NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 74.3e9}
+# DRAM bytes (read + written) of the six grouped-GEMM launches of one step, from a counter capture
+# of the kernels as they stand now.  The large workload is too big to capture with counters; its
+# figure is the capture of "cfg5_slice" (one eighth of the experts, the same tokens per expert,
+# widths and tile forms) times eight: every expert's tiles are independent problems, so the traffic
+# grows with the number of experts.  None: no capture of the current kernels.
+NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": None}
+NCU_DRAM_TRAFFIC_SOURCE = {}
 
 METRIC = "MoHGE layer fwd+bwd tokens/s"
 METRIC_FWD = "MoHGE layer fwd tokens/s"
@@ -102,62 +104,73 @@ class ClockSampler:
         return out
 
 
-def oracle_sample_run(wl: Workload, sample_tokens: int, steps: int, warmup: int, inp_cpu=None):
-    """Times the oracle (as it stands) on `sample_tokens` tokens of the workload; tokens/s."""
+ORACLE_SAMPLE_TOKENS = 256      # the one sample size of both oracle arms (cpu_baseline and --impl reference)
+ORACLE_BUDGET_S = 120.0         # timed oracle steps stop once this much time has been spent
+
+
+def oracle_sample_run(wl: Workload, sample_tokens: int, steps: int, warmup: int, inp_cpu=None,
+                      budget_s: float = ORACLE_BUDGET_S):
+    """Times the oracle (as it stands) on `sample_tokens` tokens of the workload.  Returns
+    (tokens/s, seconds per step, steps run, seconds to convert every expert's weights to fp64).
+    The oracle's step time is dominated by that conversion, which it repeats for every expert a
+    step touches, so tokens/s is not linear in the sample: both oracle arms use the same sample."""
     import numpy as np
-    sys.path.insert(0, os.path.join(ROOT, "tests"))
     import oracle as O
-    from _util import oracle_cfg, to_np64
     from paper_2604_23108_b200.inputs import make_inputs
     if inp_cpu is None:
         inp_cpu = make_inputs(wl, T=sample_tokens)
-    ocfg = oracle_cfg(wl)
+    to_np64 = lambda t: t.detach().to("cpu").to(torch.float64).numpy()
+    ocfg = O.OracleConfig(d_model=wl.d_model, n_groups=wl.n_groups, experts_per_group=wl.experts_per_group,
+                          k_groups=wl.k_groups, k_experts=wl.k_experts, group_width=list(wl.group_width))
     x, w_r, dy = to_np64(inp_cpu["x"][:sample_tokens]), to_np64(inp_cpu["w_router"]), to_np64(inp_cpu["dy"][:sample_tokens])
     bias = None if inp_cpu.get("logit_bias") is None else to_np64(inp_cpu["logit_bias"])
     w13, w2 = inp_cpu["w13"], inp_cpu["w2"]       # converted to fp64 expert by expert inside the oracle
     w13n = [w.to(torch.float32).numpy() for w in w13]
     w2n = [w.to(torch.float32).numpy() for w in w2]
-    times = []
+    t0 = time.perf_counter()
+    for w in w13n + w2n:
+        w.astype(np.float64)
+    t_conv = time.perf_counter() - t0
+    times, spent = [], 0.0
     for it in range(warmup + steps):
         t0 = time.perf_counter()
         fwd = O.layer_forward(ocfg, x, w_r, w13n, w2n, logit_bias=bias, mode="spec")
         O.layer_backward(fwd, w13n, w2n, dy, with_aux=True)
         t1 = time.perf_counter()
+        spent += t1 - t0
         if it >= warmup:
             times.append(t1 - t0)
+            if spent > budget_s:
+                break
     per = sum(times) / len(times)
-    return sample_tokens / per, per
+    return sample_tokens / per, per, len(times), t_conv
+
+
+def oracle_baseline_dict(val, per, n, t_conv, sample, cores):
+    return {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "steps_run": n,
+            "sample": "oracle fwd+bwd on the first %d tokens of the workload, all experts' weights "
+                      "(%.1f s per step, of which about %.1f s convert the weights of the experts hit to "
+                      "fp64)" % (sample, per, min(per, 2.0 * t_conv))}
 
 
 def run_reference(args, wl: Workload, rank: int):
     if rank != 0:
         return
-    cores = torch.get_num_threads()
-    # The oracle's time per step is set by how many distinct experts the sample hits (it converts
-    # each one's weights to fp64).  A two-token probe gives the cost per expert; the sample is then
-    # the largest power of two of tokens (at most --ref-sample) for which steps + warm-up fit in
-    # about 150 s.
     from paper_2604_23108_b200.inputs import make_inputs
-    inp_cpu = make_inputs(wl, T=min(wl.T, args.ref_sample))
-    Ne, Ke = wl.n_experts, wl.k_experts
-    hits = lambda n: Ne * (1.0 - (1.0 - min(1.0, Ke / Ne)) ** n)
-    probe = min(2, wl.T)
-    _, t_probe = oracle_sample_run(wl, probe, 1, 0, inp_cpu=inp_cpu)
-    per_expert = t_probe / max(1.0, hits(probe))
-    n_steps = max(1, args.steps) + min(args.warmup, 1)
-    sample = min(wl.T, args.ref_sample)
-    while sample > 1 and n_steps * per_expert * hits(sample) > 150.0:
-        sample //= 2
-    val, per = oracle_sample_run(wl, sample, max(1, args.steps), min(args.warmup, 1), inp_cpu=inp_cpu)
+    cores = torch.get_num_threads()
+    sample = min(wl.T, ORACLE_SAMPLE_TOKENS)
+    inp_cpu = make_inputs(wl, T=sample)
+    # the same sample as the cpu_baseline leg of the default line; as many of the requested steps
+    # as fit into the time budget (one warm-up step at most)
+    val, per, n, t_conv = oracle_sample_run(wl, sample, max(1, args.steps), min(args.warmup, 1), inp_cpu=inp_cpu)
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
         "config": {"workload": wl.name, "T": wl.T, "d_model": wl.d_model,
-                   "sample": "first %d tokens, all experts" % sample},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
-                         "sample": "oracle fwd+bwd on the first %d tokens of the workload" % sample},
+                   "sample": "first %d tokens, all experts" % sample, "steps_run": n},
+        "cpu_baseline": oracle_baseline_dict(val, per, n, t_conv, sample, cores),
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
@@ -187,6 +200,162 @@ def flops_per_step(wl: Workload, counts, shared_width: int = 0) -> float:
     return 18.0 * wl.d_model * tot
 
 
+def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=False):
+    """One pass of the whole hot path through the C ABI.  Returns (step, gemm_marks): with
+    mark=True a step records CUDA events around mohge_expert_fwd and mohge_expert_bwd_dgate."""
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    gemm_marks = []
+
+    def step(mark=False, y=None, dx=None, after_fwd=None, before_bwd=None):
+        y = buf.y if y is None else y
+        dx = buf.dx if dx is None else dx
+        B.mohge_route(gcfg, T, inp["x"], inp["w_router"], inp["logit_bias"], None, buf.logits,
+                      buf.group_idx, buf.expert_idx, buf.gate_w, buf.gs, buf.esp, buf.ws)
+        B.mohge_aux_stats(gcfg, T, buf.gs, buf.esp, buf.group_idx, buf.expert_idx, buf.group_count,
+                          buf.group_psum, buf.cnt_routed, buf.cnt_lit, buf.expert_psum, buf.loss, buf.ws)
+        B.mohge_dispatch(gcfg, T, inp["x"], buf.expert_idx, buf.counts, buf.offsets, buf.aligned,
+                         buf.row_of, buf.prow_of, buf.src_of, buf.x_perm, buf.ws)
+        if mark:
+            e0, e1, e2, e3 = ev(), ev(), ev(), ev()
+            e0.record()
+        B.mohge_expert_fwd(gcfg, T, buf.x_perm, buf.counts, buf.aligned, inp["w13"], inp["w2"],
+                           buf.au, buf.h, buf.y_perm, buf.ws)
+        if shared is not None:
+            B.mohge_shared_fwd(gcfg, T, shared_width, inp["x"], shared[0], shared[1], buf.au_sh,
+                               buf.h_sh, buf.y_sh, buf.ws)
+        if mark:
+            e1.record()
+        B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, y,
+                        y_add=buf.y_sh if shared is not None else None)
+        if after_fwd is not None:
+            after_fwd()                     # y is final here (the end-to-end arm starts its download)
+        if forward_only:
+            if mark:
+                gemm_marks.append((e0, e1, e1, e1))
+            return
+        if before_bwd is not None:
+            before_bwd()                    # dy is first read below (the end-to-end arm waits for its upload)
+        # the gate gradient comes out of the experts' backward, so combine_bwd reads no y_perm
+        B.mohge_combine_bwd(gcfg, T, inp["dy"], None, buf.prow_of, buf.gate_w, buf.counts,
+                            buf.aligned, buf.dy_perm, None)
+        if mark:
+            e2.record()
+        B.mohge_expert_bwd_dgate(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts,
+                                 buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13,
+                                 buf.dw2, 0, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate,
+                                 buf.ws)
+        if shared is not None:
+            B.mohge_shared_bwd(gcfg, T, shared_width, inp["dy"], inp["x"], buf.au_sh, buf.h_sh,
+                               shared[0], shared[1], buf.dau_sh, buf.dx_sh, buf.dw13_sh, buf.dw2_sh,
+                               0, buf.ws)
+        if mark:
+            e3.record()
+            gemm_marks.append((e0, e1, e2, e3))
+        B.mohge_dispatch_bwd(gcfg, T, buf.dx_perm, buf.prow_of, dx,
+                             dx_add=buf.dx_sh if shared is not None else None)
+        cnt_e = buf.cnt_lit if gcfg.fe_mode == 0 else buf.cnt_routed
+        B.mohge_route_bwd(gcfg, T, inp["x"], inp["w_router"], buf.dgate, buf.gs, buf.esp,
+                          buf.group_idx, buf.expert_idx, buf.group_count, cnt_e, buf.dlogits,
+                          dx, buf.dw_router, buf.ws)
+
+    return step, gemm_marks
+
+
+def hbm_step_rooflines(B, gcfg, wl: Workload, inp, buf, hbm_peak_gbs: float, reps: int = 10):
+    """CUDA-event time of every HBM-bound entry point of the step, each called `reps` times back
+    to back on the buffers a full step has left behind, against its algorithmic bytes
+    (s = bytes per element, R = T K_e routed rows, NL = N_g + N_e router outputs):
+      route         x and the router weight read once, logits written and read, scores, indices
+                    and gates written: T d s + NL d s + 3 T NL 4 + T (8 K_e + 4 K_g)
+      aux_stats     saved scores and indices read: T NL 4 + T (K_e + K_g) 4
+      dispatch      (T + R) d s + 16 R (index arrays)
+      combine       (R + T) d s          combine_bwd (scaled rows)  (T + R) d s
+      dispatch_bwd  (R + T) d s          route_bwd   x read, dx read and written: 3 T d s + 2 T NL 4
+    Small workloads fit in L2, where the figure exceeds the HBM rate; that is said in `l2`."""
+    T, d, Ke, Kg, NL = wl.T, wl.d_model, wl.k_experts, wl.k_groups, wl.n_logits
+    s_ = 2 if wl.dtype == "bf16" else 4
+    R = T * Ke
+    cnt_e = buf.cnt_lit if gcfg.fe_mode == 0 else buf.cnt_routed
+    calls = {
+        "route": (lambda: B.mohge_route(gcfg, T, inp["x"], inp["w_router"], inp["logit_bias"], None, buf.logits,
+                                        buf.group_idx, buf.expert_idx, buf.gate_w, buf.gs, buf.esp, buf.ws),
+                  T * d * s_ + NL * d * s_ + 3 * T * NL * 4 + T * (8 * Ke + 4 * Kg)),
+        "aux_stats": (lambda: B.mohge_aux_stats(gcfg, T, buf.gs, buf.esp, buf.group_idx, buf.expert_idx,
+                                                buf.group_count, buf.group_psum, buf.cnt_routed, buf.cnt_lit,
+                                                buf.expert_psum, buf.loss, buf.ws),
+                      T * NL * 4 + T * (Ke + Kg) * 4),
+        "dispatch": (lambda: B.mohge_dispatch(gcfg, T, inp["x"], buf.expert_idx, buf.counts, buf.offsets,
+                                              buf.aligned, buf.row_of, buf.prow_of, buf.src_of, buf.x_perm, buf.ws),
+                     (T + R) * d * s_ + 16 * R),
+        "combine": (lambda: B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, buf.y),
+                    (R + T) * d * s_),
+        "combine_bwd": (lambda: B.mohge_combine_bwd(gcfg, T, inp["dy"], None, buf.prow_of, buf.gate_w, buf.counts,
+                                                    buf.aligned, buf.dy_perm, None),
+                        (T + R) * d * s_),
+        "dispatch_bwd": (lambda: B.mohge_dispatch_bwd(gcfg, T, buf.dx_perm, buf.prow_of, buf.dx),
+                         (R + T) * d * s_),
+        "route_bwd": (lambda: B.mohge_route_bwd(gcfg, T, inp["x"], inp["w_router"], buf.dgate, buf.gs, buf.esp,
+                                                buf.group_idx, buf.expert_idx, buf.group_count, cnt_e,
+                                                buf.dlogits, buf.dx, buf.dw_router, buf.ws),
+                      3 * T * d * s_ + 2 * T * NL * 4),
+    }
+    out = []
+    for name, (fn, nbytes) in calls.items():
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out.append({"step": name, "bound": "hbm", "bytes": nbytes, "ms": ms, "achieved": gbs,
+                    "peak": hbm_peak_gbs, "unit": "GB/s", "frac": gbs / hbm_peak_gbs})
+    return out
+
+
+def count_ratio(counts):
+    """Largest over smallest per-expert token count of the batch (None when an expert is empty)."""
+    lo = min(counts)
+    return None if lo == 0 else max(counts) / lo
+
+
+def quick_workload_line(B, name: str, dev, pk, steps: int = 20, warmup: int = 3):
+    """A short measurement of another benchmark workload for the default line's
+    `other_workloads` list: tokens/s of the step and the rate of its grouped GEMMs."""
+    wl = WORKLOADS[name]
+    gcfg = B.Config(d_model=wl.d_model, n_groups=wl.n_groups, experts_per_group=wl.experts_per_group,
+                    k_groups=wl.k_groups, k_experts=wl.k_experts, group_width=list(wl.group_width),
+                    dtype=wl.dtype, row_align=128 if wl.dtype == "bf16" else 1)
+    inp = make_device_inputs(wl, dev)
+    buf = B.LayerBuffers(gcfg, wl.T, device=dev)
+    step, marks = make_step(B, gcfg, wl.T, inp, buf)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(steps):
+        step(mark=True)
+    e1.record()
+    host_ms = (time.perf_counter() - t0) * 1e3 / steps
+    torch.cuda.synchronize()
+    status = B.mohge_get_device_status(buf.ws)
+    ms = e0.elapsed_time(e1) / steps
+    gemm_ms = sum(a.elapsed_time(b) + c.elapsed_time(d_) for a, b, c, d_ in marks) / len(marks)
+    counts = buf.counts.cpu().tolist()
+    tf = flops_per_step(wl, counts) / (gemm_ms * 1e-3) / 1e12
+    bf16 = wl.dtype == "bf16"
+    return {"workload": wl.name, "dtype": wl.dtype, "T": wl.T, "steps": steps, "value": wl.T / (ms * 1e-3),
+            "unit": UNIT, "ms_per_step": ms, "host_enqueue_ms_per_step": host_ms,
+            "gemm_ms_per_step": gemm_ms, "gemm_tflops": tf,
+            "gemm_frac_of_sustained_bf16": tf / pk["tf_sustained"] if bf16 else None,
+            "count_ratio": count_ratio(counts), "device_status": status}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -194,9 +363,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-sample", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip what the default line adds outside the timed region: the per-step "
+                         "HBM rooflines and the short runs of the other benchmark workloads")
     ap.add_argument("--forward-only", action="store_true",
                     help="time the forward pass alone (inference-shaped workloads); the roofline "
                          "object then describes mohge_expert_fwd against HBM bandwidth")
@@ -241,59 +412,7 @@ def main():
         shared = make_shared_weights(wl, args.shared_width, device=dev, seed=replica_seed(wl, rank))
     T = wl.T
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    gemm_marks = []
-
-    def step(mark=False, y=None, dx=None, after_fwd=None, before_bwd=None):
-        y = buf.y if y is None else y
-        dx = buf.dx if dx is None else dx
-        B.mohge_route(gcfg, T, inp["x"], inp["w_router"], inp["logit_bias"], None, buf.logits,
-                      buf.group_idx, buf.expert_idx, buf.gate_w, buf.gs, buf.esp, buf.ws)
-        B.mohge_aux_stats(gcfg, T, buf.gs, buf.esp, buf.group_idx, buf.expert_idx, buf.group_count,
-                          buf.group_psum, buf.cnt_routed, buf.cnt_lit, buf.expert_psum, buf.loss, buf.ws)
-        B.mohge_dispatch(gcfg, T, inp["x"], buf.expert_idx, buf.counts, buf.offsets, buf.aligned,
-                         buf.row_of, buf.prow_of, buf.src_of, buf.x_perm, buf.ws)
-        if mark:
-            e0, e1, e2, e3 = ev(), ev(), ev(), ev()
-            e0.record()
-        B.mohge_expert_fwd(gcfg, T, buf.x_perm, buf.counts, buf.aligned, inp["w13"], inp["w2"],
-                           buf.au, buf.h, buf.y_perm, buf.ws)
-        if shared is not None:
-            B.mohge_shared_fwd(gcfg, T, args.shared_width, inp["x"], shared[0], shared[1], buf.au_sh,
-                               buf.h_sh, buf.y_sh, buf.ws)
-        if mark:
-            e1.record()
-        B.mohge_combine(gcfg, T, buf.y_perm, buf.prow_of, buf.gate_w, y,
-                        y_add=buf.y_sh if shared is not None else None)
-        if after_fwd is not None:
-            after_fwd()                     # y is final here (the end-to-end arm starts its download)
-        if args.forward_only:
-            if mark:
-                gemm_marks.append((e0, e1, e1, e1))
-            return
-        if before_bwd is not None:
-            before_bwd()                    # dy is first read below (the end-to-end arm waits for its upload)
-        # the gate gradient comes out of the experts' backward, so combine_bwd reads no y_perm
-        B.mohge_combine_bwd(gcfg, T, inp["dy"], None, buf.prow_of, buf.gate_w, buf.counts,
-                            buf.aligned, buf.dy_perm, None)
-        if mark:
-            e2.record()
-        B.mohge_expert_bwd_dgate(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts,
-                                 buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13,
-                                 buf.dw2, 0, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate,
-                                 buf.ws)
-        if shared is not None:
-            B.mohge_shared_bwd(gcfg, T, args.shared_width, inp["dy"], inp["x"], buf.au_sh, buf.h_sh,
-                               shared[0], shared[1], buf.dau_sh, buf.dx_sh, buf.dw13_sh, buf.dw2_sh,
-                               0, buf.ws)
-        if mark:
-            e3.record()
-            gemm_marks.append((e0, e1, e2, e3))
-        B.mohge_dispatch_bwd(gcfg, T, buf.dx_perm, buf.prow_of, dx,
-                             dx_add=buf.dx_sh if shared is not None else None)
-        cnt_e = buf.cnt_lit if gcfg.fe_mode == 0 else buf.cnt_routed
-        B.mohge_route_bwd(gcfg, T, inp["x"], inp["w_router"], buf.dgate, buf.gs, buf.esp,
-                          buf.group_idx, buf.expert_idx, buf.group_count, cnt_e, buf.dlogits,
-                          dx, buf.dw_router, buf.ws)
+    step, gemm_marks = make_step(B, gcfg, T, inp, buf, shared, args.shared_width, args.forward_only)
 
     def barrier():
         if dist is not None:
@@ -327,6 +446,7 @@ def main():
     l0 = B.mohge_launch_count()
     barrier()
     t_start, t_end = ev(), ev()
+    host_t0 = time.perf_counter()
     t_start.record()
     for _ in range(args.steps):
         if graph is not None:
@@ -334,6 +454,7 @@ def main():
         else:
             step(mark=True)
     t_end.record()
+    host_enqueue_ms = (time.perf_counter() - host_t0) * 1e3 / args.steps   # host time to enqueue a step
     barrier()
     launches = launches_per_replay * args.steps if graph is not None else B.mohge_launch_count() - l0
     clocks = sampler.stop() if sampler else None
@@ -442,11 +563,20 @@ def main():
         return
 
     pk = _peaks()
+    # ---- outside the timed region: every HBM-bound entry point on its own, then short runs of the
+    # other benchmark workloads (default line only) ----
+    hbm_steps, others = None, None
+    if not args.no_extras and world == 1 and not args.forward_only and not args.shared_width:
+        hbm_steps = hbm_step_rooflines(B, gcfg, wl, inp, buf, pk["hbm"])
+        if args.workload == DEFAULT_WORKLOAD:
+            others = [quick_workload_line(B, n, dev, pk) for n in
+                      ("cfg1_tiny_f32", "cfg2_bf16", "cfg3_bf16_aux", "cfg4_bf16_skew")]
     flops = flops_per_step(wl, counts, args.shared_width)
     achieved = flops / (gemm_ms_step * 1e-3) / 1e12
     roofline = {"bound": "tensor", "achieved": achieved, "peak": pk["tf_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / pk["tf_sustained"], "traffic": NCU_DRAM_TRAFFIC_PER_STEP.get(wl.name),
                 "traffic_unit": "bytes of DRAM traffic per step (six launches)",
+                "traffic_source": NCU_DRAM_TRAFFIC_SOURCE.get(wl.name),
                 "kernel": "tc_grouped_kernel (6 launches per step: fwd1, fwd2, dgrad x2, wgrad x2)",
                 "of": pk["source"], "flops_per_step": flops, "gemm_ms_per_step": gemm_ms_step,
                 "frac_of_nominal_2250": achieved / 2250.0}
@@ -467,14 +597,10 @@ def main():
                         kernel="simt_grouped_kernel (FP32 FMA; correctness configuration)")
     cpu_baseline = None
     if not args.no_cpu_baseline and world == 1:      # timed at N = 1 only: the other GPUs would wait
-        sample = min(wl.T, args.ref_sample)
-        cpu_inp = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in inp.items()
-                   if k not in ("w13", "w2")}
-        cpu_inp["w13"] = [w.cpu() for w in inp["w13"]]
-        cpu_inp["w2"] = [w.cpu() for w in inp["w2"]]
-        val, per = oracle_sample_run(wl, sample, 1, 0, inp_cpu=cpu_inp)
-        cpu_baseline = {"value": val, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-                        "sample": "oracle fwd+bwd on the first %d tokens of the workload (%.1f s)" % (sample, per)}
+        from paper_2604_23108_b200.inputs import make_inputs
+        sample = min(wl.T, ORACLE_SAMPLE_TOKENS)
+        val, per, n, t_conv = oracle_sample_run(wl, sample, 1, 0, inp_cpu=make_inputs(wl, T=sample))
+        cpu_baseline = oracle_baseline_dict(val, per, n, t_conv, sample, torch.get_num_threads())
     line = {
         "metric": METRIC_FWD if args.forward_only else METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
@@ -483,10 +609,13 @@ def main():
                    "experts_per_group": wl.experts_per_group, "group_width": list(wl.group_width),
                    "k_groups": wl.k_groups, "k_experts": wl.k_experts, "shared_width": args.shared_width,
                    "pass": "forward only" if args.forward_only else "forward + backward",
+                   "count_ratio": count_ratio(counts),
                    "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only",
                    "launch": "CUDA graph replay" if args.graph else "stream launches"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "device_status": status,
-        "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "host_enqueue_ms_per_step": host_enqueue_ms,
+        "roofline": roofline, "roofline_hbm_steps": hbm_steps, "cpu_baseline": cpu_baseline,
+        "other_workloads": others,
     }
     print(json.dumps(line), flush=True)
     if dist is not None:

@@ -19,6 +19,9 @@
  *     allocates no caller-visible memory, frees nothing, and never synchronises the device:
  *     work is enqueued on `stream` (a cudaStream_t passed as void*) and the call returns.
  *   - Arguments are validated before anything is launched; an invalid call launches nothing.
+ *   - Several GPUs: every call works on the device that is current on the calling thread; what
+ *     the library remembers about a device (SM count, kernel attributes, cached tensor maps) is
+ *     kept per device ordinal, so one process may drive several GPUs.
  *   - Stream capture: launch shapes depend on the config and T only; everything that depends on
  *     the batch (counts, offsets, tile lists, statistics) stays in device memory.  A sequence of
  *     calls captured into a CUDA graph therefore serves every later batch of the same T held in
@@ -61,10 +64,10 @@ enum mohge_status {
   MOHGE_OK = 0,
   MOHGE_ERR_INVALID_ARG = -1,
   MOHGE_ERR_UNSUPPORTED = -2,
-  MOHGE_ERR_WORKSPACE = -3,
+  MOHGE_ERR_WORKSPACE = -3,      /* mohge_workspace_init: the workspace is too small */
   MOHGE_ERR_CUDA = -4,
-  MOHGE_ERR_TIMEOUT = -5,        /* a device-side bounded wait gave up (status word) */
-  MOHGE_ERR_DEVICE_CHECK = -6    /* a device-side index check failed (status word) */
+  MOHGE_ERR_TIMEOUT = -5,        /* mohge_get_device_status: a device-side bounded wait gave up */
+  MOHGE_ERR_DEVICE_CHECK = -6    /* mohge_get_device_status: a device-side input check failed */
 };
 
 typedef struct mohge_config {
@@ -97,13 +100,37 @@ int64_t mohge_workspace_bytes(const mohge_config* cfg, int64_t T);
  * row_align (an upper bound of aligned_offsets[N_e]). */
 int64_t mohge_perm_rows(const mohge_config* cfg, int64_t T);
 
-/* Clears the device status word.  Call once after allocating the workspace. */
-int32_t mohge_workspace_init(const mohge_config* cfg, int64_t T, void* ws, void* stream);
+/* Clears the device status word.  Call once after allocating the workspace of `ws_bytes` bytes;
+ * returns MOHGE_ERR_WORKSPACE (and touches nothing) when that is less than
+ * mohge_workspace_bytes(cfg, T).  The other entry points take `ws` on trust. */
+int32_t mohge_workspace_init(const mohge_config* cfg, int64_t T, void* ws, int64_t ws_bytes, void* stream);
 
 /* Copies the device status word to *host_out (HOST) and synchronises `stream`; the only
- * device-to-host transfer in the library, off the hot path.  0 = no device-side error;
- * otherwise (code << 24) | detail with code 1 = bounded wait expired, 2 = index check. */
+ * device-to-host transfer in the library, off the hot path.  The word is 0 when nothing was
+ * reported, else (code << 24) | detail, first report wins:
+ *   code 1  a bounded wait in the grouped GEMM kernel expired   -> returns MOHGE_ERR_TIMEOUT
+ *   code 2  an index check failed and the entry was skipped     -> returns MOHGE_ERR_DEVICE_CHECK
+ *   code 3  NaN among the router logits (read as the most negative float, i.e. ranked below
+ *           every number: Eq. 2-5 order real numbers and define nothing for NaN)
+ *                                                               -> returns MOHGE_ERR_DEVICE_CHECK
+ * Returns MOHGE_OK when the word is 0. */
 int32_t mohge_get_device_status(const void* ws, int32_t* host_out, void* stream);
+
+/* Debugging switches (no paper counterpart).  Names: "pdl" (0: launch without programmatic
+ * dependent launch), "tc_cg" (1 | 2: force single CTAs or CTA pairs in the grouped GEMMs),
+ * "tc_wide" (bit mask over the six expert GEMM roles: force double-width entries per role),
+ * "force_simt" (1: run the BF16 GEMMs on the FP32-FMA kernel).  -1 = not set, the library's own
+ * rule decides.  Each switch is read ONCE from its environment variable (MOHGE_PDL, MOHGE_TC_CG,
+ * MOHGE_TC_WIDE, MOHGE_FORCE_SIMT) when a switch is first consulted; later changes of the
+ * environment are not seen, mohge_set_switch is the only way to change a switch afterwards.
+ * mohge_get_switch returns INT32_MIN for an unknown name.  HOST. */
+int32_t mohge_get_switch(const char* name);
+int32_t mohge_set_switch(const char* name, int32_t value);
+
+/* Diagnostics (no paper counterpart): hits and misses of the cache of encoded TMA tensor maps
+ * (keyed by device, GEMM role, operand addresses and shapes) since the process started.  A layer
+ * stepped on the same buffers misses once per GEMM launch site and hits ever after.  HOST. */
+void mohge_map_cache_stats(int64_t* hits, int64_t* misses);
 
 /*
  * Two-level router, Sec. 3.2, Eq. 2-6.

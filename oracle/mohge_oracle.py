@@ -206,10 +206,19 @@ def route_spec(cfg: OracleConfig, logits32):
     S = tree sum of p, r = sigmoid_spec(l_g)/S, key_i = p_i * r, ES'_i = p_i/S.
     Experts of unselected groups get key -1.  Experts: K_e rounds of arg-max
     over the keys.  gate_k = key_k / (left-to-right sum of the K_e keys).
+
+    NaN logits: Eq. 2-5 order real numbers and say nothing about NaN.  Reading:
+    a NaN logit is invalid input that ranks below every number; it is read as
+    the most negative finite float32, ties among such entries go to the lowest
+    index as everywhere else, and the number of NaN entries is returned in
+    "nan_logits" (an implementation reports them through its status word).
     """
     cfg.check()
     N_g, N = cfg.n_groups, cfg.experts_per_group
     logits32 = np.asarray(logits32, dtype=_F)
+    nan_logits = int(np.isnan(logits32).sum())
+    if nan_logits:
+        logits32 = np.where(np.isnan(logits32), -np.finfo(_F).max, logits32).astype(_F)
     T = logits32.shape[0]
     lG = logits32[:, :N_g]
     lE = logits32[:, N_g:].reshape(T, N_g, N)
@@ -218,7 +227,8 @@ def route_spec(cfg: OracleConfig, logits32):
     gsel[np.arange(T)[:, None], group_idx] = True
     GS = sigmoid_spec(lG)
     m = lE.max(axis=2, keepdims=True)
-    p = exp_spec((lE - m).astype(_F))
+    with np.errstate(over="ignore"):                      # -FLT_MAX - m may round to -inf: exp gives 0
+        p = exp_spec((lE - m).astype(_F))
     S = tree_sum_f32(p)                                   # [T, N_g]
     r = (GS / S).astype(_F)
     key = (p * r[:, :, None]).astype(_F)
@@ -230,9 +240,10 @@ def route_spec(cfg: OracleConfig, logits32):
     ssum = ksel[:, 0].copy()
     for k in range(1, cfg.k_experts):
         ssum = (ssum + ksel[:, k]).astype(_F)
-    gate = (ksel / ssum[:, None]).astype(_F)
+    with np.errstate(invalid="ignore"):                   # all keys 0 (chosen groups all NaN): 0/0
+        gate = (ksel / ssum[:, None]).astype(_F)
     return dict(group_idx=group_idx, expert_idx=expert_idx, gate=gate, GS=GS,
-                ESp=ESp, key=key, group_mask=gsel)
+                ESp=ESp, key=key, group_mask=gsel, nan_logits=nan_logits)
 
 
 # --------------------------------------------------------------------------

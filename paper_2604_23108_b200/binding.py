@@ -40,7 +40,10 @@ _SIGS = {
     "mohge_launch_count": (C.c_int64, []),
     "mohge_workspace_bytes": (C.c_int64, [C.POINTER(mohge_config), C.c_int64]),
     "mohge_perm_rows": (C.c_int64, [C.POINTER(mohge_config), C.c_int64]),
-    "mohge_workspace_init": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, _P, _P]),
+    "mohge_workspace_init": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, _P, C.c_int64, _P]),
+    "mohge_get_switch": (C.c_int32, [C.c_char_p]),
+    "mohge_set_switch": (C.c_int32, [C.c_char_p, C.c_int32]),
+    "mohge_map_cache_stats": (None, [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]),
     "mohge_get_device_status": (C.c_int32, [_P, C.POINTER(C.c_int32), _P]),
     "mohge_route": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12),
     "mohge_aux_stats": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12),
@@ -164,13 +167,40 @@ def mohge_perm_rows(cfg: Config, T: int) -> int:
 
 
 def mohge_workspace_init(cfg, T, ws):
-    _check(lib().mohge_workspace_init(C.byref(cfg.c()), T, _ptr(ws), _stream()), "mohge_workspace_init")
+    _check(lib().mohge_workspace_init(C.byref(cfg.c()), T, _ptr(ws), ws.numel() * ws.element_size(),
+                                      _stream()), "mohge_workspace_init")
+
+
+MOHGE_ERR_TIMEOUT, MOHGE_ERR_DEVICE_CHECK = -5, -6
+
+
+def mohge_get_device_status_rc(ws):
+    """(return code, status word): the code is 0, MOHGE_ERR_TIMEOUT or MOHGE_ERR_DEVICE_CHECK as
+    decoded from the word by the library."""
+    out = C.c_int32(0)
+    rc = lib().mohge_get_device_status(_ptr(ws), C.byref(out), _stream())
+    if rc not in (0, MOHGE_ERR_TIMEOUT, MOHGE_ERR_DEVICE_CHECK):
+        _check(rc, "mohge_get_device_status")
+    return rc, out.value
 
 
 def mohge_get_device_status(ws) -> int:
-    out = C.c_int32(0)
-    _check(lib().mohge_get_device_status(_ptr(ws), C.byref(out), _stream()), "mohge_get_device_status")
-    return out.value
+    """The device status word (0 = nothing reported)."""
+    return mohge_get_device_status_rc(ws)[1]
+
+
+def mohge_get_switch(name: str) -> int:
+    return int(lib().mohge_get_switch(name.encode()))
+
+
+def mohge_set_switch(name: str, value: int) -> None:
+    _check(lib().mohge_set_switch(name.encode(), int(value)), "mohge_set_switch")
+
+
+def mohge_map_cache_stats():
+    h, m = C.c_int64(0), C.c_int64(0)
+    lib().mohge_map_cache_stats(C.byref(h), C.byref(m))
+    return h.value, m.value
 
 
 def mohge_route(cfg, T, x, w_router, logit_bias, logits_in, logits_out, group_idx, expert_idx,

@@ -1,6 +1,9 @@
 """Builds libmohge.so (sm_100a only) next to this file with nvcc.
 
-Usage: python -m paper_2604_23108_b200.build [--force]
+Usage: python -m paper_2604_23108_b200.build [--force] [-v] [--counters]
+
+--counters builds libmohge_counters.so instead: the same library compiled with
+-DMOHGE_TC_COUNTERS (per-CTA clock counters of the grouped GEMM, read by tc_counters.py).
 """
 from __future__ import annotations
 
@@ -41,8 +44,11 @@ def _stale(target: str, deps) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJ, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, counters: bool = False) -> str:
+    out = os.path.join(HERE, "libmohge_counters.so") if counters else OUT
+    obj_dir = os.path.join(OBJ, "counters") if counters else OBJ
+    common = COMMON + (["-DMOHGE_TC_COUNTERS"] if counters else [])
+    os.makedirs(obj_dir, exist_ok=True)
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
     headers.append(os.path.join(ROOT, "include", "mohge.h"))
     nvcc = _nvcc()
@@ -50,10 +56,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     objs = []
     for src, extra in SOURCES.items():
         s = os.path.join(CSRC, src)
-        o = os.path.join(OBJ, src.replace(".cu", ".o"))
+        o = os.path.join(obj_dir, src.replace(".cu", ".o"))
         objs.append(o)
         if force or _stale(o, [s] + headers):
-            cmd = [nvcc] + COMMON + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = [nvcc] + common + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
     def run(cmd):
@@ -66,10 +72,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         for log in ex.map(run, jobs):
             if verbose and log:
                 print(log)
-    if force or jobs or _stale(OUT, objs):
-        run([nvcc, "-shared", "-o", OUT] + objs)
-    return OUT
+    if force or jobs or _stale(out, objs):
+        run([nvcc, "-shared", "-o", out] + objs)
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, counters="--counters" in sys.argv))

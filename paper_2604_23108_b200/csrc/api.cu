@@ -5,6 +5,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mohge {
@@ -67,11 +70,56 @@ int32_t make_dims(const mohge_config* c, int64_t T, Dims* D) {
   return MOHGE_OK;
 }
 
-// Programmatic dependent launch (see common.cuh): on unless MOHGE_PDL=0.  Measured 1.5-2.5 % of the
-// step at the 8k- and 16k-token workloads, nothing at the large one.
-bool dependent_launch() {
-  const char* e = getenv("MOHGE_PDL");
-  return !(e && e[0] == '0');
+// ---------------------------------------------------------------- switches
+static const char* const kSwitchName[SW_COUNT] = {"pdl", "tc_cg", "tc_wide", "force_simt"};
+static const char* const kSwitchEnv[SW_COUNT] = {"MOHGE_PDL", "MOHGE_TC_CG", "MOHGE_TC_WIDE", "MOHGE_FORCE_SIMT"};
+static std::atomic<int> g_switch[SW_COUNT];
+static std::once_flag g_switch_once;
+
+static void read_switches_from_env() {
+  for (int i = 0; i < SW_COUNT; ++i) {
+    const char* e = getenv(kSwitchEnv[i]);
+    g_switch[i].store((e && e[0]) ? atoi(e) : -1);
+  }
+}
+static int switch_index(const char* name) {
+  for (int i = 0; name && i < SW_COUNT; ++i)
+    if (strcmp(name, kSwitchName[i]) == 0) return i;
+  return -1;
+}
+
+int switch_value(int which) {
+  std::call_once(g_switch_once, read_switches_from_env);
+  return g_switch[which].load(std::memory_order_relaxed);
+}
+
+// Programmatic dependent launch (see common.cuh): on unless the switch is 0.  Measured 1.5-2.5 %
+// of the step at the 8k- and 16k-token workloads, nothing at the large one.
+bool dependent_launch() { return switch_value(SW_PDL) != 0; }
+
+// ---------------------------------------------------------------- per-device facts
+int32_t current_device(DeviceInfo* out) {
+  static DeviceInfo table[kMaxDevices];
+  static std::atomic<bool> known[kMaxDevices];
+  static std::mutex mu;
+  int dev = 0;
+  MOHGE_CUDA(cudaGetDevice(&dev));
+  MOHGE_CHECK_ARG(dev >= 0 && dev < kMaxDevices, "device ordinal %d is not supported (at most %d devices)",
+                  dev, kMaxDevices);
+  if (!known[dev].load(std::memory_order_acquire)) {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!known[dev].load(std::memory_order_relaxed)) {
+      DeviceInfo di;
+      di.ordinal = dev;
+      MOHGE_CUDA(cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev));
+      MOHGE_CUDA(cudaDeviceGetAttribute(&di.cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+      MOHGE_CUDA(cudaDeviceGetAttribute(&di.cc_minor, cudaDevAttrComputeCapabilityMinor, dev));
+      table[dev] = di;
+      known[dev].store(true, std::memory_order_release);
+    }
+  }
+  *out = table[dev];
+  return MOHGE_OK;
 }
 
 static int64_t up256(int64_t v) { return (v + 255) / 256 * 256; }
@@ -148,10 +196,7 @@ static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 #define REQ_PTR(p) MOHGE_CHECK_ARG((p) != nullptr && aligned16(p), #p " must be a non-NULL 16-byte aligned device pointer")
 #define OPT_PTR(p) MOHGE_CHECK_ARG(aligned16(p), #p " must be 16-byte aligned")
 
-static bool force_simt() {
-  const char* e = getenv("MOHGE_FORCE_SIMT");
-  return e && e[0] == '1';
-}
+static bool force_simt() { return switch_value(SW_FORCE_SIMT) == 1; }
 
 static int32_t group_ptrs(const Dims& D, const void* const* w13, const void* const* w2,
                           float* const* dw13, float* const* dw2, GroupPtrs* P) {
@@ -187,11 +232,35 @@ int64_t mohge_perm_rows(const mohge_config* cfg, int64_t T) {
   return D.Rcap;
 }
 
-int32_t mohge_workspace_init(const mohge_config* cfg, int64_t T, void* ws, void* stream) {
+int32_t mohge_get_switch(const char* name) {
+  const int i = switch_index(name);
+  if (i < 0) {
+    set_error("unknown switch '%s' (pdl, tc_cg, tc_wide, force_simt)", name ? name : "(null)");
+    return INT32_MIN;
+  }
+  return switch_value(i);
+}
+
+int32_t mohge_set_switch(const char* name, int32_t value) {
+  const int i = switch_index(name);
+  MOHGE_CHECK_ARG(i >= 0, "unknown switch '%s' (pdl, tc_cg, tc_wide, force_simt)", name ? name : "(null)");
+  MOHGE_CHECK_ARG(value >= -1, "switch value %d: -1 (library's rule) or a non-negative value", value);
+  (void)switch_value(i);          // the environment is consulted first, once, and never again
+  g_switch[i].store(value);
+  return MOHGE_OK;
+}
+
+int32_t mohge_workspace_init(const mohge_config* cfg, int64_t T, void* ws, int64_t ws_bytes, void* stream) {
   Dims D;
   int32_t rc = make_dims(cfg, T, &D);
   if (rc) return rc;
   REQ_PTR(ws);
+  const int64_t need = ws_layout(D).total;
+  if (ws_bytes < need) {
+    set_error("workspace of %lld bytes is too small: this configuration and T = %lld need %lld",
+              (long long)ws_bytes, (long long)T, (long long)need);
+    return MOHGE_ERR_WORKSPACE;
+  }
   MOHGE_CUDA(cudaMemsetAsync(ws, 0, 256, (cudaStream_t)stream));
   return MOHGE_OK;
 }
@@ -200,7 +269,15 @@ int32_t mohge_get_device_status(const void* ws, int32_t* host_out, void* stream)
   MOHGE_CHECK_ARG(ws != nullptr && host_out != nullptr, "ws and host_out must be non-NULL");
   MOHGE_CUDA(cudaMemcpyAsync(host_out, ws, sizeof(int32_t), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   MOHGE_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
-  return MOHGE_OK;
+  const int32_t word = *host_out, code = word >> 24, site = word & 0xffffff;
+  if (word == 0) return MOHGE_OK;
+  if (code == 1) {
+    set_error("a device-side wait gave up after its time budget (site %d of the grouped GEMM kernel)", site);
+    return MOHGE_ERR_TIMEOUT;
+  }
+  set_error(code == 2 ? "a device-side index check failed (site %d): the entry was skipped"
+                      : "NaN among the router logits (code %d): ranked below every number", code == 2 ? site : code);
+  return MOHGE_ERR_DEVICE_CHECK;
 }
 
 int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const void* w_router,
@@ -230,7 +307,8 @@ int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const voi
       MOHGE_CUDA(cudaMemcpyAsync(logits_out, logits_in, sizeof(float) * T * D.NL,
                                  cudaMemcpyDeviceToDevice, st));
   }
-  return launch_router_select(D, logits, group_idx, expert_idx, gate_w, gs_saved, esp_saved, st);
+  return launch_router_select(D, logits, group_idx, expert_idx, gate_w, gs_saved, esp_saved,
+                              carve(D, ws).status, st);
 }
 
 int32_t mohge_aux_stats(const mohge_config* cfg, int64_t T, const float* gs_saved,

@@ -50,7 +50,22 @@ __device__ __forceinline__ void pdl_enter() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 #endif
-bool dependent_launch();   // false when MOHGE_PDL=0
+bool dependent_launch();   // false when the "pdl" switch is 0
+
+// ---------------------------------------------------------------- switches and per-device facts
+// Debugging switches.  Each is read ONCE from its environment variable, the first time any
+// switch is asked for, and can afterwards be changed only through mohge_set_switch(); -1 means
+// "not set: the library's own rule decides".
+enum Switch { SW_PDL = 0, SW_TC_CG = 1, SW_TC_WIDE = 2, SW_FORCE_SIMT = 3, SW_COUNT = 4 };
+int switch_value(int which);
+// What the launchers need to know about the current device, looked up once per device ordinal
+// (a process may drive several GPUs; kernel attributes such as the dynamic shared-memory limit
+// are per device too, see launch_role in gemm_tc.cu).
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+  int ordinal, sm_count, cc_major, cc_minor;
+};
+int32_t current_device(DeviceInfo* out);
 
 template <typename... KArgs, typename... Args>
 inline void launch_dep(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args&&... args) {
@@ -150,7 +165,7 @@ GroupShape make_group_shape(const Dims& D);
 // router.cu
 int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_idx,
                              int32_t* expert_idx, float* gate_w, float* gs, float* esp,
-                             cudaStream_t st);
+                             int32_t* status, cudaStream_t st);
 int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs, const float* esp,
                          const int32_t* group_idx, const int32_t* expert_idx, int32_t* group_count,
                          float* group_psum, int32_t* cnt_routed, int32_t* cnt_lit,

@@ -34,6 +34,9 @@
 
 #include <cuda.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mohge {
@@ -1262,6 +1265,59 @@ int32_t encode_stage_map_f32(CUtensorMap* m, const void* base, uint64_t cols, ui
   return encode_map(m, base, 3, dims, str, box, true);
 }
 
+// Encoded tensor maps are kept per (device, role, tile form, operand addresses, shapes): a layer
+// that is stepped on the same buffers encodes each map once instead of on every launch (up to
+// five cuTensorMapEncodeTiled calls per group and launch, about a hundred per step; host time on
+// the critical path of the launch-bound small workloads).  A map depends on nothing but the
+// address and the shape, so a hit can never be stale.  Fixed size, oldest entry replaced first.
+struct MapKey {
+  int32_t role, cg, device, accumulate_unused;
+  int32_t d, Ng, N, Wmax, W[MOHGE_MAX_GROUPS];
+  int64_t rows, T, b_pitch;
+  const void *A, *B, *C, *C2;
+  const void* w[4][MOHGE_MAX_GROUPS];
+};
+struct MapEntry {
+  MapKey key;
+  CUtensorMap mapA[MOHGE_MAX_GROUPS], mapB[MOHGE_MAX_GROUPS], mapO[3][MOHGE_MAX_GROUPS], mapE[2][MOHGE_MAX_GROUPS];
+  int BN[MOHGE_MAX_GROUPS];
+  unsigned char a_blk[MOHGE_MAX_GROUPS], b_blk[MOHGE_MAX_GROUPS];
+  bool valid;
+};
+constexpr int kMapCacheEntries = 64;
+MapEntry g_map_cache[kMapCacheEntries];
+int g_map_cache_next = 0;
+std::mutex g_map_cache_mu;
+std::atomic<long long> g_map_hits{0}, g_map_misses{0};
+
+bool map_cache_find(const MapKey& key, TcParams* p) {
+  std::lock_guard<std::mutex> lock(g_map_cache_mu);
+  for (int i = 0; i < kMapCacheEntries; ++i) {
+    const MapEntry& e = g_map_cache[i];
+    if (e.valid && memcmp(&e.key, &key, sizeof(MapKey)) == 0) {
+      memcpy(p->mapA, e.mapA, sizeof(e.mapA)); memcpy(p->mapB, e.mapB, sizeof(e.mapB));
+      memcpy(p->mapO, e.mapO, sizeof(e.mapO)); memcpy(p->mapE, e.mapE, sizeof(e.mapE));
+      memcpy(p->BN, e.BN, sizeof(e.BN)); memcpy(p->a_blk, e.a_blk, sizeof(e.a_blk));
+      memcpy(p->b_blk, e.b_blk, sizeof(e.b_blk));
+      ++g_map_hits;
+      return true;
+    }
+  }
+  ++g_map_misses;
+  return false;
+}
+void map_cache_store(const MapKey& key, const TcParams& p) {
+  std::lock_guard<std::mutex> lock(g_map_cache_mu);
+  MapEntry& e = g_map_cache[g_map_cache_next];
+  g_map_cache_next = (g_map_cache_next + 1) % kMapCacheEntries;
+  e.key = key;
+  memcpy(e.mapA, p.mapA, sizeof(e.mapA)); memcpy(e.mapB, p.mapB, sizeof(e.mapB));
+  memcpy(e.mapO, p.mapO, sizeof(e.mapO)); memcpy(e.mapE, p.mapE, sizeof(e.mapE));
+  memcpy(e.BN, p.BN, sizeof(e.BN)); memcpy(e.a_blk, p.a_blk, sizeof(e.a_blk));
+  memcpy(e.b_blk, p.b_blk, sizeof(e.b_blk));
+  e.valid = true;
+}
+
 // Tile width per group.  Candidates come widest first.  A narrower tile is taken only when it
 // cuts the padded extent by more than a fifth: a 128-wide tile needs half again as many operand
 // bytes per FLOP as a 256-wide one, which costs more than a few percent of padded columns
@@ -1280,12 +1336,16 @@ int pick_bn(int extent, const int* cand, int ncand) {
 }
 
 template <int ROLE, int CG, int WIDE = 0>
-int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+int32_t launch_role(const TcParams& p, const DeviceInfo& di, cudaStream_t st) {
+  // The dynamic shared-memory limit of a kernel and the number of CTA pairs that fit are facts
+  // of one device: both are kept per device ordinal (0 = not yet known on that device).
+  static std::atomic<int> attr_set[kMaxDevices];
+  static std::atomic<int> max_clusters[kMaxDevices];
+  const int grid = is_plain<ROLE>() ? (p.plain_total < di.sm_count ? p.plain_total : di.sm_count) : di.sm_count;
+  if (!attr_set[di.ordinal].load(std::memory_order_acquire)) {
     MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE, CG, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     Geo<CG, WIDE>::kSmemBytes));
-    attr_set = true;
+    attr_set[di.ordinal].store(1, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
@@ -1306,13 +1366,13 @@ int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
     // Persistent kernel: launch exactly as many CTA pairs as can be resident at once (SMs that
     // cannot be paired stay idle); a pair that had to wait for a free slot would run its whole
     // share of the tile list after everyone else.
-    static int max_clusters = 0;
-    if (!max_clusters) {
-      cfg.gridDim = dim3(grid / CG * CG);
-      MOHGE_CUDA(cudaOccupancyMaxActiveClusters(&max_clusters, tc_grouped_kernel<ROLE, CG, WIDE>, &cfg));
-      if (max_clusters < 1) max_clusters = 1;
+    int mc = max_clusters[di.ordinal].load(std::memory_order_acquire);
+    if (!mc) {
+      MOHGE_CUDA(cudaOccupancyMaxActiveClusters(&mc, tc_grouped_kernel<ROLE, CG, WIDE>, &cfg));
+      if (mc < 1) mc = 1;
+      max_clusters[di.ordinal].store(mc, std::memory_order_release);
     }
-    const int want = grid / CG < max_clusters ? grid / CG : max_clusters;
+    const int want = grid / CG < mc ? grid / CG : mc;
     cfg.gridDim = dim3(want * CG);
   }
   cfg.numAttrs = dependent_launch() ? 2 : 1;
@@ -1333,8 +1393,12 @@ int32_t launch_role(const TcParams& p, int grid, cudaStream_t st) {
 // switch MOHGE_TC_WIDE=<bit mask over roles 0..5> overrides the rule.
 constexpr double kWideMinK = 3000.0;
 bool wide_tiles(const Dims& D, int role) {
-  const char* e = getenv("MOHGE_TC_WIDE");
-  if (e && e[0]) return (atoi(e) >> role) & 1;
+  const int mask = switch_value(SW_TC_WIDE);
+  if (mask >= 0) return (mask >> role) & 1;
+  // The SwiGLU backward has the longest epilogue of all roles (it also reads A and U); exposed at
+  // every entry boundary it costs more than the saved operand traffic brings (measured at the
+  // large workload: step 44.1 -> 43.8 ms with this role on single-width tiles).
+  if (role == ROLE_DGRAD_DOWN) return false;
   double num = 0.0, den = 0.0;            // mean contraction length, weighted by the group's width
   for (int g = 0; g < D.Ng; ++g) {
     double k;
@@ -1356,9 +1420,8 @@ bool wide_tiles(const Dims& D, int role) {
 // and A loads on rows of the next expert, so single CTAs with 128-row tiles run instead (measured
 // 5.6 against 4.9 TB/s of weight traffic at 16 rows per expert).  MOHGE_TC_CG=1|2 forces a form.
 int cta_group_size(const Dims& D) {
-  const char* e = getenv("MOHGE_TC_CG");
-  if (e && e[0] == '1') return 1;
-  if (e && e[0] == '2') return 2;
+  const int forced = switch_value(SW_TC_CG);
+  if (forced == 1 || forced == 2) return forced;
   return D.R <= 128 * (int64_t)D.Ne ? 1 : 2;
 }
 
@@ -1413,13 +1476,14 @@ int router_logits_splits(const Dims& D, int n_tiles) {
 
 int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
                         void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st) {
-  static int sm_count = 0;
-  if (!sm_count) {
-    int dev = 0;
-    MOHGE_CUDA(cudaGetDevice(&dev));
-    MOHGE_CUDA(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-  }
   if (D.T == 0) return MOHGE_OK;
+  DeviceInfo di;
+  int32_t rcd = current_device(&di);
+  if (rcd) return rcd;
+  if (di.cc_major != 10) {
+    set_error("the BF16 path needs an sm_100 device (found sm_%d%d)", di.cc_major, di.cc_minor);
+    return MOHGE_ERR_UNSUPPORTED;
+  }
   TcParams p;
   memset(&p, 0, sizeof(p));
   p.gs = make_group_shape(D);
@@ -1429,31 +1493,44 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
   uint64_t dims[2], str[1];
   uint32_t box[2];
   int32_t rc;
+  // shapes
   if (role == ROLE_LOGITS) {
     p.plain_M = (int)T; p.plain_N = D.NL; p.plain_K = D.d;
-    p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 15) / 16 * 16;
     p.Cf = (float*)C;
-    dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = BK; box[1] = BM;
-    if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
-    dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = BK; box[1] = p.BN[0];
-    if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
   } else if (role == ROLE_ROUTER_DW) {
     p.plain_M = D.d; p.plain_N = D.NL; p.plain_K = (int)T;
-    p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 63) / 64 * 64;
     p.Cf = (float*)C;
-    dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = 64; box[1] = BK;
-    if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
-    dims[0] = NL; dims[1] = T; str[0] = (uint64_t)b_pitch_elems * 2; box[0] = 64; box[1] = BK;
-    if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
   } else {  // ROLE_ROUTER_DX
     p.plain_M = (int)T; p.plain_N = D.d; p.plain_K = D.NL;
-    p.BN[0] = D.d >= 256 ? 256 : (D.d + 63) / 64 * 64;
     p.C = (__nv_bfloat16*)C;
-    dims[0] = NL; dims[1] = T; str[0] = (uint64_t)b_pitch_elems * 2; box[0] = BK; box[1] = BM;
-    if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
-    dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = 64; box[1] = BK;
-    if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
-    if ((rc = encode_stage_map(&p.mapO[0][0], C, d, T, d * 2))) return rc;    // dx, read and written
+  }
+  // tensor maps: from the cache, or encoded now
+  MapKey key;
+  memset(&key, 0, sizeof(key));
+  key.role = role; key.cg = 1; key.device = di.ordinal; key.d = D.d; key.Ng = D.Ng; key.N = D.N;
+  key.T = D.T; key.b_pitch = b_pitch_elems; key.A = A; key.B = B; key.C = C;
+  if (!map_cache_find(key, &p)) {
+    if (role == ROLE_LOGITS) {
+      p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 15) / 16 * 16;
+      dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = BK; box[1] = BM;
+      if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
+      dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = BK; box[1] = p.BN[0];
+      if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+    } else if (role == ROLE_ROUTER_DW) {
+      p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 63) / 64 * 64;
+      dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = 64; box[1] = BK;
+      if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
+      dims[0] = NL; dims[1] = T; str[0] = (uint64_t)b_pitch_elems * 2; box[0] = 64; box[1] = BK;
+      if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+    } else {
+      p.BN[0] = D.d >= 256 ? 256 : (D.d + 63) / 64 * 64;
+      dims[0] = NL; dims[1] = T; str[0] = (uint64_t)b_pitch_elems * 2; box[0] = BK; box[1] = BM;
+      if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
+      dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = 64; box[1] = BK;
+      if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+      if ((rc = encode_stage_map(&p.mapO[0][0], C, d, T, d * 2))) return rc;    // dx, read and written
+    }
+    map_cache_store(key, p);
   }
   p.plain_ntn = (p.plain_N + p.BN[0] - 1) / p.BN[0];
   const int total_kb = (p.plain_K + BK - 1) / BK;
@@ -1470,11 +1547,10 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
     if (p.plain_splits > 1) p.Cf = partials;
   }
   p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn * p.plain_splits;
-  const int grid = p.plain_total < sm_count ? p.plain_total : sm_count;
   switch (role) {
     case ROLE_LOGITS: {
-      const int32_t rc2 = p.BN[0] <= 160 ? launch_role<ROLE_LOGITS, 1, 2>(p, grid, st)
-                                          : launch_role<ROLE_LOGITS, 1>(p, grid, st);
+      const int32_t rc2 = p.BN[0] <= 160 ? launch_role<ROLE_LOGITS, 1, 2>(p, di, st)
+                                          : launch_role<ROLE_LOGITS, 1>(p, di, st);
       if (rc2 || p.plain_splits == 1) return rc2;
       const size_t n = (size_t)D.T * D.NL;
       launch_dep(sum_partials_bias_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), st, partials, p.plain_splits, n, D.NL,
@@ -1483,14 +1559,14 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
       return MOHGE_OK;
     }
     case ROLE_ROUTER_DW: {
-      const int32_t rc2 = launch_role<ROLE_ROUTER_DW, 1>(p, grid, st);
+      const int32_t rc2 = launch_role<ROLE_ROUTER_DW, 1>(p, di, st);
       if (rc2 || p.plain_splits == 1) return rc2;
       const size_t n = (size_t)D.NL * D.d;
       launch_dep(sum_partials_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), st, partials, p.plain_splits, n, (float*)C);
       MOHGE_LAUNCH_CHECK("sum_partials_kernel");
       return MOHGE_OK;
     }
-    default: return launch_role<ROLE_ROUTER_DX, 1>(p, grid, st);
+    default: return launch_role<ROLE_ROUTER_DX, 1>(p, di, st);
   }
 }
 
@@ -1532,17 +1608,12 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
                           int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt,
                           float* dgate_part, int dgate_slots) {
-  static int sm_count = 0;
-  if (!sm_count) {
-    int dev = 0;
-    MOHGE_CUDA(cudaGetDevice(&dev));
-    cudaDeviceProp prop;
-    MOHGE_CUDA(cudaGetDeviceProperties(&prop, dev));
-    if (prop.major != 10) {
-      set_error("the BF16 path needs an sm_100 device (found sm_%d%d)", prop.major, prop.minor);
-      return MOHGE_ERR_UNSUPPORTED;
-    }
-    sm_count = prop.multiProcessorCount;
+  DeviceInfo di;
+  int32_t rcd = current_device(&di);
+  if (rcd) return rcd;
+  if (di.cc_major != 10) {
+    set_error("the BF16 path needs an sm_100 device (found sm_%d%d)", di.cc_major, di.cc_minor);
+    return MOHGE_ERR_UNSUPPORTED;
   }
   TcParams p;
   memset(&p, 0, sizeof(p));
@@ -1564,7 +1635,18 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   int bn_plan[MOHGE_MAX_GROUPS];
   int32_t rc = MOHGE_OK;
   for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) { p.BN[g] = 128; bn_plan[g] = 128; }
-  for (int g = 0; g < D.Ng && rc == MOHGE_OK; ++g) {
+  if (role == ROLE_DGRAD_DOWN) p.E = (const __nv_bfloat16*)B;
+  MapKey key;
+  memset(&key, 0, sizeof(key));
+  key.role = role; key.cg = CG; key.device = di.ordinal;
+  key.d = D.d; key.Ng = D.Ng; key.N = D.N; key.Wmax = D.Wmax; key.rows = D.Rcap;
+  key.A = A; key.B = B; key.C = C; key.C2 = C2;
+  for (int g = 0; g < D.Ng; ++g) {
+    key.W[g] = D.W[g];
+    key.w[0][g] = P.w13[g]; key.w[1][g] = P.w2[g]; key.w[2][g] = P.dw13[g]; key.w[3][g] = P.dw2[g];
+  }
+  const bool cached = map_cache_find(key, &p);
+  for (int g = 0; g < D.Ng && rc == MOHGE_OK && !cached; ++g) {
     const uint64_t W = D.W[g], N = D.N;
     uint64_t dims[3], str[2];
     uint32_t box[3];
@@ -1598,7 +1680,6 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
       } break;
       case ROLE_DGRAD_DOWN: {
         p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
-        p.E = (const __nv_bfloat16*)B;
         dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
         rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
         if (rc) break;
@@ -1640,6 +1721,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
     }
   }
   if (rc) return rc;
+  if (!cached) map_cache_store(key, p);
   const TilePlan plan = tc_tile_plan(D, role);
   const bool wide = plan.wide != 0;
   if (!list_prebuilt) {
@@ -1648,35 +1730,40 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   }
   if (CG == 2 && wide) {
     switch (role) {
-      case ROLE_FWD1: return launch_role<ROLE_FWD1, 2, 1>(p, sm_count, st);
-      case ROLE_FWD2: return launch_role<ROLE_FWD2, 2, 1>(p, sm_count, st);
-      case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 2, 1>(p, sm_count, st);
-      case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 2, 1>(p, sm_count, st);
-      case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 2, 1>(p, sm_count, st);
-      default: return launch_role<ROLE_WGRAD_13, 2, 1>(p, sm_count, st);
+      case ROLE_FWD1: return launch_role<ROLE_FWD1, 2, 1>(p, di, st);
+      case ROLE_FWD2: return launch_role<ROLE_FWD2, 2, 1>(p, di, st);
+      case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 2, 1>(p, di, st);
+      case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 2, 1>(p, di, st);
+      case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 2, 1>(p, di, st);
+      default: return launch_role<ROLE_WGRAD_13, 2, 1>(p, di, st);
     }
   }
   if (CG == 2) {
     switch (role) {
-      case ROLE_FWD1: return launch_role<ROLE_FWD1, 2>(p, sm_count, st);
-      case ROLE_FWD2: return launch_role<ROLE_FWD2, 2>(p, sm_count, st);
-      case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 2>(p, sm_count, st);
-      case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 2>(p, sm_count, st);
-      case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 2>(p, sm_count, st);
-      default: return launch_role<ROLE_WGRAD_13, 2>(p, sm_count, st);
+      case ROLE_FWD1: return launch_role<ROLE_FWD1, 2>(p, di, st);
+      case ROLE_FWD2: return launch_role<ROLE_FWD2, 2>(p, di, st);
+      case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 2>(p, di, st);
+      case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 2>(p, di, st);
+      case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 2>(p, di, st);
+      default: return launch_role<ROLE_WGRAD_13, 2>(p, di, st);
     }
   }
   switch (role) {
-    case ROLE_FWD1: return launch_role<ROLE_FWD1, 1>(p, sm_count, st);
-    case ROLE_FWD2: return launch_role<ROLE_FWD2, 1>(p, sm_count, st);
-    case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 1>(p, sm_count, st);
-    case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 1>(p, sm_count, st);
-    case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 1>(p, sm_count, st);
-    default: return launch_role<ROLE_WGRAD_13, 1>(p, sm_count, st);
+    case ROLE_FWD1: return launch_role<ROLE_FWD1, 1>(p, di, st);
+    case ROLE_FWD2: return launch_role<ROLE_FWD2, 1>(p, di, st);
+    case ROLE_DGRAD_DOWN: return launch_role<ROLE_DGRAD_DOWN, 1>(p, di, st);
+    case ROLE_DGRAD_13: return launch_role<ROLE_DGRAD_13, 1>(p, di, st);
+    case ROLE_WGRAD_DOWN: return launch_role<ROLE_WGRAD_DOWN, 1>(p, di, st);
+    default: return launch_role<ROLE_WGRAD_13, 1>(p, di, st);
   }
 }
 
 }  // namespace mohge
+
+extern "C" void mohge_map_cache_stats(int64_t* hits, int64_t* misses) {
+  if (hits) *hits = (int64_t)mohge::g_map_hits.load();
+  if (misses) *misses = (int64_t)mohge::g_map_misses.load();
+}
 
 #ifdef MOHGE_TC_COUNTERS
 // Copies the counter table [9 roles][160 CTAs][12 slots] (uint64) to `host_out` after a device

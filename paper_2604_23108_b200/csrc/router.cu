@@ -18,6 +18,9 @@
 //            key_i = p_i * r; ES'_i = p_i / S.  Experts of unselected groups: key = -1.
 //   experts  K_e rounds of arg-max over (key descending, e ascending)
 //   gate_k = key_k / (left-to-right sum of the K_e selected keys)
+//   NaN      a NaN logit is invalid input: it is read as -FLT_MAX (the most negative finite
+//            float32), i.e. it ranks below every number, ties among such entries go to the lowest
+//            index as everywhere else, and the device status word records (3 << 24)
 //
 // Slot layout inside a warp: group g owns P = next_pow2(N) consecutive slots, slot s = g*P + i
 // lives in lane s % 32, register s / 32; a group never straddles a register because P | 32.
@@ -108,16 +111,21 @@ template <int J>
 __global__ void __launch_bounds__(256)
 router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* __restrict__ group_idx,
                      int32_t* __restrict__ expert_idx, float* __restrict__ gate_w,
-                     float* __restrict__ gs_saved, float* __restrict__ esp_saved) {
+                     float* __restrict__ gs_saved, float* __restrict__ esp_saved, int32_t* status) {
   pdl_enter();
   const int lane = threadIdx.x & 31;
+  bool saw_nan = false;
+  auto clean = [&](float v) {                 // NaN logits rank below every number
+    if (v != v) { saw_nan = true; return -3.402823466e+38f; }
+    return v;
+  };
   const int warps_total = (gridDim.x * blockDim.x) >> 5;
   for (int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < s.T; t += warps_total) {
     const float* L = logits + (size_t)t * s.NL;
     // ---- Eq. 2: top-K_g groups by raw logit ----
     float lg[MOHGE_MAX_GROUPS];
 #pragma unroll
-    for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) lg[g] = g < s.Ng ? L[g] : 0.0f;
+    for (int g = 0; g < MOHGE_MAX_GROUPS; ++g) lg[g] = g < s.Ng ? clean(L[g]) : 0.0f;
     unsigned gmask = 0;
     for (int k = 0; k < s.Kg; ++k) {
       int best = -1;
@@ -132,7 +140,7 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
       gmask |= 1u << best;
       if (lane == 0) group_idx[(size_t)t * s.Kg + k] = best;
     }
-    const float gsv = lane < s.Ng ? sig_s(L[lane]) : 0.0f;      // GS of group `lane`
+    const float gsv = lane < s.Ng ? sig_s(clean(L[lane])) : 0.0f;      // GS of group `lane`
     if (lane < s.Ng) gs_saved[(size_t)t * s.Ng + lane] = gsv;
     // ---- Eq. 3, 4: keys of the lane's slots ----
     float key[J];
@@ -144,7 +152,7 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
       const int i = sl & (s.P - 1);
       const bool valid = g < s.Ng && i < s.N;
       const int e = g * s.N + i;
-      const float l = valid ? L[s.Ng + e] : -INFINITY;
+      const float l = valid ? clean(L[s.Ng + e]) : -INFINITY;
       float m = l;
       for (int mask = s.P >> 1; mask > 0; mask >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, mask));
       const float p = valid ? exp_s(__fsub_rn(l, m)) : 0.0f;
@@ -173,6 +181,7 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
       gate_w[(size_t)t * s.Ke + lane] = __fdiv_rn(wk, sum);
     }
   }
+  if (saw_nan && status != nullptr) atomicCAS(status, 0, 3 << 24);
 }
 
 // the three count arrays start at zero (one launch instead of three memsets)
@@ -456,12 +465,12 @@ int slots_per_lane(const Dims& D) {
 
 int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_idx,
                              int32_t* expert_idx, float* gate_w, float* gs, float* esp,
-                             cudaStream_t st) {
+                             int32_t* status, cudaStream_t st) {
   if (D.T == 0) return MOHGE_OK;
   const RouterShape s = make_shape(D);
   const int blocks = (int)((D.T + 7) / 8) < 148 * 8 ? (int)((D.T + 7) / 8) : 148 * 8;
   MOHGE_DISPATCH_J(slots_per_lane(D), (launch_dep(router_select_kernel<JJ>, dim3(blocks), dim3(256), st,
-                                          s, logits, group_idx, expert_idx, gate_w, gs, esp)));
+                                          s, logits, group_idx, expert_idx, gate_w, gs, esp, status)));
   MOHGE_LAUNCH_CHECK("router_select_kernel");
   return MOHGE_OK;
 }
@@ -535,7 +544,6 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
 namespace mohge {
 namespace {
 static __device__ __align__(256) double g_static_partials[kStatsBlocks * MOHGE_STATIC_MAX_LOGITS];
-constexpr int kMaxDevices = 64;
 double* g_static_ptr[kMaxDevices] = {nullptr};
 }  // namespace
 }  // namespace mohge

@@ -36,6 +36,18 @@ def max_rel(a, b) -> float:
     return float(np.max(np.abs(a - b)) / den)
 
 
+def elementwise_outliers(a, b, tol) -> float:
+    """Share of elements with |a - b| > tol |b| + tol rms(b): the secondary, element-wise figure
+    reported beside max_rel (a per-tensor maximum cannot see a large relative error on a small
+    element; this one can, down to elements of the size of tol rms)."""
+    a = np.asarray(a, np.float64)
+    b = np.asarray(b, np.float64)
+    if b.size == 0:
+        return 0.0
+    rms = float(np.sqrt(np.mean(b * b)))
+    return float(np.mean(np.abs(a - b) > tol * np.abs(b) + tol * rms))
+
+
 def tol_for(dtype: str) -> float:
     return 2e-2 if dtype == "bf16" else 1e-5
 
@@ -72,3 +84,25 @@ def gpu_layer(wl: Workload, inp, gcfg=None, logits32=None, with_aux=True, accumu
     torch.cuda.synchronize()
     assert B.mohge_get_device_status(b.ws) == 0
     return b, dev
+
+
+class forced_switches:
+    """Context manager: sets debugging switches of the library ("MOHGE_TC_CG=2,MOHGE_TC_WIDE=63"
+    in the spelling of their environment variables) and puts the library's own rules back after."""
+
+    def __init__(self, spec: str):
+        self.items = [kv.split("=") for kv in spec.split(",") if kv]
+
+    @staticmethod
+    def _name(env_name: str) -> str:
+        return env_name[len("MOHGE_"):].lower()
+
+    def __enter__(self):
+        for name, value in self.items:
+            B.mohge_set_switch(self._name(name), int(value))
+        return self
+
+    def __exit__(self, *exc):
+        for name, _ in self.items:
+            B.mohge_set_switch(self._name(name), -1)
+        return False

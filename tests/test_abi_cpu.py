@@ -80,6 +80,46 @@ def test_combine_bwd_takes_y_perm_and_dgate_together_or_not_at_all():
     assert rc == -1 and b"y_perm" in lib.mohge_last_error()
 
 
+def test_switches_are_read_from_the_environment_once():
+    """The debugging switches come from the environment the first time one is consulted; later
+    changes of the environment are not seen, mohge_set_switch is the only way to change one.
+    Runs in a child process so that the first consultation is under the test's control."""
+    import subprocess
+    import sys
+    code = r'''
+import os, sys
+sys.path.insert(0, %r)
+os.environ["MOHGE_TC_CG"] = "1"
+os.environ.pop("MOHGE_TC_WIDE", None)
+from paper_2604_23108_b200 import binding as B
+assert B.mohge_get_switch("tc_cg") == 1              # first consultation reads the environment
+assert B.mohge_get_switch("tc_wide") == -1           # not set: the library's rule decides
+os.environ["MOHGE_TC_CG"] = "2"
+os.environ["MOHGE_TC_WIDE"] = "63"
+assert B.mohge_get_switch("tc_cg") == 1              # the environment is not read again
+assert B.mohge_get_switch("tc_wide") == -1
+B.mohge_set_switch("tc_cg", 2)
+assert B.mohge_get_switch("tc_cg") == 2
+B.mohge_set_switch("tc_cg", -1)
+assert B.mohge_get_switch("tc_cg") == -1
+assert B.lib().mohge_get_switch(b"no_such_switch") == -2**31
+assert B.lib().mohge_set_switch(b"no_such_switch", 1) == -1
+assert B.lib().mohge_set_switch(b"pdl", -7) == -1
+print("ok")
+''' % ROOT
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True)
+    assert out.returncode == 0 and out.stdout.strip() == "ok", out.stderr
+
+
+def test_workspace_init_refuses_a_workspace_that_is_too_small():
+    lib = B.lib()
+    cfg = B.Config(1024, 3, 8, 2, 4, [1408, 704, 352])
+    need = B.mohge_workspace_bytes(cfg, 8192)
+    rc = lib.mohge_workspace_init(C.byref(cfg.c()), 8192, C.c_void_p(256), need - 1, None)
+    assert rc == -3                                    # MOHGE_ERR_WORKSPACE, nothing touched
+    assert str(need).encode() in lib.mohge_last_error()
+
+
 def test_header_and_library_are_usable_from_plain_c(tmp_path):
     """A C99 program includes mohge.h, links libmohge.so and asks for sizes (no device needed)."""
     import shutil

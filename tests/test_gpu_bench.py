@@ -22,11 +22,17 @@ def _run(*extra):
 
 
 def test_bench_line_has_the_whole_contract():
-    d = _run("--ref-sample", "64")
+    d = _run()
     for k in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
               "scaling", "vs_baseline", "dtype", "data", "config", "clocks", "e2e", "gpu_launches",
-              "roofline", "cpu_baseline", "device_status"):
+              "roofline", "cpu_baseline", "device_status", "roofline_hbm_steps", "other_workloads",
+              "host_enqueue_ms_per_step"):
         assert k in d, k
+    assert d["other_workloads"] is None                # only the default workload's line carries them
+    steps = {r["step"]: r for r in d["roofline_hbm_steps"]}
+    assert set(steps) == {"route", "aux_stats", "dispatch", "combine", "combine_bwd", "dispatch_bwd", "route_bwd"}
+    assert all(r["ms"] > 0 and r["bytes"] > 0 and r["unit"] == "GB/s" for r in steps.values())
+    assert d["config"]["count_ratio"] is None or d["config"]["count_ratio"] >= 1.0
     assert d["unit"] == "tokens/s" and d["n_gpus"] == 1 and d["steps"] == 5 and d["warmup"] == 3
     assert d["value"] > 0 and abs(d["value"] - 256 / (d["ms_per_step"] * 1e-3)) <= 1e-6 * d["value"]
     assert d["config"]["workload"] == "cfg1_tiny_f32" and d["dtype"] == "f32" and d["data"] == "synthetic"
@@ -35,7 +41,7 @@ def test_bench_line_has_the_whole_contract():
     assert d["e2e"]["d2h_bytes_per_step"] > d["e2e"]["h2d_bytes_per_step"]
     assert set(("bound", "achieved", "peak", "unit", "frac", "traffic")) <= set(d["roofline"])
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
-    assert d["cpu_baseline"]["value"] > 0 and "64" in d["cpu_baseline"]["sample"]
+    assert d["cpu_baseline"]["value"] > 0 and "256 tokens" in d["cpu_baseline"]["sample"]
     assert set(("sm_mhz", "sm_max_mhz", "reasons")) <= set(d["clocks"])
 
 

@@ -8,7 +8,7 @@ import oracle as O
 from paper_2604_23108_b200 import binding as B
 from paper_2604_23108_b200.inputs import Workload, make_inputs
 
-from _util import gpu_cfg, gpu_layer, max_rel, oracle_cfg, oracle_layer, to_np64, tol_for
+from _util import forced_switches, gpu_cfg, gpu_layer, max_rel, oracle_cfg, oracle_layer, to_np64, tol_for
 
 pytestmark = pytest.mark.gpu
 
@@ -109,28 +109,113 @@ def test_out_of_range_expert_index_sets_the_status_word_without_faulting():
     B.mohge_dispatch(gcfg, 64, x, idx, b.counts, b.offsets, b.aligned, b.row_of, b.prow_of,
                      b.src_of, b.x_perm, b.ws)
     torch.cuda.synchronize()
-    assert B.mohge_get_device_status(b.ws) >> 24 == 2
+    rc, word = B.mohge_get_device_status_rc(b.ws)
+    assert word >> 24 == 2 and rc == B.MOHGE_ERR_DEVICE_CHECK      # decoded from the word
+    assert b"index check" in B.lib().mohge_last_error()
     assert int(b.counts.sum()) == 127
+
+
+def test_nan_logits_rank_below_every_number_and_are_reported():
+    """NaN router logits are invalid input: they lose against every number (ties among them to
+    the lowest index), the indices still equal the oracle's under that reading bit for bit, and
+    the status word says so."""
+    wl = Workload("nan_logits", "f32", 300, 32, 3, 4, (32, 24, 16), 2, 5, seed=4)
+    gcfg, ocfg = gpu_cfg(wl), oracle_cfg(wl)
+    rng = np.random.default_rng(12)
+    lg = rng.normal(size=(wl.T, wl.n_logits)).astype(np.float32)
+    nan_at = rng.random(lg.shape) < 0.15
+    nan_at[0] = True
+    nan_at[1, :3] = True
+    nan_at[2, 3:7] = True
+    lg[nan_at] = np.nan
+    s = O.route_spec(ocfg, lg)
+    assert s["nan_logits"] == int(nan_at.sum())
+    b = B.LayerBuffers(gcfg, wl.T)
+    B.mohge_route(gcfg, wl.T, None, None, None, torch.from_numpy(lg).cuda(), None, b.group_idx,
+                  b.expert_idx, b.gate_w, b.gs, b.esp, b.ws)
+    torch.cuda.synchronize()
+    assert (b.group_idx.cpu().numpy() == s["group_idx"]).all()
+    assert (b.expert_idx.cpu().numpy() == s["expert_idx"]).all()
+    ok = ~nan_at[:, :3].any(axis=1)                      # tokens whose group logits are numbers
+    assert (b.gate_w.cpu().numpy()[ok] == s["gate"][ok]).all()
+    rc, word = B.mohge_get_device_status_rc(b.ws)
+    assert word == 3 << 24 and rc == B.MOHGE_ERR_DEVICE_CHECK
+    assert b"NaN" in B.lib().mohge_last_error()
+    # a batch without NaN leaves the word alone
+    B.mohge_workspace_init(gcfg, wl.T, b.ws)
+    B.mohge_route(gcfg, wl.T, None, None, None, torch.from_numpy(np.nan_to_num(lg)).cuda(), None,
+                  b.group_idx, b.expert_idx, b.gate_w, b.gs, b.esp, b.ws)
+    torch.cuda.synchronize()
+    assert B.mohge_get_device_status_rc(b.ws) == (0, 0)
+
+
+def test_tensor_maps_are_encoded_once_per_launch_site():
+    """A layer stepped on the same buffers encodes its TMA tensor maps on the first step only."""
+    wl = Workload("map_cache", "bf16", 700, 256, 3, 4, (352, 176, 88), 2, 4, seed=3)
+    inp = make_inputs(wl)
+    gcfg = gpu_cfg(wl)
+    dev = {k: (v.cuda() if isinstance(v, torch.Tensor) else v) for k, v in inp.items() if k not in ("w13", "w2")}
+    w13, w2 = [w.cuda() for w in inp["w13"]], [w.cuda() for w in inp["w2"]]
+    b = B.LayerBuffers(gcfg, wl.T)
+
+    def step():
+        B.layer_forward(gcfg, b, dev["x"], dev["w_router"], w13, w2, aux=True)
+        B.layer_backward(gcfg, b, dev["x"], dev["w_router"], w13, w2, dev["dy"], aux=True)
+
+    step()
+    h0, m0 = B.mohge_map_cache_stats()
+    step()
+    step()
+    torch.cuda.synchronize()
+    h1, m1 = B.mohge_map_cache_stats()
+    assert m1 == m0                                     # no new encodes
+    assert h1 - h0 == 2 * 9                             # nine tensor-core GEMM launches per step
+    y = b.y.clone()
+    step()
+    torch.cuda.synchronize()
+    assert torch.equal(y, b.y) and B.mohge_get_device_status(b.ws) == 0
+
+
+@pytest.mark.skipif(not torch.cuda.is_available() or torch.cuda.device_count() < 2,
+                    reason="needs two visible GPUs")
+def test_layer_on_a_second_device_of_the_same_process():
+    """Kernel attributes, SM count and cached tensor maps are kept per device ordinal: a process
+    that has already used device 0 runs the same layer on device 1 and gets the same bits."""
+    wl = Workload("second_device", "bf16", 600, 256, 3, 4, (352, 176, 88), 2, 4, seed=6)
+    inp = make_inputs(wl)
+    gcfg = gpu_cfg(wl)
+    outs = []
+    for ordinal in (0, 1):
+        with torch.cuda.device(ordinal):
+            d = torch.device("cuda", ordinal)
+            x, w_r, dy = inp["x"].to(d), inp["w_router"].to(d), inp["dy"].to(d)
+            w13, w2 = [w.to(d) for w in inp["w13"]], [w.to(d) for w in inp["w2"]]
+            b = B.LayerBuffers(gcfg, wl.T, device=d)
+            B.layer_forward(gcfg, b, x, w_r, w13, w2, aux=True)
+            B.layer_backward(gcfg, b, x, w_r, w13, w2, dy, aux=True)
+            torch.cuda.synchronize()
+            assert B.mohge_get_device_status(b.ws) == 0
+            outs.append((b.y.cpu(), b.dx.cpu(), b.dw13[0].cpu()))
+    for a, c in zip(*outs):
+        assert torch.equal(a, c)
 
 
 @pytest.mark.parametrize("switch", ["MOHGE_TC_CG=2,MOHGE_TC_WIDE=63", "MOHGE_TC_CG=2,MOHGE_TC_WIDE=0",
                                     "MOHGE_TC_CG=1", "MOHGE_PDL=0", "MOHGE_FORCE_SIMT=1"])
-def test_every_form_of_the_grouped_gemm_on_small_ragged_cases(switch, monkeypatch):
+def test_every_form_of_the_grouped_gemm_on_small_ragged_cases(switch):
     """The double-width form is chosen by default only for long contractions (the large
     workload) and single CTAs only for batches with few rows per expert, and the GEMM kernels are
     launched as programmatic dependents of their predecessors unless switched off; here each form is forced
     on small ragged shapes, so that every kernel form meets odd widths, ragged tails, empty experts
     and both a few and a few hundred rows per expert."""
-    for kv in switch.split(","):
-        name, value = kv.split("=")
-        monkeypatch.setenv(name, value)
-    for wl in (Workload("forms_a", "bf16", 1000, 256, 3, 4, (352, 176, 88), 2, 4, seed=1),
-               Workload("forms_few", "bf16", 90, 256, 3, 4, (352, 176, 88), 2, 4, seed=2),
-               Workload("forms_b", "bf16", 1500, 256, 4, 8, (256, 192, 128, 64), 2, 6,
-                        zipf_beta=3.0, seed=5)):
-        inp = make_inputs(wl)
-        _, _, logits32 = oracle_layer(wl, inp)
-        _compare(wl, inp, logits32)
+    with forced_switches(switch):
+        for wl in (Workload("forms_a", "bf16", 1000, 256, 3, 4, (352, 176, 88), 2, 4, seed=1),
+                   Workload("forms_few", "bf16", 90, 256, 3, 4, (352, 176, 88), 2, 4, seed=2),
+                   Workload("forms_b", "bf16", 1500, 256, 4, 8, (256, 192, 128, 64), 2, 6,
+                            zipf_beta=3.0, seed=5)):
+            inp = make_inputs(wl)
+            _, _, logits32 = oracle_layer(wl, inp)
+            _compare(wl, inp, logits32)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])

@@ -9,7 +9,10 @@ full for all T tokens.  Floating-point results are compared
     row of a random sample of tokens (y, dx, gate and logit gradients, the permuted
     intermediates of their routed copies), every row and both weight gradients of whole sampled
     experts (narrowest and widest group), and the statistics of all tokens.
-Bars: bit-exact integers given identical float32 logits; max|a-b|/max|b| <= 2e-2 for BF16.
+Bars: bit-exact integers given identical float32 logits; max|a-b|/max|b| <= 2e-2 for BF16, per
+tensor and, for the weight gradients, per expert (a cold expert's gradient is much smaller than
+a hot one's of the same group).  A second, element-wise figure is printed beside it (run pytest
+with -s to see it): the share of elements with |a-b| > tol |b| + tol rms(b).
 """
 import numpy as np
 import pytest
@@ -19,14 +22,14 @@ import oracle as O
 from paper_2604_23108_b200 import binding as B
 from paper_2604_23108_b200.inputs import WORKLOADS, make_device_inputs
 
-from _util import gpu_cfg, max_rel, oracle_cfg, to_np64
+from _util import elementwise_outliers, gpu_cfg, max_rel, oracle_cfg, to_np64
 
 pytestmark = pytest.mark.gpu
 
 TOL = 2e-2
 FULL_ORACLE = {"cfg2_bf16": True, "cfg3_bf16_aux": True, "cfg4_bf16_skew": True,
                "cfg5_bf16_large": False, "paper_3b_layer": True, "paper_14b_layer": True,
-               "decode_256_large": False}
+               "decode_256_large": False, "cfg5_slice": False}
 N_SAMPLE_TOKENS = 48
 
 
@@ -43,6 +46,13 @@ def _run_gpu(wl):
     torch.cuda.synchronize()
     assert B.mohge_get_device_status(b.ws) == 0
     return gcfg, inp, b
+
+
+def _close(name, what, got, want, tol=TOL):
+    """The bar (max|a-b| / max|b| <= tol) plus the element-wise figure, which is only reported."""
+    m = max_rel(got, want)
+    print("%s %s: max_rel %.2e, element-wise outliers %.2e" % (name, what, m, elementwise_outliers(got, want, tol)))
+    assert m <= tol, (name, what, m)
 
 
 @pytest.mark.parametrize("name", list(FULL_ORACLE))
@@ -70,8 +80,10 @@ def test_full_size_workload(name):
     assert (b.prow_of.cpu().numpy() == dp["prow_of"]).all()
     assert (b.src_of.cpu().numpy() == dp["src_of"]).all()
     if wl.zipf_beta:
-        cnt = dp["counts"][dp["counts"] > 0]
-        assert cnt.max() / cnt.min() > 30          # the skewed workload really is skewed
+        cnt = dp["counts"]
+        ratio = cnt.max() / max(1, cnt.min())      # the skewed workload: counts span about 100x
+        print("%s: per-expert token counts %d..%d, ratio %.0f" % (name, cnt.min(), cnt.max(), ratio))
+        assert 50 <= ratio <= 200
 
     # ---- statistics of all tokens (Eq. 7-14) ----
     v = O.route_values(ocfg, logits32.astype(np.float64), s["group_idx"])
@@ -99,10 +111,10 @@ def test_full_size_workload(name):
     cE = st["cE_lit"] if ocfg.fe_mode == 0 else st["cE_route"]
     bs = O.layer_backward(fs, w13n, w2n, dy_s, with_aux=True, aux_counts=(st["cG"], cE, T))
     tok_t = torch.from_numpy(tok).cuda()
-    assert max_rel(to_np64(b.y[tok_t]), fs["y"]) <= TOL
-    assert max_rel(to_np64(b.dx[tok_t]), bs["dx"]) <= TOL
-    assert max_rel(to_np64(b.dgate[tok_t]), bs["dgate"]) <= TOL
-    assert max_rel(to_np64(b.dlogits[tok_t]), bs["dlogits"]) <= TOL
+    _close(name, "y (sampled tokens)", to_np64(b.y[tok_t]), fs["y"])
+    _close(name, "dx (sampled tokens)", to_np64(b.dx[tok_t]), bs["dx"])
+    _close(name, "dgate (sampled tokens)", to_np64(b.dgate[tok_t]), bs["dgate"])
+    _close(name, "dlogits (sampled tokens)", to_np64(b.dlogits[tok_t]), bs["dlogits"])
     for e, c in fs["per_expert"].items():            # routed copies of the sampled tokens
         W = wl.group_width[e // N]
         rows = torch.from_numpy(prow_of[tok[c["t"]], c["k"]].astype(np.int64)).cuda()
@@ -136,8 +148,8 @@ def test_full_size_workload(name):
         dau = to_np64(b.dau[r0:r0 + n])
         assert max_rel(dau[:, :W], eb["dA"]) <= TOL and max_rel(dau[:, W:2 * W], eb["dU"]) <= TOL
         assert max_rel(to_np64(b.dx_perm[r0:r0 + n]), eb["dx"]) <= TOL
-        assert max_rel(to_np64(b.dw13[g][i]), eb["dw13"]) <= TOL
-        assert max_rel(to_np64(b.dw2[g][i]), eb["dw2"]) <= TOL
+        _close(name, "dw13 of expert %d" % e, to_np64(b.dw13[g][i]), eb["dw13"])
+        _close(name, "dw2 of expert %d" % e, to_np64(b.dw2[g][i]), eb["dw2"])
         pad = int(aligned[e + 1]) - r0 - n                               # padding rows stay zero
         if pad:
             assert float(b.x_perm[r0 + n:r0 + n + pad].abs().max()) == 0.0
@@ -148,6 +160,14 @@ def test_full_size_workload(name):
         ff = O.layer_forward(ocfg, to_np64(x_cpu), w_r, w13n, w2n, logits=logits32.astype(np.float64),
                              mode="spec")
         assert max_rel(to_np64(b.y), ff["y"]) <= TOL
+    # ---- router weight gradient, all tokens: dW_r = dlogits^T x in fp64 from the GPU's own
+    # dlogits (checked against the oracle on the sampled tokens above and, where the full oracle
+    # runs, in full below); this pins the split-K sum over the tokens at every batch size ----
+    dl = to_np64(b.dlogits)
+    dw_r = np.zeros((wl.n_logits, wl.d_model))
+    for t0 in range(0, T, 8192):
+        dw_r += dl[t0:t0 + 8192].T @ to_np64(x_cpu[t0:t0 + 8192])
+    _close(name, "dw_router (from the GPU's dlogits)", to_np64(b.dw_router), dw_r)
     if not FULL_ORACLE[name]:
         return
     # ---- every element against the full oracle ----
@@ -156,11 +176,15 @@ def test_full_size_workload(name):
     fwd = O.layer_forward(ocfg, to_np64(x_cpu), w_r, w13d, w2d, logits=logits32.astype(np.float64),
                           mode="spec")
     bwd = O.layer_backward(fwd, w13d, w2d, to_np64(dy_cpu), with_aux=True)
-    assert max_rel(to_np64(b.y), fwd["y"]) <= TOL
-    assert max_rel(to_np64(b.dx), bwd["dx"]) <= TOL
-    assert max_rel(to_np64(b.dgate), bwd["dgate"]) <= TOL
-    assert max_rel(to_np64(b.dlogits), bwd["dlogits"]) <= TOL
-    assert max_rel(to_np64(b.dw_router), bwd["dw_r"]) <= TOL
+    _close(name, "y", to_np64(b.y), fwd["y"])
+    _close(name, "dx", to_np64(b.dx), bwd["dx"])
+    _close(name, "dgate", to_np64(b.dgate), bwd["dgate"])
+    _close(name, "dlogits", to_np64(b.dlogits), bwd["dlogits"])
+    _close(name, "dw_router", to_np64(b.dw_router), bwd["dw_r"])
     for g in range(wl.n_groups):
-        assert max_rel(to_np64(b.dw13[g]), bwd["dw13"][g]) <= TOL, g
-        assert max_rel(to_np64(b.dw2[g]), bwd["dw2"][g]) <= TOL, g
+        dw13, dw2 = to_np64(b.dw13[g]), to_np64(b.dw2[g])
+        assert max_rel(dw13, bwd["dw13"][g]) <= TOL, g
+        assert max_rel(dw2, bwd["dw2"][g]) <= TOL, g
+        for i in range(N):                           # per expert: cold experts have small gradients
+            assert max_rel(dw13[i], bwd["dw13"][g][i]) <= TOL, (g, i)
+            assert max_rel(dw2[i], bwd["dw2"][g][i]) <= TOL, (g, i)

@@ -12,7 +12,7 @@ import oracle as O
 from paper_2604_23108_b200 import binding as B
 from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_inputs
 
-from _util import gpu_cfg, gpu_layer, max_rel, oracle_cfg, oracle_layer, to_np64, tol_for
+from _util import forced_switches, gpu_cfg, gpu_layer, max_rel, oracle_cfg, oracle_layer, to_np64, tol_for
 
 pytestmark = pytest.mark.gpu
 
@@ -160,22 +160,20 @@ def test_deterministic_rerun(case):
 
 @pytest.mark.parametrize("switch", ["", "MOHGE_TC_CG=1", "MOHGE_TC_CG=2,MOHGE_TC_WIDE=63",
                                     "MOHGE_FORCE_SIMT=1"])
-def test_accumulate_adds_into_weight_gradients(switch, monkeypatch):
+def test_accumulate_adds_into_weight_gradients(switch):
     """accumulate = 1 adds the weight gradients into dw13 / dw2 (TMA reduce-add in the tensor-core
     forms, read-modify-write in the FFMA kernel); checked in every form of the grouped GEMM."""
-    for kv in filter(None, switch.split(",")):
-        name, value = kv.split("=")
-        monkeypatch.setenv(name, value)
     wl = CASES["bf16_small"]
     inp = make_inputs(wl)
     _, _, logits32 = oracle_layer(wl, inp)
-    b, dev = gpu_layer(wl, inp, logits32=logits32)
-    gcfg = gpu_cfg(wl)
-    ref13 = [t.clone() for t in b.dw13]
-    ref2 = [t.clone() for t in b.dw2]
-    B.layer_backward(gcfg, b, dev["x"], dev["w_router"], dev["w13"], dev["w2"], dev["dy"],
-                     aux=True, accumulate=True)
-    torch.cuda.synchronize()
+    with forced_switches(switch):
+        b, dev = gpu_layer(wl, inp, logits32=logits32)
+        gcfg = gpu_cfg(wl)
+        ref13 = [t.clone() for t in b.dw13]
+        ref2 = [t.clone() for t in b.dw2]
+        B.layer_backward(gcfg, b, dev["x"], dev["w_router"], dev["w13"], dev["w2"], dev["dy"],
+                         aux=True, accumulate=True)
+        torch.cuda.synchronize()
     for g in range(wl.n_groups):
         assert max_rel(to_np64(b.dw13[g]), 2 * to_np64(ref13[g])) <= 1e-6
         assert max_rel(to_np64(b.dw2[g]), 2 * to_np64(ref2[g])) <= 1e-6

@@ -198,3 +198,37 @@ def test_spec_tie_breaks_and_group_order():
     assert list(s["group_idx"][2]) == [0, 1]
     assert list(s["expert_idx"][0]) == [0, 1, 2, 3, 4]
     assert list(s["expert_idx"][1]) == [4, 5, 6, 7, 8]
+
+
+def test_nan_logits_rank_below_every_number():
+    """Reading of Eq. 2-5 for NaN scores (the paper orders real numbers only): a NaN logit loses
+    against every number, ties among NaNs go to the lowest index, and the entries are counted.
+    Pinned without route_spec's own arithmetic: the selections must equal those of the same
+    logits with every NaN replaced by a number far below all others, and an all-NaN token must
+    select what the all-equal (zero) token selects."""
+    cfg = O.OracleConfig(d_model=8, n_groups=3, experts_per_group=4, k_groups=2, k_experts=5,
+                         group_width=[8, 8, 8])
+    rng = np.random.default_rng(5)
+    lg = rng.normal(size=(64, 3 + 12)).astype(np.float32)
+    nan_at = rng.random(lg.shape) < 0.2
+    nan_at[0] = True                                   # one token with nothing but NaN
+    nan_at[1, :3] = True                               # all group logits NaN
+    nan_at[2, 3:7] = True                              # a whole group of expert logits NaN
+    with_nan = np.where(nan_at, np.nan, lg).astype(np.float32)
+    very_low = np.where(nan_at, -1e30, lg).astype(np.float32)
+    a, b = O.route_spec(cfg, with_nan), O.route_spec(cfg, very_low)
+    assert a["nan_logits"] == int(nan_at.sum()) and b["nan_logits"] == 0
+    assert (a["group_idx"] == b["group_idx"]).all() and (a["expert_idx"] == b["expert_idx"]).all()
+    zero = O.route_spec(cfg, np.zeros((1, 15), np.float32))
+    assert (a["group_idx"][0] == zero["group_idx"][0]).all()
+    assert (a["expert_idx"][0] == zero["expert_idx"][0]).all()
+    # gates stay a convex combination wherever the chosen groups have numbers for logits (a NaN
+    # group logit has sigmoid 0, so a token whose chosen groups are all NaN has only zero keys)
+    ok = ~nan_at[:, :3].any(axis=1)
+    assert np.isfinite(a["gate"][ok]).all() and np.allclose(a["gate"][ok].sum(axis=1), 1.0, atol=1e-6)
+    # a NaN expert is only ever picked when fewer than K_e numbers are on offer in the chosen groups
+    picked_nan = np.take_along_axis(nan_at[:, 3:], a["expert_idx"].astype(np.int64), axis=1)
+    for t in np.nonzero(ok)[0]:
+        chosen = a["group_idx"][t]
+        numbers = sum(int((~nan_at[t, 3 + 4 * g:3 + 4 * g + 4]).sum()) for g in chosen)
+        assert int(picked_nan[t].sum()) == max(0, cfg.k_experts - numbers)
