@@ -35,8 +35,12 @@ from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs
 # figure is the capture of "cfg5_slice" (one eighth of the experts, the same tokens per expert,
 # widths and tile forms) times eight: every expert's tiles are independent problems, so the traffic
 # grows with the number of experts.  None: no capture of the current kernels.
-NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": None}
-NCU_DRAM_TRAFFIC_SOURCE = {}
+NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 8 * 8.994e9, "cfg5_slice": 8.994e9}
+NCU_DRAM_TRAFFIC_SOURCE = {
+    "cfg5_bf16_large": "ncu counters of the six launches at cfg5_slice (one eighth of the experts, same tokens per "
+                       "expert, widths and tile forms) times 8; not measured in this run",
+    "cfg5_slice": "ncu counters of the six launches of one step; not measured in this run",
+}
 
 METRIC = "MoHGE layer fwd+bwd tokens/s"
 METRIC_FWD = "MoHGE layer fwd tokens/s"
