@@ -24,6 +24,11 @@
 //
 // Slot layout inside a warp: group g owns P = next_pow2(N) consecutive slots, slot s = g*P + i
 // lives in lane s % 32, register s / 32; a group never straddles a register because P | 32.
+// Only the K_g selected groups take part in Eq. 3-5 (experts of the others can never be picked,
+// their ES' is 0), so the selection and the router backward work on a COMPACT layout: the
+// selected groups in ascending order, slot c = (rank of the group among the selected) * P + i,
+// K_g * P slots instead of N_g * P.  Expert ids stay ascending in c, so ties still go to the
+// lowest expert id.
 
 #include "common.cuh"
 
@@ -107,7 +112,24 @@ struct RouterShape {
   int T, Ng, N, P, logP, NL, Ne, Kg, Ke;
 };
 
-template <int J>
+// Compact slot c of a token whose selected groups are the set bits of gmask: the group (the
+// (c >> logP)-th set bit, ascending), the expert inside it, the flat expert id; valid = false for
+// slots past the K_g selected groups or past the N experts of a group.
+struct CompactSlot {
+  int g, i, e;
+  bool valid;
+};
+__device__ __forceinline__ CompactSlot compact_slot(const RouterShape& s, unsigned gmask, int c) {
+  CompactSlot q;
+  const int rank = c >> s.logP;
+  q.i = c & (s.P - 1);
+  q.valid = rank < s.Kg && q.i < s.N;
+  q.g = q.valid ? (int)__fns(gmask, 0, rank + 1) : 0;      // position of the (rank + 1)-th set bit
+  q.e = q.g * s.N + q.i;
+  return q;
+}
+
+template <int J, int JC>
 __global__ void __launch_bounds__(256)
 router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* __restrict__ group_idx,
                      int32_t* __restrict__ expert_idx, float* __restrict__ gate_w,
@@ -142,38 +164,38 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
     }
     const float gsv = lane < s.Ng ? sig_s(clean(L[lane])) : 0.0f;      // GS of group `lane`
     if (lane < s.Ng) gs_saved[(size_t)t * s.Ng + lane] = gsv;
-    // ---- Eq. 3, 4: keys of the lane's slots ----
-    float key[J];
-    int eid[J];
+    // ES' of the experts of unselected groups is 0 (Eq. 3)
 #pragma unroll
     for (int j = 0; j < J; ++j) {
       const int sl = lane + 32 * j;
-      const int g = sl >> s.logP;
-      const int i = sl & (s.P - 1);
-      const bool valid = g < s.Ng && i < s.N;
-      const int e = g * s.N + i;
-      const float l = valid ? clean(L[s.Ng + e]) : -INFINITY;
+      const int g = sl >> s.logP, i = sl & (s.P - 1);
+      if (g < s.Ng && i < s.N && !((gmask >> g) & 1u)) esp_saved[(size_t)t * s.Ne + g * s.N + i] = 0.0f;
+    }
+    // ---- Eq. 3, 4: keys of the lane's compact slots (selected groups only) ----
+    float key[JC];
+    int eid[JC];
+#pragma unroll
+    for (int j = 0; j < JC; ++j) {
+      const CompactSlot q = compact_slot(s, gmask, lane + 32 * j);
+      const float l = q.valid ? clean(L[s.Ng + q.e]) : -INFINITY;
       float m = l;
       for (int mask = s.P >> 1; mask > 0; mask >>= 1) m = fmaxf(m, __shfl_xor_sync(kFull, m, mask));
-      const float p = valid ? exp_s(__fsub_rn(l, m)) : 0.0f;
+      const float p = q.valid ? exp_s(__fsub_rn(l, m)) : 0.0f;
       float S = p;
       for (int mask = 1; mask < s.P; mask <<= 1) S = __fadd_rn(S, __shfl_xor_sync(kFull, S, mask));
-      const bool sel = valid && ((gmask >> g) & 1u);
-      const float sg = __shfl_sync(kFull, gsv, g & 31);           // GS of this slot's group
-      float kv = valid ? -1.0f : -2.0f;
-      float ev = 0.0f;
-      if (sel) {
+      const float sg = __shfl_sync(kFull, gsv, q.g & 31);          // GS of this slot's group
+      float kv = -2.0f;
+      if (q.valid) {
         kv = __fmul_rn(p, __fdiv_rn(sg, S));
-        ev = __fdiv_rn(p, S);
+        esp_saved[(size_t)t * s.Ne + q.e] = __fdiv_rn(p, S);
       }
       key[j] = kv;
-      eid[j] = valid ? e : (0x7ffffff0 + j);
-      if (valid) esp_saved[(size_t)t * s.Ne + e] = ev;
+      eid[j] = q.valid ? q.e : (0x7ffffff0 + j);
     }
     // ---- Eq. 5: top-K_e experts, Eq. 6: normalise ----
     int we;
     float wk;
-    warp_topk<J>(key, eid, s.Ke, lane, we, wk);
+    warp_topk<JC>(key, eid, s.Ke, lane, we, wk);
     float sum = __shfl_sync(kFull, wk, 0);
     for (int k = 1; k < s.Ke; ++k) sum = __fadd_rn(sum, __shfl_sync(kFull, wk, k));
     if (lane < s.Ke) {
@@ -200,7 +222,7 @@ __global__ void zero_counts_kernel(int32_t* group_count, int Ng, int32_t* cnt_ro
 constexpr int kStatsThreads = 512;
 constexpr int kStatsWarps = kStatsThreads / 32;
 
-template <int J>
+template <int J, int JC>
 __global__ void __launch_bounds__(kStatsThreads)
 aux_stats_kernel(RouterShape s, float eps, const float* __restrict__ gs, const float* __restrict__ esp,
                  const int32_t* __restrict__ group_idx, const int32_t* __restrict__ expert_idx,
@@ -234,27 +256,30 @@ aux_stats_kernel(RouterShape s, float eps, const float* __restrict__ gs, const f
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) gsum += __shfl_xor_sync(kFull, gsum, off);
     if (lane < s.Ng) accG += (double)(gv / gsum);
-    // Eq. 14 and the Eq. 12 indicator
-    float key[J];
-    int eid[J];
+    // Eq. 14: S_e = ES'_e / (sum over the group + eps); ES' of unselected groups is 0
 #pragma unroll
     for (int j = 0; j < J; ++j) {
       const int sl = lane + 32 * j;
       const int g = sl >> s.logP;
       const int i = sl & (s.P - 1);
       const bool valid = g < s.Ng && i < s.N;
-      const int e = g * s.N + i;
-      const float ev = valid ? esp[(size_t)t * s.Ne + e] : 0.0f;
+      const float ev = valid ? esp[(size_t)t * s.Ne + g * s.N + i] : 0.0f;
       float grp = ev;
       for (int mask = 1; mask < s.P; mask <<= 1) grp += __shfl_xor_sync(kFull, grp, mask);
       if (valid) accE[j] += (double)(ev / (grp + eps));
-      const bool sel = valid && ((gmask >> g) & 1u);
-      key[j] = sel ? ev : (valid ? -1.0f : -2.0f);
-      eid[j] = valid ? e : (0x7ffffff0 + j);
+    }
+    // Eq. 12 indicator: top-K_e of ES' over the experts of the selected groups (compact slots)
+    float key[JC];
+    int eid[JC];
+#pragma unroll
+    for (int j = 0; j < JC; ++j) {
+      const CompactSlot q = compact_slot(s, gmask, lane + 32 * j);
+      key[j] = q.valid ? esp[(size_t)t * s.Ne + q.e] : -2.0f;
+      eid[j] = q.valid ? q.e : (0x7ffffff0 + j);
     }
     int we;
     float wk;
-    warp_topk<J>(key, eid, s.Ke, lane, we, wk);
+    warp_topk<JC>(key, eid, s.Ke, lane, we, wk);
     if (lane < s.Ke) atomicAdd(&s_cl[we], 1);
   }
   // fixed-order reduction over the warps of the block, then one partial row per block
@@ -341,7 +366,7 @@ struct BwdParams {
 
 constexpr int kBwdWarps = 8;
 
-template <int J>
+template <int J, int JC>
 __global__ void __launch_bounds__(kBwdWarps * 32)
 router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
                   const float* __restrict__ gs, const float* __restrict__ esp,
@@ -376,20 +401,29 @@ router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
     __syncwarp();
     if (lane < s.Ke) s_dkey[warp][ek] = (dgk - dot) / ssum;
     __syncwarp();
-    // Eq. 4, 3 backward on the lane's slots
+    // experts of unselected groups: ES' is the constant 0, so no gradient reaches their logits
 #pragma unroll
     for (int j = 0; j < J; ++j) {
       const int sl = lane + 32 * j;
-      const int g = sl >> s.logP;
-      const int i = sl & (s.P - 1);
-      const bool valid = g < s.Ng && i < s.N;
-      const int e = g * s.N + i;
+      const int g = sl >> s.logP, i = sl & (s.P - 1);
+      if (g < s.Ng && i < s.N && !((gmask >> g) & 1u)) {
+        dlogits[(size_t)t * s.NL + s.Ng + g * s.N + i] = 0.0f;
+        if (dl16) dl16[(size_t)t * dl16_pitch + s.Ng + g * s.N + i] = __float2bfloat16(0.0f);
+      }
+    }
+    if (lane < s.Ng) s_dgs[warp][lane] = 0.0f;
+    __syncwarp();
+    // Eq. 4, 3 backward on the lane's compact slots (selected groups)
+#pragma unroll
+    for (int j = 0; j < JC; ++j) {
+      const CompactSlot q = compact_slot(s, gmask, lane + 32 * j);
+      const bool valid = q.valid;
+      const int e = q.e, g = q.g;
       const float ev = valid ? esp[(size_t)t * s.Ne + e] : 0.0f;
       const float gv = valid ? gs[(size_t)t * s.Ng + g] : 0.0f;
       const float dpp = valid ? s_dkey[warp][e] : 0.0f;
       float dgs = dpp * ev;                 // dGS_g = sum_i dES''_i ES'_i
       float desp = dpp * gv;                // dES'_i = dES''_i GS_g
-      const bool sel = valid && ((gmask >> g) & 1u);
       if (bp.with_aux) {
         // L_E: S_e = ES'_e / D, D = sum_j ES'_j + eps (selected groups only; ES' is the constant 0 elsewhere)
         const float fe = valid ? (float)s.N / s.Ke * (float)expert_count[e] * fn : 0.0f;
@@ -399,7 +433,7 @@ router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
           fes += __shfl_xor_sync(kFull, fes, mask);
         }
         const float Dn = grp + bp.eps;
-        if (sel) desp += bp.alpha_e * invT * (fe / Dn - fes / (Dn * Dn));
+        if (valid) desp += bp.alpha_e * invT * (fe / Dn - fes / (Dn * Dn));
       }
       float inner = ev * desp;
       for (int mask = 1; mask < s.P; mask <<= 1) {
@@ -411,7 +445,7 @@ router_bwd_kernel(RouterShape s, BwdParams bp, const float* __restrict__ dgate,
         dlogits[(size_t)t * s.NL + s.Ng + e] = dl;
         if (dl16) dl16[(size_t)t * dl16_pitch + s.Ng + e] = __float2bfloat16(dl);
       }
-      if (valid && i == 0) s_dgs[warp][g] = dgs;
+      if (valid && q.i == 0) s_dgs[warp][g] = dgs;
     }
     __syncwarp();
     // Eq. 2 backward (+ L_G through Eq. 10)
@@ -452,15 +486,29 @@ int slots_per_lane(const Dims& D) {
   while (J * 32 < slots) J *= 2;
   return J;
 }
+int compact_slots_per_lane(const Dims& D) {     // K_g selected groups of P slots each
+  const int slots = D.Kg * D.P;
+  int J = 1;
+  while (J * 32 < slots) J *= 2;
+  return J;
+}
 
 }  // namespace
 
-#define MOHGE_DISPATCH_J(J_, ...)                      \
-  switch (J_) {                                        \
-    case 1: { constexpr int JJ = 1; __VA_ARGS__; } break; \
-    case 2: { constexpr int JJ = 2; __VA_ARGS__; } break; \
-    case 4: { constexpr int JJ = 4; __VA_ARGS__; } break; \
-    default: { constexpr int JJ = 8; __VA_ARGS__; } break; \
+// JJ = registers per lane of the full slot layout, JC = of the compact one (JC <= JJ)
+#define MOHGE_DISPATCH_JC(JJ_, JC_, ...)                   \
+  switch (JC_) {                                           \
+    case 1: { constexpr int JJ = JJ_, JC = 1; __VA_ARGS__; } break; \
+    case 2: { constexpr int JJ = JJ_, JC = JJ_ < 2 ? JJ_ : 2; __VA_ARGS__; } break; \
+    case 4: { constexpr int JJ = JJ_, JC = JJ_ < 4 ? JJ_ : 4; __VA_ARGS__; } break; \
+    default: { constexpr int JJ = JJ_, JC = JJ_; __VA_ARGS__; } break; \
+  }
+#define MOHGE_DISPATCH_J(D_, ...)                                          \
+  switch (slots_per_lane(D_)) {                                            \
+    case 1: MOHGE_DISPATCH_JC(1, compact_slots_per_lane(D_), __VA_ARGS__); break; \
+    case 2: MOHGE_DISPATCH_JC(2, compact_slots_per_lane(D_), __VA_ARGS__); break; \
+    case 4: MOHGE_DISPATCH_JC(4, compact_slots_per_lane(D_), __VA_ARGS__); break; \
+    default: MOHGE_DISPATCH_JC(8, compact_slots_per_lane(D_), __VA_ARGS__); break; \
   }
 
 int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_idx,
@@ -469,7 +517,7 @@ int32_t launch_router_select(const Dims& D, const float* logits, int32_t* group_
   if (D.T == 0) return MOHGE_OK;
   const RouterShape s = make_shape(D);
   const int blocks = (int)((D.T + 7) / 8) < 148 * 8 ? (int)((D.T + 7) / 8) : 148 * 8;
-  MOHGE_DISPATCH_J(slots_per_lane(D), (launch_dep(router_select_kernel<JJ>, dim3(blocks), dim3(256), st,
+  MOHGE_DISPATCH_J(D, (launch_dep(router_select_kernel<JJ, JC>, dim3(blocks), dim3(256), st,
                                           s, logits, group_idx, expert_idx, gate_w, gs, esp, status)));
   MOHGE_LAUNCH_CHECK("router_select_kernel");
   return MOHGE_OK;
@@ -485,8 +533,8 @@ int32_t launch_aux_stats(const Dims& D, const mohge_config& cfg, const float* gs
   int blocks = ceil_div(D.T, kStatsWarps);
   if (blocks > kStatsBlocks) blocks = kStatsBlocks;
   if (blocks > 0) {
-    MOHGE_DISPATCH_J(slots_per_lane(D),
-                     (launch_dep(aux_stats_kernel<JJ>, dim3(blocks), dim3(kStatsThreads), st,
+    MOHGE_DISPATCH_J(D,
+                     (launch_dep(aux_stats_kernel<JJ, JC>, dim3(blocks), dim3(kStatsThreads), st,
                          s, cfg.eps, gs, esp, group_idx, expert_idx, group_count, cnt_routed,
                          cnt_lit, partials)));
     MOHGE_LAUNCH_CHECK("aux_stats_kernel");
@@ -520,8 +568,8 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
     bp.w_over_wmax[g] = g < D.Ng ? (float)D.W[g] / (float)D.Wmax : 0.0f;
   int blocks = ceil_div(D.T, kBwdWarps);
   if (blocks > 148 * 8) blocks = 148 * 8;
-  MOHGE_DISPATCH_J(slots_per_lane(D),
-                   (launch_dep(router_bwd_kernel<JJ>, dim3(blocks), dim3(kBwdWarps * 32), st,
+  MOHGE_DISPATCH_J(D,
+                   (launch_dep(router_bwd_kernel<JJ, JC>, dim3(blocks), dim3(kBwdWarps * 32), st,
                        s, bp, dgate, gs, esp, group_idx, expert_idx, group_count, expert_count,
                        dlogits, dl16, dl16_pitch)));
   MOHGE_LAUNCH_CHECK("router_bwd_kernel");
