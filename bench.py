@@ -449,8 +449,18 @@ def main():
     sampler = ClockSampler(local_rank) if rank == 0 else None
     l0 = B.mohge_launch_count()
     barrier()
-    t_start, t_end = ev(), ev()
+    # host time to enqueue one step, taken on an empty launch queue (inside the timed loop of a
+    # large workload the host mostly waits for room in the queue)
     host_t0 = time.perf_counter()
+    for _ in range(3):
+        if graph is not None:
+            graph.replay()
+        else:
+            step()
+    host_enqueue_ms = (time.perf_counter() - host_t0) * 1e3 / 3
+    barrier()
+    l0 = B.mohge_launch_count()
+    t_start, t_end = ev(), ev()
     t_start.record()
     for _ in range(args.steps):
         if graph is not None:
@@ -458,7 +468,6 @@ def main():
         else:
             step(mark=True)
     t_end.record()
-    host_enqueue_ms = (time.perf_counter() - host_t0) * 1e3 / args.steps   # host time to enqueue a step
     barrier()
     launches = launches_per_replay * args.steps if graph is not None else B.mohge_launch_count() - l0
     clocks = sampler.stop() if sampler else None
