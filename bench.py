@@ -204,7 +204,7 @@ def flops_per_step(wl: Workload, counts, shared_width: int = 0) -> float:
     return 18.0 * wl.d_model * tot
 
 
-def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=False):
+def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=False, gather=False):
     """One pass of the whole hot path through the C ABI.  Returns (step, gemm_marks): with
     mark=True a step records CUDA events around mohge_expert_fwd and mohge_expert_bwd_dgate."""
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -217,13 +217,21 @@ def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=Fa
                       buf.group_idx, buf.expert_idx, buf.gate_w, buf.gs, buf.esp, buf.ws)
         B.mohge_aux_stats(gcfg, T, buf.gs, buf.esp, buf.group_idx, buf.expert_idx, buf.group_count,
                           buf.group_psum, buf.cnt_routed, buf.cnt_lit, buf.expert_psum, buf.loss, buf.ws)
-        B.mohge_dispatch(gcfg, T, inp["x"], buf.expert_idx, buf.counts, buf.offsets, buf.aligned,
-                         buf.row_of, buf.prow_of, buf.src_of, buf.x_perm, buf.ws)
+        if gather:      # no x_perm: the GEMMs gather the rows of x
+            B.mohge_dispatch_indices(gcfg, T, buf.expert_idx, buf.counts, buf.offsets, buf.aligned,
+                                     buf.row_of, buf.prow_of, buf.src_of, buf.tok_of_prow, buf.ws)
+        else:
+            B.mohge_dispatch(gcfg, T, inp["x"], buf.expert_idx, buf.counts, buf.offsets, buf.aligned,
+                             buf.row_of, buf.prow_of, buf.src_of, buf.x_perm, buf.ws)
         if mark:
             e0, e1, e2, e3 = ev(), ev(), ev(), ev()
             e0.record()
-        B.mohge_expert_fwd(gcfg, T, buf.x_perm, buf.counts, buf.aligned, inp["w13"], inp["w2"],
-                           buf.au, buf.h, buf.y_perm, buf.ws)
+        if gather:
+            B.mohge_expert_fwd_gather(gcfg, T, inp["x"], buf.tok_of_prow, buf.counts, buf.aligned, inp["w13"],
+                                      inp["w2"], buf.au, buf.h, buf.y_perm, buf.ws)
+        else:
+            B.mohge_expert_fwd(gcfg, T, buf.x_perm, buf.counts, buf.aligned, inp["w13"], inp["w2"],
+                               buf.au, buf.h, buf.y_perm, buf.ws)
         if shared is not None:
             B.mohge_shared_fwd(gcfg, T, shared_width, inp["x"], shared[0], shared[1], buf.au_sh,
                                buf.h_sh, buf.y_sh, buf.ws)
@@ -244,10 +252,16 @@ def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=Fa
                             buf.aligned, buf.dy_perm, None)
         if mark:
             e2.record()
-        B.mohge_expert_bwd_dgate(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts,
-                                 buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13,
-                                 buf.dw2, 0, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate,
-                                 buf.ws)
+        if gather:
+            B.mohge_expert_bwd_gather(gcfg, T, buf.dy_perm, inp["x"], buf.tok_of_prow, buf.au, buf.h, buf.counts,
+                                      buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13,
+                                      buf.dw2, 0, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate,
+                                      buf.ws)
+        else:
+            B.mohge_expert_bwd_dgate(gcfg, T, buf.dy_perm, buf.x_perm, buf.au, buf.h, buf.counts,
+                                     buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13,
+                                     buf.dw2, 0, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate,
+                                     buf.ws)
         if shared is not None:
             B.mohge_shared_bwd(gcfg, T, shared_width, inp["dy"], inp["x"], buf.au_sh, buf.h_sh,
                                shared[0], shared[1], buf.dau_sh, buf.dx_sh, buf.dw13_sh, buf.dw2_sh,
@@ -378,6 +392,9 @@ def main():
     ap.add_argument("--shared-width", type=int, default=0,
                     help="hidden width of the shared experts (N_s FFNs concatenated); 0 = none, "
                          "the benchmark configurations have none")
+    ap.add_argument("--gather", action="store_true",
+                    help="time the route that never writes x_perm (mohge_dispatch_indices, "
+                         "mohge_expert_fwd_gather, mohge_expert_bwd_gather); BF16 workloads only")
     ap.add_argument("--graph", action="store_true",
                     help="capture one step in a CUDA graph and time its replays (launch-bound small "
                          "workloads); the GEMM share for the roofline object is then taken from a "
@@ -416,7 +433,8 @@ def main():
         shared = make_shared_weights(wl, args.shared_width, device=dev, seed=replica_seed(wl, rank))
     T = wl.T
     ev = lambda: torch.cuda.Event(enable_timing=True)
-    step, gemm_marks = make_step(B, gcfg, T, inp, buf, shared, args.shared_width, args.forward_only)
+    step, gemm_marks = make_step(B, gcfg, T, inp, buf, shared, args.shared_width, args.forward_only,
+                                 args.gather)
 
     def barrier():
         if dist is not None:
@@ -579,7 +597,7 @@ def main():
     # ---- outside the timed region: every HBM-bound entry point on its own, then short runs of the
     # other benchmark workloads (default line only) ----
     hbm_steps, others = None, None
-    if not args.no_extras and world == 1 and not args.forward_only and not args.shared_width:
+    if not args.no_extras and world == 1 and not args.forward_only and not args.shared_width and not args.gather:
         hbm_steps = hbm_step_rooflines(B, gcfg, wl, inp, buf, pk["hbm"])
         if args.workload == DEFAULT_WORKLOAD:
             others = [quick_workload_line(B, n, dev, pk) for n in
@@ -624,7 +642,8 @@ def main():
                    "pass": "forward only" if args.forward_only else "forward + backward",
                    "count_ratio": count_ratio(counts),
                    "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only",
-                   "launch": "CUDA graph replay" if args.graph else "stream launches"},
+                   "launch": "CUDA graph replay" if args.graph else "stream launches",
+                   "x_perm": "never written (rows gathered by the GEMMs)" if args.gather else "materialised"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "device_status": status,
         "host_enqueue_ms_per_step": host_enqueue_ms,
         "roofline": roofline, "roofline_hbm_steps": hbm_steps, "cpu_baseline": cpu_baseline,

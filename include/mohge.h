@@ -276,6 +276,42 @@ int32_t mohge_expert_bwd_dgate(const mohge_config* cfg, int64_t T, const void* d
                                void* stream);
 
 /*
+ * The same path without the permuted copy of x.  Eq. 15 is evaluated expert by expert, which
+ * needs the rows of x in expert order; mohge_dispatch materialises them (x_perm), these three
+ * calls do not: the dispatch only builds the permutation and a row map, and the two GEMMs that
+ * read x_perm (the gate/up projection of the forward pass and the gate/up weight gradient) gather
+ * the rows of x themselves (16-byte asynchronous copies by the producer warp into the swizzled
+ * operand tile).  They save the 2 x (T + R) d bytes of writing and re-reading x_perm and one
+ * kernel, but on B200 a row gather feeds the tensor cores far more slowly than a TMA box does
+ * (measured at T = 65536, d = 4096: step 44 -> 53 ms), so the calls above stay the fast path.
+ * BF16 tensor-core path only (MOHGE_ERR_UNSUPPORTED otherwise); T > 0.  Everything not listed is
+ * as in the calls above.
+ *   mohge_dispatch_indices   as mohge_dispatch without x and x_perm, plus
+ *       tok_of_prow [mohge_perm_rows + 128] int32: the token whose row sits at physical row r,
+ *       T (out of range: reads as zeros) for padding rows and past the last segment
+ *   mohge_expert_fwd_gather  as mohge_expert_fwd with x [T, d] and tok_of_prow instead of x_perm
+ *   mohge_expert_bwd_gather  as mohge_expert_bwd_dgate with x and tok_of_prow instead of x_perm
+ * Results are bit-identical to the calls they replace (the same tiles multiply the same values).
+ */
+int32_t mohge_dispatch_indices(const mohge_config* cfg, int64_t T, const int32_t* expert_idx,
+                               int32_t* counts, int32_t* offsets, int32_t* aligned_offsets,
+                               int32_t* row_of, int32_t* prow_of, int32_t* src_of,
+                               int32_t* tok_of_prow, void* ws, void* stream);
+int32_t mohge_expert_fwd_gather(const mohge_config* cfg, int64_t T, const void* x,
+                                const int32_t* tok_of_prow, const int32_t* counts,
+                                const int32_t* aligned_offsets, const void* const* w13,
+                                const void* const* w2, void* au_saved, void* h_saved, void* y_perm,
+                                void* ws, void* stream);
+int32_t mohge_expert_bwd_gather(const mohge_config* cfg, int64_t T, const void* dy_perm,
+                                const void* x, const int32_t* tok_of_prow, const void* au_saved,
+                                const void* h_saved, const int32_t* counts,
+                                const int32_t* aligned_offsets, const void* const* w13,
+                                const void* const* w2, void* dau, void* dx_perm, float* const* dw13,
+                                float* const* dw2, int32_t accumulate, const void* dy,
+                                const void* y_perm, const int32_t* prow_of, const float* gate_w,
+                                float* dgate_w, void* ws, void* stream);
+
+/*
  * Backward of the permutation: dx[t, :] = sum_k dx_perm[prow_of[t,k], :] (+ dx_add[t, :]).
  *   dx [T, d] dtype;  dx_add [T, d] dtype, nullable (the shared experts' input gradient).
  */

@@ -56,6 +56,10 @@ _SIGS = {
                          + [C.c_int32, _P, _P]),
     "mohge_expert_bwd_dgate": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 12
                                + [C.c_int32] + [_P] * 7),
+    "mohge_dispatch_indices": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 10),
+    "mohge_expert_fwd_gather": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 11),
+    "mohge_expert_bwd_gather": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 13
+                                + [C.c_int32] + [_P] * 7),
     "mohge_dispatch_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 5),
     "mohge_shared_fwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 8),
     "mohge_shared_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 10
@@ -277,6 +281,36 @@ def mohge_expert_bwd_dgate(cfg, T, dy_perm, x_perm, au_saved, h_saved, counts, a
                                         _ptr(ws), _stream()), "mohge_expert_bwd_dgate")
 
 
+def mohge_dispatch_indices(cfg, T, expert_idx, counts, offsets, aligned_offsets, row_of, prow_of,
+                           src_of, tok_of_prow, ws):
+    _check(lib().mohge_dispatch_indices(C.byref(cfg.c()), T, _ptr(expert_idx), _ptr(counts),
+                                        _ptr(offsets), _ptr(aligned_offsets), _ptr(row_of),
+                                        _ptr(prow_of), _ptr(src_of), _ptr(tok_of_prow), _ptr(ws),
+                                        _stream()), "mohge_dispatch_indices")
+
+
+def mohge_expert_fwd_gather(cfg, T, x, tok_of_prow, counts, aligned_offsets, w13, w2, au_saved, h_saved,
+                            y_perm, ws):
+    a13, a2 = _ptr_array(w13), _ptr_array(w2)
+    _check(lib().mohge_expert_fwd_gather(C.byref(cfg.c()), T, _ptr(x), _ptr(tok_of_prow), _ptr(counts),
+                                         _ptr(aligned_offsets), C.cast(a13, _P), C.cast(a2, _P),
+                                         _ptr(au_saved), _ptr(h_saved), _ptr(y_perm), _ptr(ws), _stream()),
+           "mohge_expert_fwd_gather")
+
+
+def mohge_expert_bwd_gather(cfg, T, dy_perm, x, tok_of_prow, au_saved, h_saved, counts, aligned_offsets,
+                            w13, w2, dau, dx_perm, dw13, dw2, accumulate, dy, y_perm, prow_of, gate_w,
+                            dgate_w, ws):
+    a13, a2, d13, d2 = _ptr_array(w13), _ptr_array(w2), _ptr_array(dw13), _ptr_array(dw2)
+    _check(lib().mohge_expert_bwd_gather(C.byref(cfg.c()), T, _ptr(dy_perm), _ptr(x), _ptr(tok_of_prow),
+                                         _ptr(au_saved), _ptr(h_saved), _ptr(counts),
+                                         _ptr(aligned_offsets), C.cast(a13, _P), C.cast(a2, _P),
+                                         _ptr(dau), _ptr(dx_perm), C.cast(d13, _P), C.cast(d2, _P),
+                                         int(accumulate), _ptr(dy), _ptr(y_perm), _ptr(prow_of),
+                                         _ptr(gate_w), _ptr(dgate_w), _ptr(ws), _stream()),
+           "mohge_expert_bwd_gather")
+
+
 def mohge_dispatch_bwd(cfg, T, dx_perm, prow_of, dx, dx_add=None):
     _check(lib().mohge_dispatch_bwd(C.byref(cfg.c()), T, _ptr(dx_perm), _ptr(prow_of),
                                     _ptr(dx_add), _ptr(dx), _stream()), "mohge_dispatch_bwd")
@@ -328,6 +362,7 @@ class LayerBuffers:
         self.counts, self.offsets, self.aligned = e(Ne, dtype=i32), e(Ne + 4, dtype=i32), e(Ne + 4, dtype=i32)
         self.row_of, self.prow_of, self.src_of = e(Tn, Ke, dtype=i32), e(Tn, Ke, dtype=i32), e(Tn * Ke, dtype=i32)
         self.x_perm, self.y_perm = e(rows, d), e(rows, d)
+        self.tok_of_prow = e(rows + 128, dtype=i32)        # row map of the gathering entry points
         self.au, self.h = e(rows, 2 * Wmax), e(rows, Wmax)
         self.y = e(Tn, d)
         # backward
@@ -346,18 +381,26 @@ class LayerBuffers:
 
 
 def layer_forward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, logit_bias=None,
-                  logits_in=None, aux=True, shared=None):
+                  logits_in=None, aux=True, shared=None, gather=False):
     """route -> aux_stats -> dispatch -> expert_fwd (-> shared_fwd) -> combine; results stay in
-    `b`.  shared = (w13_shared, w2_shared) adds the shared experts (b.shared_width wide)."""
+    `b`.  shared = (w13_shared, w2_shared) adds the shared experts (b.shared_width wide).
+    gather: no x_perm is written; the GEMMs gather the rows of x (mohge_dispatch_indices,
+    mohge_expert_fwd_gather)."""
     T = b.T
     mohge_route(cfg, T, x, w_router, logit_bias, logits_in, b.logits, b.group_idx, b.expert_idx,
                 b.gate_w, b.gs, b.esp, b.ws)
     if aux:
         mohge_aux_stats(cfg, T, b.gs, b.esp, b.group_idx, b.expert_idx, b.group_count, b.group_psum,
                         b.cnt_routed, b.cnt_lit, b.expert_psum, b.loss, b.ws)
-    mohge_dispatch(cfg, T, x, b.expert_idx, b.counts, b.offsets, b.aligned, b.row_of, b.prow_of,
-                   b.src_of, b.x_perm, b.ws)
-    mohge_expert_fwd(cfg, T, b.x_perm, b.counts, b.aligned, w13, w2, b.au, b.h, b.y_perm, b.ws)
+    if gather:
+        mohge_dispatch_indices(cfg, T, b.expert_idx, b.counts, b.offsets, b.aligned, b.row_of, b.prow_of,
+                               b.src_of, b.tok_of_prow, b.ws)
+        mohge_expert_fwd_gather(cfg, T, x, b.tok_of_prow, b.counts, b.aligned, w13, w2, b.au, b.h,
+                                b.y_perm, b.ws)
+    else:
+        mohge_dispatch(cfg, T, x, b.expert_idx, b.counts, b.offsets, b.aligned, b.row_of, b.prow_of,
+                       b.src_of, b.x_perm, b.ws)
+        mohge_expert_fwd(cfg, T, b.x_perm, b.counts, b.aligned, w13, w2, b.au, b.h, b.y_perm, b.ws)
     if shared is not None:
         mohge_shared_fwd(cfg, T, b.shared_width, x, shared[0], shared[1], b.au_sh, b.h_sh, b.y_sh, b.ws)
     mohge_combine(cfg, T, b.y_perm, b.prow_of, b.gate_w, b.y,
@@ -366,12 +409,17 @@ def layer_forward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, logit_bias
 
 
 def layer_backward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, dy, aux=True, accumulate=False,
-                   shared=None, fused_dgate=True):
+                   shared=None, fused_dgate=True, gather=False):
     """combine_bwd -> expert_bwd (-> shared_bwd) -> dispatch_bwd -> route_bwd; results stay in `b`.
     fused_dgate: the gate gradient comes out of the experts' backward (mohge_expert_bwd_dgate) and
     combine_bwd does not read y_perm; otherwise combine_bwd computes it from y_perm."""
     T = b.T
-    if fused_dgate:
+    if gather:      # after a forward with gather=True: x_perm was never written
+        mohge_combine_bwd(cfg, T, dy, None, b.prow_of, b.gate_w, b.counts, b.aligned, b.dy_perm, None)
+        mohge_expert_bwd_gather(cfg, T, b.dy_perm, x, b.tok_of_prow, b.au, b.h, b.counts, b.aligned, w13,
+                                w2, b.dau, b.dx_perm, b.dw13, b.dw2, accumulate, dy, b.y_perm, b.prow_of,
+                                b.gate_w, b.dgate, b.ws)
+    elif fused_dgate:
         mohge_combine_bwd(cfg, T, dy, None, b.prow_of, b.gate_w, b.counts, b.aligned, b.dy_perm, None)
         mohge_expert_bwd_dgate(cfg, T, b.dy_perm, b.x_perm, b.au, b.h, b.counts, b.aligned, w13, w2,
                                b.dau, b.dx_perm, b.dw13, b.dw2, accumulate, dy, b.y_perm, b.prow_of,

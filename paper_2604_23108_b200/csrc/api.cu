@@ -342,12 +342,27 @@ int32_t mohge_dispatch(const mohge_config* cfg, int64_t T, const void* x,
                          x_perm, w.hist, w.base, w.status, (cudaStream_t)stream);
 }
 
+int32_t mohge_dispatch_indices(const mohge_config* cfg, int64_t T, const int32_t* expert_idx,
+                               int32_t* counts, int32_t* offsets, int32_t* aligned_offsets,
+                               int32_t* row_of, int32_t* prow_of, int32_t* src_of,
+                               int32_t* tok_of_prow, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(expert_idx); REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR(aligned_offsets);
+  REQ_PTR(row_of); REQ_PTR(prow_of); REQ_PTR(src_of); REQ_PTR(tok_of_prow); REQ_PTR(ws);
+  const Ws w = carve(D, ws);
+  return launch_dispatch(D, nullptr, expert_idx, counts, offsets, aligned_offsets, row_of, prow_of, src_of,
+                         nullptr, w.hist, w.base, w.status, (cudaStream_t)stream, tok_of_prow);
+}
+
 // Forward of the grouped SwiGLU experts for already validated arguments.  Shared by the routed
 // experts and by the shared experts (one segment of T rows).
+// gather != nullptr: x_perm is x itself and row r of the permuted numbering is row gather[r] of it.
 static int32_t expert_fwd_impl(const Dims& D, const GroupPtrs& P, const void* x_perm,
                                const int32_t* counts, const int32_t* aligned_offsets,
                                void* au_saved, void* h_saved, void* y_perm, const Ws& w,
-                               cudaStream_t st) {
+                               cudaStream_t st, const int32_t* gather = nullptr) {
   int32_t rc;
   if (D.bf16 && !force_simt()) {
     MOHGE_CHECK_ARG(D.align == 128, "the BF16 tensor-core path needs row_align = 128");
@@ -357,11 +372,16 @@ static int32_t expert_fwd_impl(const Dims& D, const GroupPtrs& P, const void* x_
                                   w.status, st);
     if (rc) return rc;
     rc = launch_tc_grouped(D, ROLE_FWD1, P, x_perm, nullptr, au_saved, h_saved, counts,
-                           aligned_offsets, 0, w.tile_count, w.tiles, w.tiles_cap, w.status, st, true);
+                           aligned_offsets, 0, w.tile_count, w.tiles, w.tiles_cap, w.status, st, true,
+                           nullptr, 0, gather);
     if (rc) return rc;
     return launch_tc_grouped(D, ROLE_FWD2, P, h_saved, nullptr, y_perm, nullptr, counts,
                              aligned_offsets, 0, w.tile_count + 64, w.tiles + w.tiles_cap,
                              w.tiles_cap, w.status, st, true);
+  }
+  if (gather) {
+    set_error("the row-gathering entry points need the BF16 tensor-core path");
+    return MOHGE_ERR_UNSUPPORTED;
   }
   rc = launch_build_tiles(D, ROLE_FWD1, 64, 64, counts, aligned_offsets, w.tile_count, w.tiles,
                           w.tiles_cap, w.status, st);
@@ -393,6 +413,25 @@ int32_t mohge_expert_fwd(const mohge_config* cfg, int64_t T, const void* x_perm,
   if (rc) return rc;
   return expert_fwd_impl(D, P, x_perm, counts, aligned_offsets, au_saved, h_saved, y_perm,
                          carve(D, ws), (cudaStream_t)stream);
+}
+
+int32_t mohge_expert_fwd_gather(const mohge_config* cfg, int64_t T, const void* x,
+                                const int32_t* tok_of_prow, const int32_t* counts,
+                                const int32_t* aligned_offsets, const void* const* w13,
+                                const void* const* w2, void* au_saved, void* h_saved, void* y_perm,
+                                void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(x); REQ_PTR(tok_of_prow); REQ_PTR(counts); REQ_PTR(aligned_offsets); REQ_PTR(au_saved);
+  REQ_PTR(h_saved); REQ_PTR(y_perm); REQ_PTR(ws);
+  MOHGE_CHECK_ARG(w13 && w2, "w13 and w2 must be host arrays of n_groups device pointers");
+  MOHGE_CHECK_ARG(D.d % 8 == 0 && T > 0, "the row-gathering entry points need T > 0");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, nullptr, nullptr, &P);
+  if (rc) return rc;
+  return expert_fwd_impl(D, P, x, counts, aligned_offsets, au_saved, h_saved, y_perm, carve(D, ws),
+                         (cudaStream_t)stream, tok_of_prow);
 }
 
 int32_t mohge_combine(const mohge_config* cfg, int64_t T, const void* y_perm,
@@ -435,8 +474,12 @@ static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy
                                const void* x_perm, const void* au_saved, const void* h_saved,
                                const int32_t* counts, const int32_t* aligned_offsets, void* dau,
                                void* dx_perm, int32_t accumulate, const Ws& w, cudaStream_t st,
-                               const DgateArgs* dg = nullptr) {
+                               const DgateArgs* dg = nullptr, const int32_t* gather = nullptr) {
   int32_t rc;
+  if (gather && !(D.bf16 && !force_simt())) {
+    set_error("the row-gathering entry points need the BF16 tensor-core path");
+    return MOHGE_ERR_UNSUPPORTED;
+  }
   if (!accumulate) {
     rc = launch_zero_empty_wgrad(D, P, counts, st);
     if (rc) return rc;
@@ -459,7 +502,7 @@ static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy
       }
       rc = launch_tc_grouped(D, roles[r], P, A, B, C, C2, counts, aligned_offsets, accumulate,
                              w.tile_count + 64 * r, w.tiles + w.tiles_cap * r, w.tiles_cap, w.status,
-                             st, true, dg ? w.dgp : nullptr, w.dgate_slots);
+                             st, true, dg ? w.dgp : nullptr, w.dgate_slots, gather);
       if (rc) return rc;
       if (dg && roles[r] == ROLE_DGRAD_DOWN) {
         int bn[MOHGE_MAX_GROUPS];
@@ -538,6 +581,30 @@ int32_t mohge_expert_bwd_dgate(const mohge_config* cfg, int64_t T, const void* d
   const DgateArgs dg = {dy, y_perm, prow_of, gate_w, dgate_w};
   return expert_bwd_impl(D, P, dy_perm, x_perm, au_saved, h_saved, counts, aligned_offsets, dau,
                          dx_perm, accumulate, carve(D, ws), (cudaStream_t)stream, &dg);
+}
+
+int32_t mohge_expert_bwd_gather(const mohge_config* cfg, int64_t T, const void* dy_perm,
+                                const void* x, const int32_t* tok_of_prow, const void* au_saved,
+                                const void* h_saved, const int32_t* counts,
+                                const int32_t* aligned_offsets, const void* const* w13,
+                                const void* const* w2, void* dau, void* dx_perm, float* const* dw13,
+                                float* const* dw2, int32_t accumulate, const void* dy,
+                                const void* y_perm, const int32_t* prow_of, const float* gate_w,
+                                float* dgate_w, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(dy_perm); REQ_PTR(x); REQ_PTR(tok_of_prow); REQ_PTR(au_saved); REQ_PTR(h_saved); REQ_PTR(counts);
+  REQ_PTR(aligned_offsets); REQ_PTR(dau); REQ_PTR(dx_perm); REQ_PTR(ws);
+  REQ_PTR(dy); REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(dgate_w);
+  MOHGE_CHECK_ARG(w13 && w2 && dw13 && dw2, "w13, w2, dw13, dw2 must be host arrays of n_groups device pointers");
+  MOHGE_CHECK_ARG(T > 0, "the row-gathering entry points need T > 0");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, dw13, dw2, &P);
+  if (rc) return rc;
+  const DgateArgs dg = {dy, y_perm, prow_of, gate_w, dgate_w};
+  return expert_bwd_impl(D, P, dy_perm, x, au_saved, h_saved, counts, aligned_offsets, dau, dx_perm,
+                         accumulate, carve(D, ws), (cudaStream_t)stream, &dg, tok_of_prow);
 }
 
 int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,

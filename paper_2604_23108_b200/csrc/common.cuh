@@ -178,10 +178,11 @@ int32_t launch_router_bwd_elementwise(const Dims& D, const mohge_config& cfg, co
                                       cudaStream_t st);
 
 // dispatch.cu
+constexpr int kGatherSlack = 128;   // rows of the gather map past mohge_perm_rows (a pair's tile may reach them)
 int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx, int32_t* counts,
                         int32_t* offsets, int32_t* aligned, int32_t* row_of, int32_t* prow_of,
                         int32_t* src_of, void* x_perm, int32_t* hist, int32_t* base,
-                        int32_t* status, cudaStream_t st);
+                        int32_t* status, cudaStream_t st, int32_t* tok_of_prow = nullptr);
 int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of,
                        const float* gate_w, const void* add, void* y, cudaStream_t st);
 int32_t launch_combine_bwd(const Dims& D, int mode, const void* dy, const void* y_perm,
@@ -212,11 +213,14 @@ int32_t launch_simt_plain(int M, int N, int K, const void* A, int a_f32, int64_t
                           int64_t sCm, const float* bias, int accumulate, cudaStream_t st);
 
 // gemm_tc.cu (tcgen05 path, BF16)
+// gather != nullptr (FWD1, WGRAD_13 only): the x_perm operand (A of FWD1, B of WGRAD_13) is x
+// itself, [T, d], and row r of the permuted numbering is row gather[r] of it (>= T: zeros)
 int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
                           const void* B, void* C, void* C2, const int32_t* counts,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
                           int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt = false,
-                          float* dgate_part = nullptr, int dgate_slots = 0);
+                          float* dgate_part = nullptr, int dgate_slots = 0,
+                          const int32_t* gather = nullptr);
 // UMMA N of a group in ROLE_DGRAD_DOWN (128 or 256): which 128-column slots of dgate_part are written
 int tc_dgrad_down_bn(const Dims& D, int g);
 TilePlan tc_tile_plan(const Dims& D, int role);

@@ -407,6 +407,29 @@ dgate_reduce_kernel(DgateShape s, int n, const float* __restrict__ part,
   }
 }
 
+// Source token of every physical row of the permuted numbering (T, which is out of range, for
+// padding rows and for the 128 rows past the last segment that a CTA pair's tile may touch):
+// the row map the experts' GEMMs use to gather rows of x themselves instead of reading x_perm.
+__global__ void __launch_bounds__(256)
+token_of_row_kernel(int n_rows, int T, int Ke, int Ne, const int32_t* __restrict__ counts,
+                    const int32_t* __restrict__ offsets, const int32_t* __restrict__ aligned,
+                    const int32_t* __restrict__ src_of, int32_t* __restrict__ tok_of_prow) {
+  pdl_enter();
+  for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < n_rows; r += gridDim.x * blockDim.x) {
+    int tok = T;
+    if (r < aligned[Ne]) {
+      int lo = 0, hi = Ne;               // aligned[lo] <= r < aligned[hi]
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (aligned[mid] <= r) lo = mid; else hi = mid;
+      }
+      const int j = r - aligned[lo];
+      if (j < counts[lo]) tok = src_of[offsets[lo] + j] / Ke;
+    }
+    tok_of_prow[r] = tok;
+  }
+}
+
 int block_for(int row_vecs) {
   int b = (row_vecs + 31) / 32 * 32;
   if (b > 256) b = 256;
@@ -416,10 +439,12 @@ int block_for(int row_vecs) {
 
 }  // namespace
 
+// x != nullptr: rows of x are copied into x_perm; tok_of_prow != nullptr: the row map for the
+// gathering GEMMs is written instead (kGatherSlack rows past mohge_perm_rows included).
 int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx, int32_t* counts,
                         int32_t* offsets, int32_t* aligned, int32_t* row_of, int32_t* prow_of,
                         int32_t* src_of, void* x_perm, int32_t* hist, int32_t* base,
-                        int32_t* status, cudaStream_t st) {
+                        int32_t* status, cudaStream_t st, int32_t* tok_of_prow) {
   const int chunks = ceil_div(D.T, kDispatchChunk);
   const int T = (int)D.T;
   if (chunks > 0) {
@@ -428,10 +453,19 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
   }
   launch_dep(dispatch_scan_kernel, dim3(1), dim3(256), st, chunks, D.Ne, D.align, hist, base, counts, offsets, aligned);
   MOHGE_LAUNCH_CHECK("dispatch_scan_kernel");
-  if (chunks == 0) return MOHGE_OK;
-  launch_dep(dispatch_scatter_kernel, dim3(chunks), dim3(kDispatchChunk), st, expert_idx, T, D.Ke, D.Ne, base, offsets,
-                                                            aligned, row_of, prow_of, src_of, status);
-  MOHGE_LAUNCH_CHECK("dispatch_scatter_kernel");
+  if (chunks > 0) {
+    launch_dep(dispatch_scatter_kernel, dim3(chunks), dim3(kDispatchChunk), st, expert_idx, T, D.Ke, D.Ne, base, offsets,
+                                                              aligned, row_of, prow_of, src_of, status);
+    MOHGE_LAUNCH_CHECK("dispatch_scatter_kernel");
+  }
+  if (tok_of_prow != nullptr) {
+    const int n_rows = (int)D.Rcap + kGatherSlack;
+    launch_dep(token_of_row_kernel, dim3((n_rows + 255) / 256 < 1184 ? (n_rows + 255) / 256 : 1184), dim3(256), st,
+               n_rows, T, D.Ke, D.Ne, (const int32_t*)counts, (const int32_t*)offsets, (const int32_t*)aligned,
+               (const int32_t*)src_of, tok_of_prow);
+    MOHGE_LAUNCH_CHECK("token_of_row_kernel");
+  }
+  if (chunks == 0 || x == nullptr) return MOHGE_OK;
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
   const int blocks = T < 148 * 16 ? T : 148 * 16;
   const int pad_blocks = D.align > 1 ? 4 * D.Ne : 0;

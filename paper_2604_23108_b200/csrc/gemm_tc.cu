@@ -7,6 +7,8 @@
 //   warps 2..5  epilogue: tcgen05.ld -> registers -> fused element-wise math -> swizzled staging
 //               buffers in shared memory -> TMA stores (every global write of the expert roles is
 //               a full 128-byte row piece; the SwiGLU backward also reads A and U through TMA)
+//   warp 6      only in the row-gathering form (GATHER = 1, see "gathering form" below): forwards
+//               the completion of the producer warp's asynchronous row copies to the MMA issuer
 // One persistent CTA per SM (a CTA pair per two SMs for the expert roles; single CTAs when the
 // batch brings 128 rows per expert or fewer) walks the device-built, cost-sorted tile list with a
 // fixed stride, in alternating directions when tile costs differ.  The kernel is launched as a
@@ -45,7 +47,16 @@ namespace {
 constexpr int BM = 128;          // UMMA M (rows of an output tile)
 constexpr int BK = 64;           // contraction elements per pipeline stage (128 bytes of BF16)
 constexpr int kABytes = BM * BK * 2;          // 16 KiB: 128 rows of A per CTA and stage
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;                 // producer, MMA issuer, four epilogue warps
+// Row-gathering form (GATHER = 1): kGatherWarps warps copy rows (the producer warp and
+// kGatherWarps - 1 more), one more warp relays their completions to the MMA issuer.  More
+// gathering warps bring nothing (measured with 1, 2 and 4: 854 / 833 / 833 clocks per k-block in
+// FWD1): the copies are bound by what an SM keeps in flight through its load path, not by issue.
+#ifndef MOHGE_GATHER_WARPS
+#define MOHGE_GATHER_WARPS 1
+#endif
+constexpr int kGatherWarps = MOHGE_GATHER_WARPS;     // 1, 2 or 4
+constexpr int kThreadsGather = kThreads + 32 * kGatherWarps;
 constexpr int kAccCols = 256;                 // tensor-memory columns per accumulator buffer
 
 // Build-time option -DMOHGE_TC_COUNTERS: every CTA adds, per role, the clocks its MMA issuer spent
@@ -112,6 +123,12 @@ struct TcParams {
   // [N, rows, cols]
   CUtensorMap mapO[3][MOHGE_MAX_GROUPS];
   CUtensorMap mapE[2][MOHGE_MAX_GROUPS];   // DGRAD_DOWN epilogue inputs: saved A and U regions
+  // Row gather (FWD1: A operand, WGRAD_13: B operand): instead of x_perm the operand is
+  // gather_src = x itself, [gather_rows, d], and row r of the permuted numbering is row
+  // gather[r] of it; indices >= gather_rows read as zeros (padding rows).
+  const int32_t* gather;
+  const void* gather_src;
+  int gather_rows;
   GroupShape gs;
   GroupPtrs gp;
   int BN[MOHGE_MAX_GROUPS];      // UMMA N per group (FWD1: gate half + up half)
@@ -273,6 +290,11 @@ __device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t bar_cluster, uin
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
   asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
 }
+// the same with release semantics at cluster scope: what this thread has observed (the landed row
+// copies of the gathering form) is visible to whoever acquires the barrier's phase
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
 // loads of the pair signal the barrier of the leader CTA (cluster address)
 __device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
   asm volatile(
@@ -293,6 +315,15 @@ __device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap* ma
   asm volatile(
       "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+// 16 bytes global -> shared, asynchronously, no registers in between (src_bytes = 0 writes zeros)
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+// the barrier receives one arrival from this thread once all its earlier cp.async have landed
+// (.noinc: the arrival is part of the barrier's expected count)
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 template <int CG>
 __device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
@@ -470,8 +501,8 @@ __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t, 
   return q;
 }
 
-template <int ROLE, int CG, int WIDE>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int ROLE, int CG, int WIDE, int GATHER = 0>
+__global__ void __launch_bounds__(GATHER ? kThreadsGather : kThreads, 1)
 tc_grouped_kernel(const __grid_constant__ TcParams p) {
   using RT = RoleTraits<ROLE>;
   using G = Geo<CG, WIDE>;
@@ -491,7 +522,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kStages + 2 + b); };
   auto ein_bar = [&](int quad, int set) { return bar0 + 8u * (2 * kStages + 4 + quad * 2 + set); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 12);
+  auto gath_bar = [&](int s) { return bar0 + 8u * (2 * kStages + 12 + s); };   // row copies of a stage have landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 12 + kStages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   // expert segment table (aligned_offsets) staged once, so that no role chases it through global
   // memory between tiles
@@ -508,8 +540,10 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(full_bar(s), CG);       // one arrive.expect_tx per CTA of the pair
+      // one arrive.expect_tx per CTA of the pair, plus one relayed arrival per CTA when rows are gathered
+      mbar_init(full_bar(s), GATHER ? 2 * CG : CG);
       mbar_init(empty_bar(s), 1);
+      mbar_init(gath_bar(s), 32 * kGatherWarps);       // every lane of the gathering warps
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
@@ -563,7 +597,137 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     return ti < 0 ? z : fetch_tile<ROLE>(p, ti);
   };
 
-  if (warp == 0) {
+  if (GATHER && (warp == 0 || (warp >= 6 && warp < 5 + kGatherWarps))) {
+    // ================= producer, gathering form =================
+    // The x_perm operand (A of FWD1, B of WGRAD_13) is not read from a permuted copy: its rows are
+    // rows of x, found through the row map p.gather.  TMA has no efficient row gather (a
+    // tile::gather4 copy of four 128-byte rows costs the TMA unit about 77 clocks, 6.6 B per
+    // clock), so the whole producer warp brings these rows with 16-byte cp.async copies straight
+    // into the swizzled stage (chunk c of row r at r * 128 + ((c ^ (r & 7)) << 4), the layout a
+    // TMA box with the 128-byte swizzle produces), while lane 0 of warp 0 still issues the TMA
+    // boxes of the other operand.  One warp keeps too few copies in flight against the memory
+    // latency (measured: 40-50 clocks per warp-wide copy instruction), so kGatherWarps warps share
+    // the rows of a stage: warp gw takes a quarter of the row slots.  Lane l takes chunk l % 8 of
+    // the rows l / 8, l / 8 + 4, ...
+    //   FWD1      A tile = 128 rows x 128 B per k-block; the 32 row indices of a lane are fixed
+    //             for a tile and live in registers
+    //   WGRAD_13  B tile = blocks of 64 k-rows x 128 B; the rows are the contraction index, so a
+    //             lane's 16 row indices change with every k-block and are fetched one ahead
+    // Each lane's copies of a stage end in cp.async.mbarrier.arrive on the stage's gather
+    // barrier; the relay warp waits for that barrier, makes the rows visible to the async proxy
+    // and arrives on the pair leader's full barrier.  Row indices >= T (padding rows) and columns
+    // past d are written as zeros.
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;
+    const int gw = warp == 0 ? 0 : warp - 5;           // 0 .. kGatherWarps - 1
+    const int c16 = lane & 7, r_lo = lane >> 3;
+    const char* const xg = reinterpret_cast<const char*>(p.gather_src);
+    const size_t pitch = 2 * (size_t)p.gs.d;
+    const int n_src = p.gather_rows;
+    Tile t_pf = prefetch_tile(it0);
+    for (int it = it0; it < it_end && alive; it += it_step) {
+      const int ti = zigzag ? tile_of(it) : it;
+      const Tile t = t_pf;
+      t_pf = prefetch_tile(it + it_step);
+      if (ti < 0) continue;
+      const TileGeom q = tile_geom<ROLE>(p, t, s_seg);
+      const CUtensorMap* mA = &p.mapA[q.g];
+      const CUtensorMap* mB = &p.mapB[q.g];
+      const int nb = q.bn / CG;
+      const int pieces = (WIDE && q.wide) ? 2 : 1;
+      const int am0 = q.m0 + BM * (int)cta_rank;
+      // bytes TMA brings per stage: the operand that is not gathered
+      const uint32_t tx = ROLE == ROLE_FWD1 ? (uint32_t)pieces * nb * BK * 2 : (uint32_t)kABytes;
+      constexpr int kRowsF = 32 / kGatherWarps;         // FWD1: row slots of this warp's lanes
+      // WGRAD_13: a stage has nblk 64-column blocks of 16 row slots (j) each; the warps share the
+      // blocks (or, with fewer blocks than warps, the slots of a block)
+      const int nblk = pieces * (nb / 64);
+      int rows[kRowsF > 16 ? kRowsF : 16];             // FWD1: row of slot j of this warp; WGRAD_13: row of slot j
+      int rows_next[16];
+      if (ROLE == ROLE_FWD1) {
+#pragma unroll
+        for (int j = 0; j < kRowsF; ++j) rows[j] = p.gather[am0 + r_lo + 4 * (gw * kRowsF + j)];
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) rows[j] = p.gather[q.r0 + r_lo + 4 * j];
+      }
+      for (int kb = 0; kb < q.num_kb; ++kb) {
+        if (ROLE == ROLE_WGRAD_13) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            rows_next[j] = kb + 1 < q.num_kb ? p.gather[q.r0 + (kb + 1) * BK + r_lo + 4 * j] : 0;
+        }
+        int ok = 1;
+        if (lane == 0) ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 1) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) { alive = false; break; }
+        const uint32_t sA = smem_base + stage * kStageBytes;
+        const uint32_t fb = CG == 2 ? mapa_rank(full_bar(stage), 0) : full_bar(stage);
+        const int k0 = kb * BK;
+        if (lane == 0 && gw == 0) {
+          if (CG == 2) mbar_expect_tx_cluster(fb, tx); else mbar_expect_tx(fb, tx);
+          if (ROLE == ROLE_FWD1) {
+            for (int pc = 0; pc < pieces; ++pc) {
+              const uint32_t sB = sA + kABytes + pc * G::kBBytes;
+              const int half = q.bn >> 1;
+              const int h0 = q.n0 + pc * half;
+              if (CG == 2) {
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i + (int)cta_rank);
+              } else {
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i);
+                tma_3d<CG>(sB + half * 128, mB, fb, k0, h0, 2 * q.i + 1);
+              }
+            }
+          } else {
+            if (p.a_blk[q.g]) {
+              tma_3d<CG>(sA, mA, fb, 0, q.r0 + k0, am0 >> 6);
+            } else {
+              tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0);
+              tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0);
+            }
+          }
+        }
+        if (ROLE == ROLE_FWD1) {
+          const int col = k0 + 8 * c16;                  // first of this lane's 8 columns
+          const uint32_t col_ok = col < p.gs.d ? 16u : 0u;
+          const size_t col_off = col < p.gs.d ? 2 * (size_t)col : 0;
+#pragma unroll
+          for (int j = 0; j < kRowsF; ++j) {
+            const int r = r_lo + 4 * (gw * kRowsF + j), src = rows[j];
+            const bool in = src < n_src;
+            cp_async_16(sA + (uint32_t)r * 128u + (uint32_t)((c16 ^ (r & 7)) << 4),
+                        xg + (in ? (size_t)src * pitch : 0) + col_off, in ? col_ok : 0u);
+          }
+        } else {
+          // blocks of this warp: blk = gw, gw + W, ... when there are at least W = kGatherWarps
+          // blocks; else every warp works on block gw % nblk and takes a part of its 16 slots
+          const int share = nblk >= kGatherWarps ? 1 : kGatherWarps / nblk;     // warps per block
+          const int j_lo = (gw / nblk) * (16 / share) * (share > 1 ? 1 : 0), j_n = 16 / share;
+          for (int blk = share > 1 ? gw % nblk : gw; blk < nblk; blk += share > 1 ? nblk : kGatherWarps) {
+            const int pc = blk / (nb / 64), jb = blk % (nb / 64);
+            const uint32_t sB = sA + kABytes + pc * G::kBBytes;
+            const int col = q.n0 + pc * q.bn + nb * (int)cta_rank + 64 * jb + 8 * c16;
+            const uint32_t col_ok = col < p.gs.d ? 16u : 0u;
+            const size_t col_off = col < p.gs.d ? 2 * (size_t)col : 0;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              if (j >= j_lo && j < j_lo + j_n) {
+                const int r = r_lo + 4 * j, src = rows[j];
+                const bool in = src < n_src;
+                cp_async_16(sB + (uint32_t)jb * 8192u + (uint32_t)r * 128u + (uint32_t)((c16 ^ (r & 7)) << 4),
+                            xg + (in ? (size_t)src * pitch : 0) + col_off, in ? col_ok : 0u);
+              }
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) rows[j] = rows_next[j];
+        }
+        cp_async_arrive(gath_bar(stage));
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
+    }
+  } else if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
       int stage = 0;
@@ -767,6 +931,30 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           atomicAdd(&cnt[2], (unsigned long long)c_full); atomicAdd(&cnt[3], (unsigned long long)c_tempty);
           atomicAdd(&cnt[8], (unsigned long long)c_tiles); atomicAdd(&cnt[9], (unsigned long long)c_kb);
           atomicAdd(&cnt[10], (unsigned long long)c_mid); atomicAdd(&cnt[11], (unsigned long long)c_midn);)
+    }
+  } else if (GATHER && warp == 5 + kGatherWarps) {
+    // ================= gather relay =================
+    // Gathering form only.  For every stage in the producer's order: wait until the 32 lanes'
+    // row copies have landed (the stage's gather barrier), make them visible to the async proxy
+    // (the MMAs read shared memory through it) and arrive on the full barrier of the pair's leader.
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      Tile t_pf = prefetch_tile(it0);
+      for (int it = it0; it < it_end && alive; it += it_step) {
+        const int ti = zigzag ? tile_of(it) : it;
+        const Tile t = t_pf;
+        t_pf = prefetch_tile(it + it_step);
+        if (ti < 0) continue;
+        const TileGeom q = tile_geom<ROLE>(p, t, s_seg);
+        for (int kb = 0; kb < q.num_kb; ++kb) {
+          if (!mbar_wait(gath_bar(stage), phase, abort_flag, p.status, 7)) { alive = false; break; }
+          fence_async_smem();
+          if (CG == 2) mbar_arrive_release_cluster(mapa_rank(full_bar(stage), 0)); else mbar_arrive(full_bar(stage));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
     }
   } else {
     // ================= epilogue warps =================
@@ -1046,7 +1234,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           for (int j = 0; j < 8; ++j)
             st_shared_v4(stg_addr(bO, lane, j), r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
         };
-        if (!next_kb && kSlots == 4 && nch > 4) {
+        if (!GATHER && !next_kb && kSlots == 4 && nch > 4) {
           // Nothing to pace against (double-width entries): four chunks go into the ring, the
           // other (up to) four wait in registers, and the accumulator is released at once.
           for (int i = 0; i < 4; ++i) {
@@ -1274,7 +1462,7 @@ struct MapKey {
   int32_t role, cg, device, accumulate_unused;
   int32_t d, Ng, N, Wmax, W[MOHGE_MAX_GROUPS];
   int64_t rows, T, b_pitch;
-  const void *A, *B, *C, *C2;
+  const void *A, *B, *C, *C2, *gather;
   const void* w[4][MOHGE_MAX_GROUPS];
 };
 struct MapEntry {
@@ -1335,7 +1523,7 @@ int pick_bn(int extent, const int* cand, int ncand) {
   return best;
 }
 
-template <int ROLE, int CG, int WIDE = 0>
+template <int ROLE, int CG, int WIDE = 0, int GATHER = 0>
 int32_t launch_role(const TcParams& p, const DeviceInfo& di, cudaStream_t st) {
   // The dynamic shared-memory limit of a kernel and the number of CTA pairs that fit are facts
   // of one device: both are kept per device ordinal (0 = not yet known on that device).
@@ -1343,14 +1531,14 @@ int32_t launch_role(const TcParams& p, const DeviceInfo& di, cudaStream_t st) {
   static std::atomic<int> max_clusters[kMaxDevices];
   const int grid = is_plain<ROLE>() ? (p.plain_total < di.sm_count ? p.plain_total : di.sm_count) : di.sm_count;
   if (!attr_set[di.ordinal].load(std::memory_order_acquire)) {
-    MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE, CG, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    MOHGE_CUDA(cudaFuncSetAttribute(tc_grouped_kernel<ROLE, CG, WIDE, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     Geo<CG, WIDE>::kSmemBytes));
     attr_set[di.ordinal].store(1, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(grid / CG * CG);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(GATHER ? kThreadsGather : kThreads);
   cfg.dynamicSmemBytes = Geo<CG, WIDE>::kSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -1368,7 +1556,7 @@ int32_t launch_role(const TcParams& p, const DeviceInfo& di, cudaStream_t st) {
     // share of the tile list after everyone else.
     int mc = max_clusters[di.ordinal].load(std::memory_order_acquire);
     if (!mc) {
-      MOHGE_CUDA(cudaOccupancyMaxActiveClusters(&mc, tc_grouped_kernel<ROLE, CG, WIDE>, &cfg));
+      MOHGE_CUDA(cudaOccupancyMaxActiveClusters(&mc, tc_grouped_kernel<ROLE, CG, WIDE, GATHER>, &cfg));
       if (mc < 1) mc = 1;
       max_clusters[di.ordinal].store(mc, std::memory_order_release);
     }
@@ -1382,7 +1570,7 @@ int32_t launch_role(const TcParams& p, const DeviceInfo& di, cudaStream_t st) {
     if (g >= CG && g < (int)cfg.gridDim.x) cfg.gridDim = dim3(g);
   }
 #endif
-  MOHGE_CUDA(cudaLaunchKernelEx(&cfg, tc_grouped_kernel<ROLE, CG, WIDE>, p));
+  MOHGE_CUDA(cudaLaunchKernelEx(&cfg, tc_grouped_kernel<ROLE, CG, WIDE, GATHER>, p));
   MOHGE_LAUNCH_CHECK("tc_grouped_kernel");
   return MOHGE_OK;
 }
@@ -1607,7 +1795,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
                           const void* B, void* C, void* C2, const int32_t* /*counts*/,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
                           int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt,
-                          float* dgate_part, int dgate_slots) {
+                          float* dgate_part, int dgate_slots, const int32_t* gather) {
   DeviceInfo di;
   int32_t rcd = current_device(&di);
   if (rcd) return rcd;
@@ -1624,6 +1812,9 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   p.accumulate = accumulate; p.status = status;
   p.dgate_part = role == ROLE_DGRAD_DOWN ? dgate_part : nullptr;
   p.dgate_slots = dgate_slots;
+  p.gather = (role == ROLE_FWD1 || role == ROLE_WGRAD_13) ? gather : nullptr;
+  p.gather_src = nullptr;
+  p.gather_rows = (int)D.T;
 
   const uint64_t d = D.d, rows = D.Rcap, pitchAU = 2ull * D.Wmax * 2, pitchH = (uint64_t)D.Wmax * 2;
   const int CG = cta_group_size(D);
@@ -1640,12 +1831,13 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   memset(&key, 0, sizeof(key));
   key.role = role; key.cg = CG; key.device = di.ordinal;
   key.d = D.d; key.Ng = D.Ng; key.N = D.N; key.Wmax = D.Wmax; key.rows = D.Rcap;
-  key.A = A; key.B = B; key.C = C; key.C2 = C2;
+  key.A = A; key.B = B; key.C = C; key.C2 = C2; key.gather = p.gather; key.T = D.T;
   for (int g = 0; g < D.Ng; ++g) {
     key.W[g] = D.W[g];
     key.w[0][g] = P.w13[g]; key.w[1][g] = P.w2[g]; key.w[2][g] = P.dw13[g]; key.w[3][g] = P.dw2[g];
   }
   const bool cached = map_cache_find(key, &p);
+  if (p.gather) p.gather_src = role == ROLE_FWD1 ? A : B;
   for (int g = 0; g < D.Ng && rc == MOHGE_OK && !cached; ++g) {
     const uint64_t W = D.W[g], N = D.N;
     uint64_t dims[3], str[2];
@@ -1654,8 +1846,12 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
       case ROLE_FWD1: {
         const int half = pick_bn(D.W[g], cand_h, CG == 2 ? 1 : 2);
         p.BN[g] = 2 * half; bn_plan[g] = half;
-        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
-        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (p.gather) {      // A = x [T, d], gathered row by row by the producer warp
+          p.gather_src = A;
+        } else {
+          dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
+          rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        }
         if (rc) break;
         dims[0] = d; dims[1] = W; dims[2] = 2 * N; str[0] = d * 2; str[1] = W * d * 2;
         box[0] = BK; box[1] = half; box[2] = 1;
@@ -1714,7 +1910,11 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
         p.BN[g] = bn_plan[g] = pick_bn(D.d, cand_n, ncand);
         rc = encode_mn_map(&p.mapA[g], A, 2 * W, rows, pitchAU, 0, 0, 2, &p.a_blk[g]);
         if (rc) break;
-        rc = encode_mn_map(&p.mapB[g], B, d, rows, d * 2, 0, 0, p.BN[g] / CG / 64, &p.b_blk[g]);
+        if (p.gather) {      // B = x [T, d], gathered row by row by the producer warp
+          p.gather_src = B;
+        } else {
+          rc = encode_mn_map(&p.mapB[g], B, d, rows, d * 2, 0, 0, p.BN[g] / CG / 64, &p.b_blk[g]);
+        }
         if (rc) break;
         rc = encode_stage_map_f32(&p.mapO[0][g], P.dw13[g], d, 2 * W, N);
       } break;
@@ -1727,6 +1927,16 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   if (!list_prebuilt) {
     rc = launch_build_tiles_plan(plan, aligned, tile_count, tiles, tiles_cap, status, st);
     if (rc) return rc;
+  }
+  if (p.gather) {          // row-gathering form of the two roles that read x_perm
+    if (role == ROLE_FWD1) {
+      if (CG == 2 && wide) return launch_role<ROLE_FWD1, 2, 1, 1>(p, di, st);
+      if (CG == 2) return launch_role<ROLE_FWD1, 2, 0, 1>(p, di, st);
+      return launch_role<ROLE_FWD1, 1, 0, 1>(p, di, st);
+    }
+    if (CG == 2 && wide) return launch_role<ROLE_WGRAD_13, 2, 1, 1>(p, di, st);
+    if (CG == 2) return launch_role<ROLE_WGRAD_13, 2, 0, 1>(p, di, st);
+    return launch_role<ROLE_WGRAD_13, 1, 0, 1>(p, di, st);
   }
   if (CG == 2 && wide) {
     switch (role) {

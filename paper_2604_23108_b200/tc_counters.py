@@ -33,6 +33,8 @@ def main():
     ap.add_argument("--workload", default="cfg5_slice", choices=list(WORKLOADS))
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--gather", action="store_true",
+                    help="use the entry points that gather the rows of x instead of reading x_perm")
     args = ap.parse_args()
     B.LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmohge_counters.so")
     wl = WORKLOADS[args.workload]
@@ -50,8 +52,9 @@ def main():
 
     def step():
         B.layer_forward(cfg, b, inp["x"], inp["w_router"], inp["w13"], inp["w2"],
-                        logit_bias=inp["logit_bias"], aux=True)
-        B.layer_backward(cfg, b, inp["x"], inp["w_router"], inp["w13"], inp["w2"], inp["dy"], aux=True)
+                        logit_bias=inp["logit_bias"], aux=True, gather=args.gather)
+        B.layer_backward(cfg, b, inp["x"], inp["w_router"], inp["w13"], inp["w2"], inp["dy"], aux=True,
+                         gather=args.gather)
 
     for _ in range(args.warmup):
         step()
@@ -69,8 +72,8 @@ def main():
     N = wl.experts_per_group
     rows_w = sum(float(m) * wl.group_width[e // N] for e, m in enumerate(counts))
     cmax, cmin = counts.max(), counts[counts > 0].min()
-    print("workload %s: %.3f ms per step, %.0f tokens/s; tokens per expert min %d max %d (x%.0f)"
-          % (wl.name, ms, wl.T / ms * 1e3, cmin, cmax, cmax / cmin))
+    print("workload %s%s: %.3f ms per step, %.0f tokens/s; tokens per expert min %d max %d (x%.0f)"
+          % (wl.name, " (gathering entry points)" if args.gather else "", ms, wl.T / ms * 1e3, cmin, cmax, cmax / cmin))
     print("| role | CTAs | ms per launch | TFLOP/s | busy min/mean | busy max/mean | clocks per k-block | steady state "
           "| issuer waits for accumulator |")
     print("|---|---|---|---|---|---|---|---|---|")
