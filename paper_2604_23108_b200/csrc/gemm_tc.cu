@@ -90,13 +90,15 @@ constexpr int kStgBytes = 4 * kSlots * kStgBufBytes;         // 64 KiB per CTA
 // bytes per FLOP by a quarter; the price is that the epilogue of an entry no longer overlaps
 // the MMAs of the next one.  It pays where the contraction is long (see launch_tc_grouped).
 // WIDE = 2 (single CTAs, router logits with at most 160 outputs): a B tile of 20 KiB instead of
-// 32, so the same shared memory holds four stages instead of three.  That GEMM streams x once and
-// is bound by the bytes it keeps in flight against the memory latency.
+// 32 and no staging ring (that epilogue stores from registers), so the shared memory holds six
+// stages instead of three.  That GEMM streams x once and is bound by the bytes it keeps in flight
+// against the memory latency.
 template <int CG, int WIDE = 0> struct Geo {
-  static constexpr int kStages = WIDE == 2 ? 4 : (CG == 2 && !WIDE) ? 5 : 3;
+  static constexpr int kStages = WIDE == 2 ? 6 : (CG == 2 && !WIDE) ? 5 : 3;
+  static constexpr int kStg = WIDE == 2 ? 0 : kStgBytes;       // epilogue staging ring
   static constexpr int kBBytes = WIDE == 2 ? 160 * BK * 2 : 256 / CG * BK * 2;   // one B tile per CTA: 32 KiB or 16 KiB
   static constexpr int kStageBytes = kABytes + kBBytes * (WIDE == 1 ? 2 : 1);
-  static constexpr int kSmemBytes = kStages * kStageBytes + kStgBytes + 1024 + 512 + 1088;   // + segment table
+  static constexpr int kSmemBytes = kStages * kStageBytes + kStg + 1024 + 512 + 1088;   // + segment table
   static constexpr int kTileM = BM * CG;
 };
 
@@ -147,6 +149,11 @@ struct TcParams {
   // plain roles: C[M, N] over contraction K; tile ti -> (ti / ntn, ti % ntn)
   int plain_total, plain_ntn, plain_M, plain_N, plain_K;
   int plain_splits, plain_kchunk;   // split-K of ROUTER_DW and LOGITS: ranges of plain_kchunk k-blocks
+  // LOGITS with more row tiles than CTAs: instead of tiles dealt round robin (512 tiles over 148
+  // CTAs leave the last of four rounds half empty) every CTA takes one contiguous range of rows,
+  // the same for all, cut into 128-row tiles and, where 64 rows or fewer remain, a last tile
+  // whose A box is 64 rows high (mapA[1]); the kernel is bound by streaming x once.
+  int plain_balanced;
   float* Cf;                     // LOGITS: logits [T, NL]; ROUTER_DW: dw_router [NL, d]
   const float* bias;             // LOGITS: optional logit bias [NL]
   // DGRAD_DOWN, optional: per physical row and 128-column slot of the hidden axis, the sum over
@@ -456,8 +463,24 @@ struct TileGeom {
   int e, g, i, W, bn, m0, n0, num_kb, r0, wide;
 };
 
+// rows per CTA of the balanced LOGITS form: the same multiple of 64 for every CTA
+__device__ __forceinline__ int balanced_rows(int M, int ctas) { return ((M + ctas - 1) / ctas + 63) / 64 * 64; }
+
 template <int ROLE>
 __device__ __forceinline__ Tile fetch_tile(const TcParams& p, int ti) {
+  if (ROLE == ROLE_LOGITS && p.plain_balanced) {
+    Tile t;
+    const int ctas = (int)gridDim.x, R = balanced_rows(p.plain_M, ctas);
+    const int local = ti / ctas;
+    t.e = 0;
+    t.n0 = 0;
+    t.m0 = (ti % ctas) * R + local * BM;
+    int ext = R - local * BM;
+    if (ext > BM) ext = BM;
+    if (ext > p.plain_M - t.m0) ext = p.plain_M - t.m0;
+    t.ext = ext > 0 ? ext : 0;                             // 0: nothing left for this CTA, tile skipped
+    return t;
+  }
   if (is_plain<ROLE>()) {
     Tile t;
     const int per_m = p.plain_ntn * p.plain_splits;       // tile index = (m, n, split), split fastest
@@ -515,8 +538,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   // layout: pipeline stages | epilogue staging (4 warps x 4 buffers x 4 KiB) | barriers
   const uint32_t stg0 = smem_base + kStages * kStageBytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * kStageBytes + kStgBytes);
-  const uint32_t bar0 = stg0 + kStgBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * kStageBytes + G::kStg);
+  const uint32_t bar0 = stg0 + G::kStg;
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kStages + b); };
@@ -527,7 +550,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   // expert segment table (aligned_offsets) staged once, so that no role chases it through global
   // memory between tiles
-  int32_t* s_seg = reinterpret_cast<int32_t*>(smem_gen + kStages * kStageBytes + kStgBytes + 512);
+  int32_t* s_seg = reinterpret_cast<int32_t*>(smem_gen + kStages * kStageBytes + G::kStg + 512);
   // Programmatic dependent launch (when the host asked for it): the next kernel of the stream may
   // be scheduled onto SMs as the CTAs of this one leave, and this kernel may itself have been
   // scheduled while its predecessor was draining.  Nothing before griddep_wait() below touches
@@ -574,7 +597,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     for (int i = threadIdx.x; i <= ne; i += blockDim.x) s_seg[i] = p.aligned[i];
     __syncthreads();
   }
-  const int total = is_plain<ROLE>() ? p.plain_total : *p.tile_count;
+  const int total = (ROLE == ROLE_LOGITS && p.plain_balanced)
+                        ? (int)gridDim.x * ((balanced_rows(p.plain_M, (int)gridDim.x) + BM - 1) / BM)
+                        : is_plain<ROLE>() ? p.plain_total : *p.tile_count;
   // Tile of this CTA (pair) in round i.  The list is sorted by cost, heaviest first.  When the
   // costs differ (zigzag), rounds alternate direction (0..n-1, then n-1..0), so no CTA always gets
   // the heaviest tile of its round; with equal costs the plain order measured slightly faster.  Returns -1 when the round has no tile left for this CTA (last, partial round).
@@ -740,12 +765,14 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         const Tile t = t_pf;
         t_pf = prefetch_tile(it + it_step);
         if (ti < 0) continue;
+        if (ROLE == ROLE_LOGITS && t.ext == 0) continue;
         const TileGeom q = tile_geom<ROLE>(p, t, s_seg);
-        const CUtensorMap* mA = &p.mapA[q.g];
+        const bool half_a = ROLE == ROLE_LOGITS && p.plain_balanced && t.ext <= 64;   // 64-row A box
+        const CUtensorMap* mA = &p.mapA[half_a ? 1 : q.g];
         const CUtensorMap* mB = &p.mapB[q.g];
         const int nb = q.bn / CG;                          // B rows staged by this CTA per B tile
         const int pieces = (WIDE && q.wide) ? 2 : 1;       // B tiles of this entry
-        const uint32_t tx = kABytes + (uint32_t)pieces * nb * BK * 2;
+        const uint32_t tx = (half_a ? kABytes / 2 : kABytes) + (uint32_t)pieces * nb * BK * 2;
         const int am0 = q.m0 + BM * (int)cta_rank;         // this CTA's 128 rows of the tile
         for (int kb = 0; kb < q.num_kb; ++kb) {
           TCC(const long long w0 = clock64();)
@@ -827,6 +854,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         const Tile t = t_pf;
         t_pf = prefetch_tile(it + it_step);
         if (ti < 0) continue;
+        if (ROLE == ROLE_LOGITS && t.ext == 0) continue;
         const TileGeom q = tile_geom<ROLE>(p, t, s_seg);
         TCC(c_tiles += 1; c_kb += q.num_kb * ((WIDE && q.wide) ? 2 : 1);)
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)RT::A_MN << 15) |
@@ -974,6 +1002,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       const Tile t = t_pf;
       t_pf = prefetch_tile(it + it_step);
       if (ti < 0) continue;
+      if (ROLE == ROLE_LOGITS && t.ext == 0) continue;
       TileGeom q = tile_geom<ROLE>(p, t, s_seg);
       // a double-width entry is drained as two pieces, one accumulator buffer each
       const int pieces = (WIDE && q.wide) ? 2 : 1;
@@ -1289,10 +1318,26 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           tmem_ld_wait();
           if (row_ok) {
             float* po = p.Cf + row * p.plain_N;
+            if ((p.plain_N & 3) == 0) {          // rows are 16-byte aligned: four columns per store
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int n = q.n0 + c + j;
-              if (n < p.plain_N) po[n] = __uint_as_float(r[j]) + (bias ? bias[n] : 0.0f);
+              for (int j = 0; j < 32; j += 4) {
+                const int n = q.n0 + c + j;
+                if (n < p.plain_N) {
+                  float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                         __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                  if (bias) {
+                    const float4 bv = *reinterpret_cast<const float4*>(bias + n);
+                    v.x += bv.x; v.y += bv.y; v.z += bv.z; v.w += bv.w;
+                  }
+                  *reinterpret_cast<float4*>(po + n) = v;
+                }
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const int n = q.n0 + c + j;
+                if (n < p.plain_N) po[n] = __uint_as_float(r[j]) + (bias ? bias[n] : 0.0f);
+              }
             }
           }
         }
@@ -1702,6 +1747,8 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
       p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 15) / 16 * 16;
       dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = BK; box[1] = BM;
       if ((rc = encode_map(&p.mapA[0], A, 2, dims, str, box))) return rc;
+      box[1] = BM / 2;                                     // last tile of a CTA's row range (balanced form)
+      if ((rc = encode_map(&p.mapA[1], A, 2, dims, str, box))) return rc;
       dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = BK; box[1] = p.BN[0];
       if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
     } else if (role == ROLE_ROUTER_DW) {
@@ -1735,6 +1782,8 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
     if (p.plain_splits > 1) p.Cf = partials;
   }
   p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn * p.plain_splits;
+  // more row tiles than CTAs and a single column tile: contiguous row ranges of equal length
+  p.plain_balanced = (role == ROLE_LOGITS && p.plain_splits == 1 && p.plain_ntn == 1 && p.plain_total > di.sm_count) ? 1 : 0;
   switch (role) {
     case ROLE_LOGITS: {
       const int32_t rc2 = p.BN[0] <= 160 ? launch_role<ROLE_LOGITS, 1, 2>(p, di, st)

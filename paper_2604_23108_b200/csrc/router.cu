@@ -206,6 +206,7 @@ router_select_kernel(RouterShape s, const float* __restrict__ logits, int32_t* _
   if (saw_nan && status != nullptr) atomicCAS(status, 0, 3 << 24);
 }
 
+
 // the three count arrays start at zero (one launch instead of three memsets)
 __global__ void zero_counts_kernel(int32_t* group_count, int Ng, int32_t* cnt_routed, int32_t* cnt_lit,
                                    int Ne) {

@@ -257,3 +257,53 @@ def test_gate_that_is_exactly_zero_still_gets_its_gradient(dtype):
     assert np.abs(bwd["dgate"][:, 1]).max() > 0
     assert max_rel(to_np64(b.dgate), bwd["dgate"]) <= tol_for(dtype)
     assert max_rel(to_np64(b.y), fwd["y"]) <= tol_for(dtype)
+
+
+@pytest.mark.parametrize("T", [148 * 128 + 1, 20000, 148 * 192, 33333])
+def test_router_logits_with_more_row_tiles_than_sms(T):
+    """With more 128-row tiles than SMs the logits GEMM gives every CTA one contiguous range of
+    rows, the last tile of a range being 64 rows high: every row must still be computed once,
+    whatever the remainder, and the selection from those logits must be the contract's."""
+    wl = Workload("balanced_logits", "bf16", T, 192, 3, 8, (64, 48, 32), 2, 4, seed=13)
+    inp = make_inputs(wl, weights=False)
+    gcfg, ocfg = gpu_cfg(wl), oracle_cfg(wl)
+    b = B.LayerBuffers(gcfg, T)
+    b.logits.fill_(float("nan"))
+    B.mohge_route(gcfg, T, inp["x"].cuda(), inp["w_router"].cuda(), None, None, b.logits, b.group_idx,
+                  b.expert_idx, b.gate_w, b.gs, b.esp, b.ws)
+    torch.cuda.synchronize()
+    assert B.mohge_get_device_status(b.ws) == 0
+    ref = O.router_logits(to_np64(inp["x"]), to_np64(inp["w_router"]), None)
+    got = b.logits.cpu().numpy()
+    assert np.isfinite(got).all()
+    assert max_rel(got, ref) <= 1e-5
+    s = O.route_spec(ocfg, got)
+    assert (b.group_idx.cpu().numpy() == s["group_idx"]).all()
+    assert (b.expert_idx.cpu().numpy() == s["expert_idx"]).all()
+
+
+@pytest.mark.parametrize("shape", [(3, 4, 2, 5), (4, 32, 2, 8), (8, 32, 3, 20), (2, 7, 2, 14), (1, 1, 1, 1), (5, 3, 5, 15)])
+def test_selection_contract_on_ties_nan_and_underflow(shape):
+    """Indices, gates and saved scores equal the oracle's float32 contract bit for bit on rows
+    full of exact ties, rows where everything ties, NaN group logits, groups of NaN expert logits
+    and scores that underflow to zero (rows whose keys all underflow have 0/0 gates on both sides)."""
+    Ng, N, Kg, Ke = shape
+    wl = Workload("contract_edges", "f32", 1000, 32, Ng, N, tuple([32] * Ng), Kg, Ke, seed=21)
+    gcfg, ocfg = gpu_cfg(wl), oracle_cfg(wl)
+    rng = np.random.default_rng(7)
+    lg = rng.normal(size=(wl.T, wl.n_logits)).astype(np.float32)
+    lg[:100] = np.round(lg[:100] * 2) / 2                  # many exact ties
+    lg[100:110] = 0.0                                      # everything ties
+    lg[110:120, 0] = np.nan                                # NaN group logit
+    lg[120:130, Ng:] = np.nan                              # all expert logits NaN
+    lg[130:140] = -200.0 * (rng.random((10, wl.n_logits)) < 0.5)   # underflowing scores
+    s = O.route_spec(ocfg, lg)
+    b = B.LayerBuffers(gcfg, wl.T)
+    B.mohge_route(gcfg, wl.T, None, None, None, torch.from_numpy(lg).cuda(), None, b.group_idx,
+                  b.expert_idx, b.gate_w, b.gs, b.esp, b.ws)
+    torch.cuda.synchronize()
+    assert (b.group_idx.cpu().numpy() == s["group_idx"]).all()
+    assert (b.expert_idx.cpu().numpy() == s["expert_idx"]).all()
+    assert np.array_equal(b.gate_w.cpu().numpy(), s["gate"], equal_nan=True)
+    assert np.array_equal(b.esp.cpu().numpy(), s["ESp"], equal_nan=True)
+    assert np.array_equal(b.gs.cpu().numpy(), s["GS"], equal_nan=True)
