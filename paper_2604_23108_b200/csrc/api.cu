@@ -71,8 +71,9 @@ int32_t make_dims(const mohge_config* c, int64_t T, Dims* D) {
 }
 
 // ---------------------------------------------------------------- switches
-static const char* const kSwitchName[SW_COUNT] = {"pdl", "tc_cg", "tc_wide", "force_simt"};
-static const char* const kSwitchEnv[SW_COUNT] = {"MOHGE_PDL", "MOHGE_TC_CG", "MOHGE_TC_WIDE", "MOHGE_FORCE_SIMT"};
+static const char* const kSwitchName[SW_COUNT] = {"pdl", "tc_cg", "tc_wide", "force_simt", "route_fused"};
+static const char* const kSwitchEnv[SW_COUNT] = {"MOHGE_PDL", "MOHGE_TC_CG", "MOHGE_TC_WIDE", "MOHGE_FORCE_SIMT",
+                                                   "MOHGE_ROUTE_FUSED"};
 static std::atomic<int> g_switch[SW_COUNT];
 static std::once_flag g_switch_once;
 
@@ -294,9 +295,14 @@ int32_t mohge_route(const mohge_config* cfg, int64_t T, const void* x, const voi
   if (!logits_in) {
     REQ_PTR(x); REQ_PTR(w_router); REQ_PTR(logits_out); OPT_PTR(logit_bias);
     const int f32 = D.bf16 ? 0 : 1;
-    if (D.bf16 && !force_simt())
-      rc = launch_tc_plain(D, ROLE_LOGITS, x, w_router, 0, logits_out, logit_bias, carve(D, ws).rdw, carve(D, ws).status, st);
-    else
+    if (D.bf16 && !force_simt()) {
+      // the tensor-core launch selects in its epilogue when it can (Eq. 2-6 on the accumulator rows)
+      const RouteOut ro = {group_idx, expert_idx, gate_w, gs_saved, esp_saved};
+      bool routed = false;
+      rc = launch_tc_plain(D, ROLE_LOGITS, x, w_router, 0, logits_out, logit_bias, carve(D, ws).rdw,
+                           carve(D, ws).status, st, &ro, &routed);
+      if (rc || routed) return rc;
+    } else
       rc = launch_simt_plain((int)T, D.NL, D.d, x, f32, D.d, 1, w_router, f32, D.d, 1, logits_out, 1,
                              D.NL, logit_bias, 0, st);
     if (rc) return rc;

@@ -56,7 +56,7 @@ bool dependent_launch();   // false when the "pdl" switch is 0
 // Debugging switches.  Each is read ONCE from its environment variable, the first time any
 // switch is asked for, and can afterwards be changed only through mohge_set_switch(); -1 means
 // "not set: the library's own rule decides".
-enum Switch { SW_PDL = 0, SW_TC_CG = 1, SW_TC_WIDE = 2, SW_FORCE_SIMT = 3, SW_COUNT = 4 };
+enum Switch { SW_PDL = 0, SW_TC_CG = 1, SW_TC_WIDE = 2, SW_FORCE_SIMT = 3, SW_ROUTE_FUSED = 4, SW_COUNT = 5 };
 int switch_value(int which);
 // What the launchers need to know about the current device, looked up once per device ordinal
 // (a process may drive several GPUs; kernel attributes such as the dynamic shared-memory limit
@@ -231,7 +231,18 @@ int32_t launch_build_tiles_multi(const TilePlan* plans, int nplans, const int32_
                                  int32_t* tile_count, Tile* tiles, int64_t tiles_cap,
                                  int32_t* status, cudaStream_t st);
 
+// Outputs of the selection (Eq. 2-6) for the LOGITS launch that selects in its epilogue.
+struct RouteOut {
+  int32_t* group_idx;
+  int32_t* expert_idx;
+  float* gate_w;
+  float* gs;
+  float* esp;
+};
+// route != nullptr (LOGITS only): the launch may also do the selection; *routed says whether it did
+// (it does when the shape is covered, the contraction is not split and the switch is not 0).
 int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
-                        void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st);
+                        void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st,
+                        const RouteOut* route = nullptr, bool* routed = nullptr);
 
 }  // namespace mohge

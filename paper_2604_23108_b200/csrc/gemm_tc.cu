@@ -40,6 +40,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "route_epilogue.cuh"
 
 namespace mohge {
 namespace {
@@ -57,6 +58,11 @@ constexpr int kThreads = 192;                 // producer, MMA issuer, four epil
 #endif
 constexpr int kGatherWarps = MOHGE_GATHER_WARPS;     // 1, 2 or 4
 constexpr int kThreadsGather = kThreads + 32 * kGatherWarps;
+// router-logits GEMM in its six-stage form: kRouteSplit epilogue warps per quarter of the rows
+constexpr int kThreadsRoute = 64 + 128 * kRouteSplit;
+template <int ROLE, int WIDE, int GATHER> __host__ __device__ constexpr int block_threads() {
+  return GATHER ? kThreadsGather : (ROLE == ROLE_LOGITS && WIDE == 2) ? kThreadsRoute : kThreads;
+}
 constexpr int kAccCols = 256;                 // tensor-memory columns per accumulator buffer
 
 // Build-time option -DMOHGE_TC_COUNTERS: every CTA adds, per role, the clocks its MMA issuer spent
@@ -95,7 +101,8 @@ constexpr int kStgBytes = 4 * kSlots * kStgBufBytes;         // 64 KiB per CTA
 // against the memory latency.
 template <int CG, int WIDE = 0> struct Geo {
   static constexpr int kStages = WIDE == 2 ? 6 : (CG == 2 && !WIDE) ? 5 : 3;
-  static constexpr int kStg = WIDE == 2 ? 0 : kStgBytes;       // epilogue staging ring
+  // epilogue staging ring; six-stage form: the lists the epilogue warps of a row quarter exchange
+  static constexpr int kStg = WIDE == 2 ? (kRouteSplit - 1) * 128 * 2 * kRouteFuseMaxKe * 4 : kStgBytes;
   static constexpr int kBBytes = WIDE == 2 ? 160 * BK * 2 : 256 / CG * BK * 2;   // one B tile per CTA: 32 KiB or 16 KiB
   static constexpr int kStageBytes = kABytes + kBBytes * (WIDE == 1 ? 2 : 1);
   static constexpr int kSmemBytes = kStages * kStageBytes + kStg + 1024 + 512 + 1088;   // + segment table
@@ -155,6 +162,7 @@ struct TcParams {
   // whose A box is 64 rows high (mapA[1]); the kernel is bound by streaming x once.
   int plain_balanced;
   float* Cf;                     // LOGITS: logits [T, NL]; ROUTER_DW: dw_router [NL, d]
+  RouteFuse rf;                  // LOGITS: selection (Eq. 2-6) in the epilogue; B staged experts first
   const float* bias;             // LOGITS: optional logit bias [NL]
   // DGRAD_DOWN, optional: per physical row and 128-column slot of the hidden axis, the sum over
   // the tile's columns of dH_j * h_j (the gate gradient times the gate, see dgate_reduce_kernel)
@@ -269,6 +277,14 @@ __device__ __forceinline__ uint32_t stg_addr(uint32_t buf, int r, int j) {
 }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void st_shared_u32(uint32_t addr, uint32_t x) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(x) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
 }
 __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
   uint4 v;
@@ -525,7 +541,7 @@ __device__ __forceinline__ TileGeom tile_geom(const TcParams& p, const Tile& t, 
 }
 
 template <int ROLE, int CG, int WIDE, int GATHER = 0>
-__global__ void __launch_bounds__(GATHER ? kThreadsGather : kThreads, 1)
+__global__ void __launch_bounds__(block_threads<ROLE, WIDE, GATHER>(), 1)
 tc_grouped_kernel(const __grid_constant__ TcParams p) {
   using RT = RoleTraits<ROLE>;
   using G = Geo<CG, WIDE>;
@@ -570,7 +586,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), 4 * CG);  // four epilogue warps per CTA
+      mbar_init(tempty_bar(b), (block_threads<ROLE, WIDE, GATHER>() == kThreadsRoute ? 4 * kRouteSplit : 4) * CG);  // every epilogue warp
     }
     for (int i = 0; i < 8; ++i) mbar_init(ein_bar(i >> 1, i & 1), 1);   // epilogue input loads
     *abort_flag = 0;
@@ -807,7 +823,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             } else {
               const int bn0 = q.n0 + pc * q.bn + nb * (int)cta_rank;   // this CTA's slice of the columns
               if (ROLE == ROLE_LOGITS) {
-                tma_2d<CG>(sB, mB, fb, q.r0 + k0, bn0);
+                if (p.rf.on) {     // expert rows of the router weight first, the group rows behind them
+                  const int ne = p.rf.Ng * p.rf.N;
+                  tma_2d<CG>(sB, &p.mapB[0], fb, q.r0 + k0, p.rf.Ng);
+                  tma_2d<CG>(sB + ne * 128, &p.mapB[1], fb, q.r0 + k0, 0);
+                } else {
+                  tma_2d<CG>(sB, mB, fb, q.r0 + k0, bn0);
+                }
               } else if (ROLE == ROLE_FWD2) {
                 tma_3d<CG>(sB, mB, fb, k0, bn0, q.i);
               } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
@@ -987,6 +1009,8 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   } else {
     // ================= epilogue warps =================
     const int quad = warp & 3;                 // tensor-memory lanes [32*quad, 32*quad + 32)
+    const int split = (GATHER ? 0 : (warp - 2) >> 2);   // > 0 only with kThreadsRoute threads
+    uint32_t list_phase = 0;
     const int row_in_tile = BM * (int)cta_rank + quad * 32 + lane;   // row of the (pair's) tile
     const uint32_t stg = stg0 + (uint32_t)quad * (kSlots * kStgBufBytes);   // this warp's staging ring
     uint32_t n_store = 0;                      // stores issued so far: ring slot = n_store % 4
@@ -1312,6 +1336,49 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         const long long row = q.m0 + row_in_tile + (long long)q.e * p.plain_M;
         const bool row_ok = row_in_tile < t.ext;
         const float* bias = p.plain_splits == 1 ? p.bias : nullptr;
+        if (p.rf.on) {
+          RouteList L;
+          bool nan = false;
+          switch (p.rf.N) {
+            case 4: nan = route_token_groups<4>(p.rf, taddr, row_ok, row, p.Cf, bias, split, L); break;
+            case 8: nan = route_token_groups<8>(p.rf, taddr, row_ok, row, p.Cf, bias, split, L); break;
+            case 16: nan = route_token_groups<16>(p.rf, taddr, row_ok, row, p.Cf, bias, split, L); break;
+            default: nan = route_token_groups<32>(p.rf, taddr, row_ok, row, p.Cf, bias, split, L); break;
+          }
+          release_acc();
+          if (nan && row_ok && p.status != nullptr) atomicCAS(p.status, 0, 3 << 24);
+          // The lists of the other warps of this row quarter arrive through shared memory: word
+          // (2 k + which) * 128 + row of the area of split s holds entry k of that row.  One
+          // barrier says "written" (ein_bar(quad, 0)), one "read" (ein_bar(quad, 1)).
+          const uint32_t area = stg0 + (uint32_t)(quad * 32 + lane) * 4u;
+          if (split > 0) {
+            const bool ok = mbar_wait(ein_bar(quad, 1), list_phase ^ 1u, abort_flag, p.status, 8);
+            if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+#pragma unroll
+            for (int k = 0; k < kRouteFuseMaxKe; ++k) {
+              st_shared_u32(area + (2 * k) * 512u, __float_as_uint(L.wk[k]));
+              st_shared_u32(area + (2 * k + 1) * 512u, (uint32_t)L.we[k]);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ein_bar(quad, 0));
+          } else {
+            if (kRouteSplit > 1 && block_threads<ROLE, WIDE, GATHER>() == kThreadsRoute) {
+              const bool ok = mbar_wait(ein_bar(quad, 0), list_phase, abort_flag, p.status, 8);
+              if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+              RouteList O;
+#pragma unroll
+              for (int k = 0; k < kRouteFuseMaxKe; ++k) {
+                O.wk[k] = __uint_as_float(ld_shared_u32(area + (2 * k) * 512u));
+                O.we[k] = (int)ld_shared_u32(area + (2 * k + 1) * 512u);
+              }
+              __syncwarp();
+              if (lane == 0) mbar_arrive(ein_bar(quad, 1));
+              route_list_merge(L, O);
+            }
+            route_token_finish(p.rf, row_ok, row, L);
+          }
+          list_phase ^= 1u;
+        } else if (split == 0)
         for (int c = 0; c < q.bn; c += 32) {
           uint32_t r[32];
           tmem_ld32(taddr + c, r);
@@ -1583,7 +1650,7 @@ int32_t launch_role(const TcParams& p, const DeviceInfo& di, cudaStream_t st) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.gridDim = dim3(grid / CG * CG);
-  cfg.blockDim = dim3(GATHER ? kThreadsGather : kThreads);
+  cfg.blockDim = dim3(block_threads<ROLE, WIDE, GATHER>());
   cfg.dynamicSmemBytes = Geo<CG, WIDE>::kSmemBytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -1708,7 +1775,9 @@ int router_logits_splits(const Dims& D, int n_tiles) {
 }  // namespace
 
 int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, int64_t b_pitch_elems,
-                        void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st) {
+                        void* C, const float* bias, float* partials, int32_t* status, cudaStream_t st,
+                        const RouteOut* route, bool* routed) {
+  if (routed) *routed = false;
   if (D.T == 0) return MOHGE_OK;
   DeviceInfo di;
   int32_t rcd = current_device(&di);
@@ -1737,10 +1806,19 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
     p.plain_M = (int)T; p.plain_N = D.d; p.plain_K = D.NL;
     p.C = (__nv_bfloat16*)C;
   }
+  // LOGITS: selection in the epilogue when the shape is one route_token covers, the logits fit the
+  // six-stage form (one column tile of at most 160) and the contraction is not split
+  bool fuse = false;
+  if (role == ROLE_LOGITS && route != nullptr && switch_value(SW_ROUTE_FUSED) != 0) {
+    const int bn = (D.NL + 15) / 16 * 16;
+    const bool shape_ok = (D.N == 4 || D.N == 8 || D.N == 16 || D.N == 32) && D.Ne % 8 == 0 && bn <= 160 &&
+                          D.Ke <= kRouteFuseMaxKe && D.Ke <= D.Kg * D.N;
+    fuse = shape_ok && (partials == nullptr || router_logits_splits(D, 1) == 1);
+  }
   // tensor maps: from the cache, or encoded now
   MapKey key;
   memset(&key, 0, sizeof(key));
-  key.role = role; key.cg = 1; key.device = di.ordinal; key.d = D.d; key.Ng = D.Ng; key.N = D.N;
+  key.role = role; key.cg = 1; key.accumulate_unused = fuse ? 1 : 0; key.device = di.ordinal; key.d = D.d; key.Ng = D.Ng; key.N = D.N;
   key.T = D.T; key.b_pitch = b_pitch_elems; key.A = A; key.B = B; key.C = C;
   if (!map_cache_find(key, &p)) {
     if (role == ROLE_LOGITS) {
@@ -1750,7 +1828,14 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
       box[1] = BM / 2;                                     // last tile of a CTA's row range (balanced form)
       if ((rc = encode_map(&p.mapA[1], A, 2, dims, str, box))) return rc;
       dims[0] = d; dims[1] = NL; str[0] = d * 2; box[0] = BK; box[1] = p.BN[0];
-      if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+      if (fuse) {            // two boxes: the Ne expert rows (from row Ng), then the group rows (from row 0)
+        box[1] = D.Ne;
+        if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+        box[1] = p.BN[0] - D.Ne;
+        if ((rc = encode_map(&p.mapB[1], B, 2, dims, str, box))) return rc;
+      } else {
+        if ((rc = encode_map(&p.mapB[0], B, 2, dims, str, box))) return rc;
+      }
     } else if (role == ROLE_ROUTER_DW) {
       p.BN[0] = D.NL >= 256 ? 256 : (D.NL + 63) / 64 * 64;
       dims[0] = d; dims[1] = T; str[0] = d * 2; box[0] = 64; box[1] = BK;
@@ -1784,6 +1869,12 @@ int32_t launch_tc_plain(const Dims& D, int role, const void* A, const void* B, i
   p.plain_total = ((p.plain_M + BM - 1) / BM) * p.plain_ntn * p.plain_splits;
   // more row tiles than CTAs and a single column tile: contiguous row ranges of equal length
   p.plain_balanced = (role == ROLE_LOGITS && p.plain_splits == 1 && p.plain_ntn == 1 && p.plain_total > di.sm_count) ? 1 : 0;
+  if (fuse) {
+    p.rf.on = 1; p.rf.Ng = D.Ng; p.rf.N = D.N; p.rf.Kg = D.Kg; p.rf.Ke = D.Ke;
+    p.rf.group_idx = route->group_idx; p.rf.expert_idx = route->expert_idx; p.rf.gate_w = route->gate_w;
+    p.rf.gs = route->gs; p.rf.esp = route->esp;
+    if (routed) *routed = true;
+  }
   switch (role) {
     case ROLE_LOGITS: {
       const int32_t rc2 = p.BN[0] <= 160 ? launch_role<ROLE_LOGITS, 1, 2>(p, di, st)

@@ -31,37 +31,12 @@
 // lowest expert id.
 
 #include "common.cuh"
+#include "select_math.cuh"
 
 namespace mohge {
 namespace {
 
 constexpr unsigned kFull = 0xffffffffu;
-
-__device__ __forceinline__ float exp_s(float z) {
-  const float zc = fmaxf(z, -100.0f);
-  const float n = rintf(__fmul_rn(zc, 0x1.715476p+0f));
-  float r = __fsub_rn(zc, __fmul_rn(n, 0x1.62e4p-1f));
-  r = __fsub_rn(r, __fmul_rn(n, 0x1.7f7d1cp-20f));
-  float p = 0x1.a01a02p-13f;
-  p = __fadd_rn(__fmul_rn(p, r), 0x1.6c16c2p-10f);
-  p = __fadd_rn(__fmul_rn(p, r), 0x1.111112p-7f);
-  p = __fadd_rn(__fmul_rn(p, r), 0x1.555556p-5f);
-  p = __fadd_rn(__fmul_rn(p, r), 0x1.555556p-3f);
-  p = __fadd_rn(__fmul_rn(p, r), 0x1p-1f);
-  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
-  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
-  int ni = (int)n;
-  ni = ni < -126 ? -126 : (ni > 0 ? 0 : ni);
-  const float scale = __int_as_float((ni + 127) << 23);
-  const float out = __fmul_rn(p, scale);
-  return z < -87.0f ? 0.0f : out;
-}
-
-__device__ __forceinline__ float sig_s(float z) {
-  const float e = exp_s(-fabsf(z));
-  const float den = __fadd_rn(1.0f, e);
-  return z >= 0.0f ? __fdiv_rn(1.0f, den) : __fdiv_rn(e, den);
-}
 
 // Order-preserving map float -> unsigned (a < b  <=>  ord_key(a) < ord_key(b), no NaNs here) and
 // its inverse, so that one integer warp reduction finds the largest key.
