@@ -12,11 +12,10 @@
 //   * the B operand of the GEMM is staged with the expert rows of the router weight first and
 //     the group rows behind them, so that group g's N logits are the accumulator columns
 //     [g N, g N + N) (aligned to N, a power of two) and the group logits the columns [Ne, Ne + Ng);
-//   * tensor memory is read with the same column address by the whole warp, so a warp walks
-//     groups and a thread works on those it selected;
-//   * kRouteSplit warps share a quarter of the accumulator rows: warp s of them takes the groups
-//     g = s (mod kRouteSplit) and keeps its own sorted list; the lists meet in shared memory and
-//     are merged by (key descending, id ascending), which is the order one list would have had.
+//   * kRouteSplit warps share a quarter of the accumulator rows: warp s of them takes, for each
+//     of its tokens, the selected groups of rank s (mod kRouteSplit) and keeps its own sorted list;
+//     the lists meet in shared memory and are merged by (key descending, id ascending), which is
+//     the order one list would have had.
 // Covered shapes: N a power of two from 4 to 32 (then the padded slot count P of the contract
 // equals N), Ne a multiple of 8, K_e <= 8.  Everything else takes the two-kernel route.
 #pragma once
@@ -77,8 +76,9 @@ struct RouteList {
 
 // Part of one token (row `t` of the batch, accumulator row of this thread at tensor-memory address
 // taddr) done by warp `split` of the kRouteSplit that share the row: group logits and Eq. 2 (every
-// split computes them, split 0 stores them), then for the groups g = split (mod kRouteSplit) the
-// logits (+ bias) to memory, Eq. 3-4 and the candidates of Eq. 5 into L.  Every lane of the warp
+// split computes them, split 0 stores them), then the expert logits (+ bias) of the groups
+// g = split (mod kRouteSplit) to memory and, for the token's selected groups of rank = split
+// (mod kRouteSplit), Eq. 3-4 and the candidates of Eq. 5 into L.  Every lane of the warp
 // must call (the tensor-memory loads are warp-collective); lanes with !row_ok store nothing.
 // Returns true when a NaN logit was met.
 template <int N>
@@ -131,76 +131,110 @@ __device__ __forceinline__ bool route_token_groups(const RouteFuse& f, uint32_t 
     for (int g = 0; g < MOHGE_MAX_GROUPS; ++g)
       if (g < Ng) f.gs[t * Ng + g] = sig_s(lg[g]);
   }
-  // ---- Eq. 3-5, the groups of this split
+  // ---- Eq. 3-5: this split takes the selected groups of rank split, split + kRouteSplit, ...
+  // (ascending group order).  Which group that is differs from thread to thread while tensor
+  // memory is read with one column address per warp, so the warp reads every group and a thread
+  // keeps the logits of its own; after that no thread works on a group it did not select.
 #pragma unroll
   for (int k = 0; k < kRouteFuseMaxKe; ++k) { L.wk[k] = -1.0f; L.we[k] = -1; }
   float* const pe = f.esp + t * Ne;
-  for (int g = split; g < Ng; g += kRouteSplit) {
-    uint32_t r[N];
-    tmem_ld_cols<N>(taddr + g * N, r);
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-    float l[N];
-    const float* bg = bias ? bias + Ng + g * N : nullptr;
+  if (split >= f.Kg) {          // no selected group falls to this split: only its share of the logits
+    for (int g = split; g < Ng; g += kRouteSplit) {
+      uint32_t r[N];
+      tmem_ld_cols<N>(taddr + g * N, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      const float* bg = bias ? bias + Ng + g * N : nullptr;
+      if (row_ok) {
+        float* pl = po + Ng + g * N;
 #pragma unroll
-    for (int i = 0; i < N; ++i) {
-      l[i] = __uint_as_float(r[i]);
-      if (bg) l[i] += bg[i];
-    }
-    if (row_ok) {
-      float* pl = po + Ng + g * N;
-      if (vec) {
-#pragma unroll
-        for (int i = 0; i < N; i += 4) *reinterpret_cast<float4*>(pl + i) = make_float4(l[i], l[i + 1], l[i + 2], l[i + 3]);
-      } else {
-#pragma unroll
-        for (int i = 0; i < N; ++i) pl[i] = l[i];
-      }
-    }
-    const bool sel = (gmask >> g) & 1u;
-    float lgg = 0.0f;                          // logit of group g (register array, static indices only)
-#pragma unroll
-    for (int gg = 0; gg < MOHGE_MAX_GROUPS; ++gg) lgg = gg == g ? lg[gg] : lgg;
-    float es[N];
-#pragma unroll
-    for (int i = 0; i < N; ++i) es[i] = 0.0f;  // ES' of the experts of unselected groups is 0 (Eq. 3)
-    if (sel) {
-      const float sgv = sig_s(lgg);
-      float m = -INFINITY;
-#pragma unroll
-      for (int i = 0; i < N; ++i) { l[i] = clean(l[i]); m = fmaxf(m, l[i]); }
-      float pr[N], tr[N];
-#pragma unroll
-      for (int i = 0; i < N; ++i) { pr[i] = exp_s(__fsub_rn(l[i], m)); tr[i] = pr[i]; }
-      // balanced binary tree, neighbours first
-#pragma unroll
-      for (int w = N; w > 1; w >>= 1) {
-#pragma unroll
-        for (int i = 0; i < (w >> 1); ++i) tr[i] = __fadd_rn(tr[2 * i], tr[2 * i + 1]);
-      }
-      const float S = tr[0];
-      const float rr = __fdiv_rn(sgv, S);
-#pragma unroll
-      for (int i = 0; i < N; ++i) {
-        es[i] = __fdiv_rn(pr[i], S);
-        const float ck = __fmul_rn(pr[i], rr);
-        const int ce = g * N + i;
-        // ids ascend inside a split's walk, so a strict comparison keeps ties in id order
-#pragma unroll
-        for (int k = kRouteFuseMaxKe - 1; k >= 0; --k) {
-          const bool gt = ck > L.wk[k];
-          if (k + 1 < kRouteFuseMaxKe) {
-            L.wk[k + 1] = gt ? L.wk[k] : L.wk[k + 1];
-            L.we[k + 1] = gt ? L.we[k] : L.we[k + 1];
-          }
-          L.wk[k] = gt ? ck : L.wk[k];
-          L.we[k] = gt ? ce : L.we[k];
+        for (int i = 0; i < N; ++i) {
+          float v = __uint_as_float(r[i]);
+          if (bg) v += bg[i];
+          pl[i] = v;
         }
       }
     }
+  }
+  for (int rk = split; rk < f.Kg; rk += kRouteSplit) {
+    const int gt = (int)__fns(gmask, 0, rk + 1);       // position of the (rk + 1)-th set bit
+    float l[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) l[i] = 0.0f;
+    float lgg = 0.0f;                                   // group logit of gt
+    for (int g = 0; g < Ng; ++g) {
+      uint32_t r[N];
+      tmem_ld_cols<N>(taddr + g * N, r);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      const float* bg = bias ? bias + Ng + g * N : nullptr;
+      float v[N];
+#pragma unroll
+      for (int i = 0; i < N; ++i) {
+        v[i] = __uint_as_float(r[i]);
+        if (bg) v[i] += bg[i];
+      }
+      // the logits of group g are stored once: by the split g falls to, in its first pass
+      if (row_ok && rk == split && (g % kRouteSplit) == split) {
+        float* pl = po + Ng + g * N;
+        if (vec) {
+#pragma unroll
+          for (int i = 0; i < N; i += 4) *reinterpret_cast<float4*>(pl + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < N; ++i) pl[i] = v[i];
+        }
+      }
+      const bool mine = g == gt;
+#pragma unroll
+      for (int i = 0; i < N; ++i) l[i] = mine ? v[i] : l[i];
+#pragma unroll
+      for (int gg = 0; gg < MOHGE_MAX_GROUPS; ++gg) lgg = (mine && gg == g) ? lg[gg] : lgg;
+    }
+    const float sgv = sig_s(lgg);
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < N; ++i) { l[i] = clean(l[i]); m = fmaxf(m, l[i]); }
+    float pr[N], tr[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) { pr[i] = exp_s(__fsub_rn(l[i], m)); tr[i] = pr[i]; }
+    // balanced binary tree, neighbours first
+#pragma unroll
+    for (int w = N; w > 1; w >>= 1) {
+#pragma unroll
+      for (int i = 0; i < (w >> 1); ++i) tr[i] = __fadd_rn(tr[2 * i], tr[2 * i + 1]);
+    }
+    const float S = tr[0];
+    const float rr = __fdiv_rn(sgv, S);
+    float es[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      es[i] = __fdiv_rn(pr[i], S);
+      const float ck = __fmul_rn(pr[i], rr);
+      const int ce = gt * N + i;
+      // ids ascend inside a split's walk, so a strict comparison keeps ties in id order
+#pragma unroll
+      for (int k = kRouteFuseMaxKe - 1; k >= 0; --k) {
+        const bool gt_k = ck > L.wk[k];
+        if (k + 1 < kRouteFuseMaxKe) {
+          L.wk[k + 1] = gt_k ? L.wk[k] : L.wk[k + 1];
+          L.we[k + 1] = gt_k ? L.we[k] : L.we[k + 1];
+        }
+        L.wk[k] = gt_k ? ck : L.wk[k];
+        L.we[k] = gt_k ? ce : L.we[k];
+      }
+    }
     if (row_ok) {
-      float* ps = pe + g * N;
+      float* ps = pe + gt * N;
 #pragma unroll
       for (int i = 0; i < N; i += 4) *reinterpret_cast<float4*>(ps + i) = make_float4(es[i], es[i + 1], es[i + 2], es[i + 3]);
+    }
+  }
+  // ES' of the experts of unselected groups is 0 (Eq. 3): the splits share those groups too
+  if (row_ok) {
+    const unsigned zmask = ~gmask & ((1u << Ng) - 1u);
+    for (int j = split; j < Ng - f.Kg; j += kRouteSplit) {
+      float* ps = pe + (int)__fns(zmask, 0, j + 1) * N;
+#pragma unroll
+      for (int i = 0; i < N; i += 4) *reinterpret_cast<float4*>(ps + i) = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
     }
   }
   return saw_nan;
