@@ -119,9 +119,10 @@ int32_t mohge_get_device_status(const void* ws, int32_t* host_out, void* stream)
 /* Debugging switches (no paper counterpart).  Names: "pdl" (0: launch without programmatic
  * dependent launch), "tc_cg" (1 | 2: force single CTAs or CTA pairs in the grouped GEMMs),
  * "tc_wide" (bit mask over the six expert GEMM roles: force double-width entries per role),
- * "force_simt" (1: run the BF16 GEMMs on the FP32-FMA kernel).  -1 = not set, the library's own
+ * "force_simt" (1: run the BF16 GEMMs on the FP32-FMA kernel), "route_fused" (0: mohge_route
+ * always runs the logits GEMM and the selection as two kernels).  -1 = not set, the library's own
  * rule decides.  Each switch is read ONCE from its environment variable (MOHGE_PDL, MOHGE_TC_CG,
- * MOHGE_TC_WIDE, MOHGE_FORCE_SIMT) when a switch is first consulted; later changes of the
+ * MOHGE_TC_WIDE, MOHGE_FORCE_SIMT, MOHGE_ROUTE_FUSED) when a switch is first consulted; later changes of the
  * environment are not seen, mohge_set_switch is the only way to change a switch afterwards.
  * mohge_get_switch returns INT32_MIN for an unknown name.  HOST. */
 int32_t mohge_get_switch(const char* name);

@@ -9,7 +9,8 @@ Runs forward + backward of the layer with libmohge_counters.so (the library comp
   * the balance of the tile scheduler: shortest and longest CTA busy time over the mean,
   * clocks per k-block (one 256 x 256 x 64 block of MMAs; 512 = tensor-pipe peak) over the whole
     launch and in the middle of long tiles (steady state),
-  * the share of the MMA issuer's time spent waiting for an accumulator (exposed epilogue).
+  * the share of the MMA issuer's time spent waiting for an accumulator (exposed epilogue) and for
+    operands (loads not keeping up), and the share of the epilogue warps' time spent waiting for MMAs.
 MOHGE_TC_WIDE=<mask>, MOHGE_TC_CG=1|2 and MOHGE_TC_GRID=<n> select tile forms and the number of CTAs.
 """
 from __future__ import annotations
@@ -75,8 +76,8 @@ def main():
     print("workload %s%s: %.3f ms per step, %.0f tokens/s; tokens per expert min %d max %d (x%.0f)"
           % (wl.name, " (gathering entry points)" if args.gather else "", ms, wl.T / ms * 1e3, cmin, cmax, cmax / cmin))
     print("| role | CTAs | ms per launch | TFLOP/s | busy min/mean | busy max/mean | clocks per k-block | steady state "
-          "| issuer waits for accumulator |")
-    print("|---|---|---|---|---|---|---|---|---|")
+          "| issuer waits for accumulator | issuer waits for operands | epilogue warps wait for MMAs |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|")
     total_ms = 0.0
     for r in range(9):
         c = cnt[r].astype(np.float64)
@@ -93,9 +94,11 @@ def main():
             total_ms += kern_ms
         kb = c[lead, 9].sum()
         steady = "%.0f" % (c[lead, 10].sum() / c[lead, 11].sum()) if c[lead, 11].sum() > 0 else ""
-        print("| %s | %d | %.3f | %s | %.3f | %.3f | %.0f | %s | %.1f %% |"
+        epi = c[act, 6].sum()
+        print("| %s | %d | %.3f | %s | %.3f | %.3f | %.0f | %s | %.1f %% | %.1f %% | %.1f %% |"
               % (ROLES[r], int(act.sum()), kern_ms, tf, busy.min() / busy.mean(), busy.max() / busy.mean(),
-                 busy.sum() / kb if kb else 0.0, steady, 100.0 * c[lead, 3].sum() / busy.sum()))
+                 busy.sum() / kb if kb else 0.0, steady, 100.0 * c[lead, 3].sum() / busy.sum(),
+                 100.0 * c[lead, 2].sum() / busy.sum(), 100.0 * c[act, 5].sum() / epi if epi else 0.0))
     print("six expert GEMMs: %.3f ms per step = %.0f TFLOP/s" % (total_ms, 18.0 * wl.d_model * rows_w / (total_ms * 1e-3) / 1e12))
 
 
