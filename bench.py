@@ -283,8 +283,8 @@ def hbm_step_rooflines(B, gcfg, wl: Workload, inp, buf, hbm_peak_gbs: float, rep
     """CUDA-event time of every HBM-bound entry point of the step, each called `reps` times back
     to back on the buffers a full step has left behind, against its algorithmic bytes
     (s = bytes per element, R = T K_e routed rows, NL = N_g + N_e router outputs):
-      route         x and the router weight read once, logits written and read, scores, indices
-                    and gates written: T d s + NL d s + 3 T NL 4 + T (8 K_e + 4 K_g)
+      route         x and the router weight read once, logits, scores, indices and gates
+                    written: T d s + NL d s + 2 T NL 4 + T (8 K_e + 4 K_g)
       aux_stats     saved scores and indices read: T NL 4 + T (K_e + K_g) 4
       dispatch      (T + R) d s + 16 R (index arrays)
       combine       (R + T) d s          combine_bwd (scaled rows)  (T + R) d s
@@ -297,7 +297,7 @@ def hbm_step_rooflines(B, gcfg, wl: Workload, inp, buf, hbm_peak_gbs: float, rep
     calls = {
         "route": (lambda: B.mohge_route(gcfg, T, inp["x"], inp["w_router"], inp["logit_bias"], None, buf.logits,
                                         buf.group_idx, buf.expert_idx, buf.gate_w, buf.gs, buf.esp, buf.ws),
-                  T * d * s_ + NL * d * s_ + 3 * T * NL * 4 + T * (8 * Ke + 4 * Kg)),
+                  T * d * s_ + NL * d * s_ + 2 * T * NL * 4 + T * (8 * Ke + 4 * Kg)),
         "aux_stats": (lambda: B.mohge_aux_stats(gcfg, T, buf.gs, buf.esp, buf.group_idx, buf.expert_idx,
                                                 buf.group_count, buf.group_psum, buf.cnt_routed, buf.cnt_lit,
                                                 buf.expert_psum, buf.loss, buf.ws),

@@ -83,9 +83,17 @@ dispatch_scan_kernel(int chunks, int Ne, int align, const int32_t* __restrict__ 
   const int e = threadIdx.x;
   if (e < Ne) {
     int run = 0;
-    for (int b = 0; b < chunks; ++b) {
-      base[(size_t)b * Ne + e] = run;
-      run += hist[(size_t)b * Ne + e];
+    // sixteen counts are requested before the first is used: one dependent load per chunk kept
+    // this single block at a memory round trip per chunk (22 us for 256 chunks)
+    for (int b0 = 0; b0 < chunks; b0 += 16) {
+      int h[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) h[j] = b0 + j < chunks ? hist[(size_t)(b0 + j) * Ne + e] : 0;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        if (b0 + j < chunks) base[(size_t)(b0 + j) * Ne + e] = run;
+        run += h[j];
+      }
     }
     counts[e] = run;
     s_cnt[e] = run;
