@@ -219,15 +219,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return true;
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(pol) : "memory");
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(pol) : "memory");
 }
 
 // L2 eviction priorities.  Epilogue outputs are written once and not read again by the same
@@ -244,6 +244,22 @@ __device__ __forceinline__ uint64_t l2_policy_evict_last() {
   return p;
 }
 
+__device__ __forceinline__ uint64_t l2_policy_evict_normal() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+// Operand loads.  An expert's weights (B of the forward and dgrad roles) are needed again by every
+// row tile of the expert, i.e. by several waves of CTAs, while 30 MB of outputs and the other
+// operand stream through L2 in between; so are both operand slabs of the weight-gradient roles
+// (each is shared by the tiles of a whole output row or column).  Marked evict-last they stay:
+// measured at the large workload, step 45.5 -> 44.8 ms (four runs each, same GPU); the
+// activation operand of the forward and dgrad roles marked evict-first instead cost 1.2 ms, marked
+// evict-last it changed nothing.
+template <int ROLE> __device__ __forceinline__ uint64_t operand_policy(int operand_b) {
+  const bool keep = ROLE == ROLE_WGRAD_DOWN || ROLE == ROLE_WGRAD_13 || (ROLE <= ROLE_DGRAD_13 && operand_b);
+  return keep ? l2_policy_evict_last() : l2_policy_evict_normal();
+}
 // ---- TMA stores from the epilogue staging buffers (bulk async-groups)
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1, uint64_t pol) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
@@ -319,25 +335,25 @@ __device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t bar_cluster
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
 }
 // loads of the pair signal the barrier of the leader CTA (cluster address)
-__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(pol) : "memory");
 }
-__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
+__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(pol) : "memory");
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
 }
-__device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+__device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol) : "memory");
 }
 // 16 bytes global -> shared, asynchronously, no registers in between (src_bytes = 0 writes zeros)
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
@@ -349,16 +365,16 @@ __device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 template <int CG>
-__device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
-  if (CG == 2) tma2_load_4d(dst, map, bar, c0, c1, c2, c3); else tma_load_4d(dst, map, bar, c0, c1, c2, c3);
+__device__ __forceinline__ void tma_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, uint64_t pol) {
+  if (CG == 2) tma2_load_4d(dst, map, bar, c0, c1, c2, c3, pol); else tma_load_4d(dst, map, bar, c0, c1, c2, c3, pol);
 }
 template <int CG>
-__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  if (CG == 2) tma2_load_2d(dst, map, bar, c0, c1); else tma_load_2d(dst, map, bar, c0, c1);
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, uint64_t pol) {
+  if (CG == 2) tma2_load_2d(dst, map, bar, c0, c1, pol); else tma_load_2d(dst, map, bar, c0, c1, pol);
 }
 template <int CG>
-__device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
-  if (CG == 2) tma2_load_3d(dst, map, bar, c0, c1, c2); else tma_load_3d(dst, map, bar, c0, c1, c2);
+__device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, uint64_t pol) {
+  if (CG == 2) tma2_load_3d(dst, map, bar, c0, c1, c2, pol); else tma_load_3d(dst, map, bar, c0, c1, c2, pol);
 }
 __device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -661,6 +677,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     int stage = 0;
     uint32_t phase = 0;
     bool alive = true;
+    const uint64_t polA = operand_policy<ROLE>(0), polB = operand_policy<ROLE>(1);
     const int gw = warp == 0 ? 0 : warp - 5;           // 0 .. kGatherWarps - 1
     const int c16 = lane & 7, r_lo = lane >> 3;
     const char* const xg = reinterpret_cast<const char*>(p.gather_src);
@@ -714,18 +731,18 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               const int half = q.bn >> 1;
               const int h0 = q.n0 + pc * half;
               if (CG == 2) {
-                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i + (int)cta_rank);
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i + (int)cta_rank, polB);
               } else {
-                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i);
-                tma_3d<CG>(sB + half * 128, mB, fb, k0, h0, 2 * q.i + 1);
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i, polB);
+                tma_3d<CG>(sB + half * 128, mB, fb, k0, h0, 2 * q.i + 1, polB);
               }
             }
           } else {
             if (p.a_blk[q.g]) {
-              tma_3d<CG>(sA, mA, fb, 0, q.r0 + k0, am0 >> 6);
+              tma_3d<CG>(sA, mA, fb, 0, q.r0 + k0, am0 >> 6, polA);
             } else {
-              tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0);
-              tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0);
+              tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0, polA);
+              tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0, polA);
             }
           }
         }
@@ -771,6 +788,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
   } else if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
+      const uint64_t polA = operand_policy<ROLE>(0), polB = operand_policy<ROLE>(1);
       int stage = 0;
       uint32_t phase = 0;
       bool alive = true;
@@ -801,13 +819,13 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           const int k0 = kb * BK;
           if (RT::A_MN) {
             if (p.a_blk[q.g]) {
-              tma_3d<CG>(sA, mA, fb, 0, q.r0 + k0, am0 >> 6);
+              tma_3d<CG>(sA, mA, fb, 0, q.r0 + k0, am0 >> 6, polA);
             } else {
-              tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0);
-              tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0);
+              tma_2d<CG>(sA, mA, fb, am0, q.r0 + k0, polA);
+              tma_2d<CG>(sA + 8192, mA, fb, am0 + 64, q.r0 + k0, polA);
             }
           } else {
-            tma_2d<CG>(sA, mA, fb, (is_plain<ROLE>() ? q.r0 : 0) + k0, am0);   // r0: split-K offset
+            tma_2d<CG>(sA, mA, fb, (is_plain<ROLE>() ? q.r0 : 0) + k0, am0, polA);   // r0: split-K offset
           }
           for (int pc = 0; pc < pieces; ++pc) {
             const uint32_t sB = sA + kABytes + pc * G::kBBytes;
@@ -815,29 +833,29 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               const int half = q.bn >> 1;
               const int h0 = q.n0 + pc * half;               // first hidden column of this piece
               if (CG == 2) {          // leader stages the gate rows, its peer the up rows
-                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i + (int)cta_rank);
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i + (int)cta_rank, polB);
               } else {
-                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i);
-                tma_3d<CG>(sB + half * 128, mB, fb, k0, h0, 2 * q.i + 1);
+                tma_3d<CG>(sB, mB, fb, k0, h0, 2 * q.i, polB);
+                tma_3d<CG>(sB + half * 128, mB, fb, k0, h0, 2 * q.i + 1, polB);
               }
             } else {
               const int bn0 = q.n0 + pc * q.bn + nb * (int)cta_rank;   // this CTA's slice of the columns
               if (ROLE == ROLE_LOGITS) {
                 if (p.rf.on) {     // expert rows of the router weight first, the group rows behind them
                   const int ne = p.rf.Ng * p.rf.N;
-                  tma_2d<CG>(sB, &p.mapB[0], fb, q.r0 + k0, p.rf.Ng);
-                  tma_2d<CG>(sB + ne * 128, &p.mapB[1], fb, q.r0 + k0, 0);
+                  tma_2d<CG>(sB, &p.mapB[0], fb, q.r0 + k0, p.rf.Ng, polB);
+                  tma_2d<CG>(sB + ne * 128, &p.mapB[1], fb, q.r0 + k0, 0, polB);
                 } else {
-                  tma_2d<CG>(sB, mB, fb, q.r0 + k0, bn0);
+                  tma_2d<CG>(sB, mB, fb, q.r0 + k0, bn0, polB);
                 }
               } else if (ROLE == ROLE_FWD2) {
-                tma_3d<CG>(sB, mB, fb, k0, bn0, q.i);
+                tma_3d<CG>(sB, mB, fb, k0, bn0, q.i, polB);
               } else if (ROLE == ROLE_DGRAD_DOWN || ROLE == ROLE_DGRAD_13) {
-                if (p.b_blk[q.g]) tma_4d<CG>(sB, mB, fb, 0, k0, bn0 >> 6, q.i);
-                else for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i);
+                if (p.b_blk[q.g]) tma_4d<CG>(sB, mB, fb, 0, k0, bn0 >> 6, q.i, polB);
+                else for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i, polB);
               } else {
-                if (p.b_blk[q.g]) tma_3d<CG>(sB, mB, fb, 0, q.r0 + k0, bn0 >> 6);
-                else for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0);
+                if (p.b_blk[q.g]) tma_3d<CG>(sB, mB, fb, 0, q.r0 + k0, bn0 >> 6, polB);
+                else for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0, polB);
               }
             }
           }
