@@ -1713,10 +1713,10 @@ constexpr double kWideMinK = 3000.0;
 bool wide_tiles(const Dims& D, int role) {
   const int mask = switch_value(SW_TC_WIDE);
   if (mask >= 0) return (mask >> role) & 1;
-  // The SwiGLU backward has the longest epilogue of all roles (it also reads A and U); exposed at
-  // every entry boundary it costs more than the saved operand traffic brings (measured at the
-  // large workload: step 44.1 -> 43.8 ms with this role on single-width tiles).
-  if (role == ROLE_DGRAD_DOWN) return false;
+  // The SwiGLU backward has the longest epilogue of all roles (it also reads A and U) and is the
+  // role that gains least: before the operand loads carried L2 priorities it was faster on
+  // single-width tiles (step 44.1 -> 43.8 ms at the large workload), with them double-width entries
+  // win (45.0-46.0 -> 44.9-45.4 ms, five runs each on two GPUs), so it follows the common rule.
   double num = 0.0, den = 0.0;            // mean contraction length, weighted by the group's width
   for (int g = 0; g < D.Ng; ++g) {
     double k;
