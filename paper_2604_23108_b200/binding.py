@@ -97,11 +97,17 @@ def _ptr(t: Optional[torch.Tensor]):
     if t is None:
         return None
     assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
-    return C.c_void_p(t.data_ptr())
+    return t.data_ptr()          # an int: ctypes converts it for a c_void_p parameter
+
+
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
 
 
 def _stream():
-    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    """The caller's current stream as a raw handle (every call is enqueued on it)."""
+    if _raw_stream is not None:
+        return _raw_stream(torch.cuda.current_device())
+    return torch.cuda.current_stream().cuda_stream
 
 
 def _ptr_array(ts: Sequence[torch.Tensor]):
@@ -129,6 +135,13 @@ class Config:
     row_align: int = 128
 
     def c(self) -> mohge_config:
+        """The POD of the C ABI; rebuilt only when a field has changed since the last call."""
+        key = (self.d_model, self.n_groups, self.experts_per_group, self.k_groups, self.k_experts,
+               tuple(self.group_width), self.dtype, self.alpha_g, self.alpha_e, self.eps,
+               self.f_norm_by_T, self.fe_mode, self.row_align)
+        cached = self.__dict__.get("_c_cache")
+        if cached is not None and cached[0] == key:
+            return cached[1]
         s = mohge_config()
         s.d_model, s.n_groups, s.experts_per_group = self.d_model, self.n_groups, self.experts_per_group
         s.k_groups, s.k_experts = self.k_groups, self.k_experts
@@ -137,6 +150,7 @@ class Config:
         s.dtype = BF16 if self.dtype == "bf16" else F32
         s.alpha_g, s.alpha_e, s.eps = self.alpha_g, self.alpha_e, self.eps
         s.f_norm_by_T, s.fe_mode, s.row_align = self.f_norm_by_T, self.fe_mode, self.row_align
+        self.__dict__["_c_cache"] = (key, s)
         return s
 
     @property
