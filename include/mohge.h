@@ -144,6 +144,10 @@ void mohge_map_cache_stats(int64_t* hits, int64_t* misses);
  * "top-K" picks exactly K entries, ties go to the lowest index; slot k of group_idx /
  * expert_idx holds the k-th largest.  The selection arithmetic is a fixed float32 sequence
  * (documented in router.cu) so that indices are reproducible bit for bit from the logits.
+ * BF16 layers: one kernel computes the logits on the tensor cores and does the selection in its
+ * epilogue when N is 4, 8, 16 or 32, N_e a multiple of 8, K_e <= 8, NL <= 160 and the batch has
+ * a few thousand tokens or more; otherwise (and for given logits, and for FP32 layers) a logits
+ * kernel is followed by a selection kernel.  The results are the same bits either way.
  *   x          [T, d] dtype                 w_router  [NL, d] dtype
  *   logit_bias [NL] float32 or NULL         logits_in [T, NL] float32 or NULL
  *     (when logits_in is given, x / w_router / logit_bias are not read)
