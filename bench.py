@@ -204,7 +204,8 @@ def flops_per_step(wl: Workload, counts, shared_width: int = 0) -> float:
     return 18.0 * wl.d_model * tot
 
 
-def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=False, gather=False):
+def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=False, gather=False,
+              dy_fused=False):
     """One pass of the whole hot path through the C ABI.  Returns (step, gemm_marks): with
     mark=True a step records CUDA events around mohge_expert_fwd and mohge_expert_bwd_dgate."""
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -248,11 +249,19 @@ def make_step(B, gcfg, T, inp, buf, shared=None, shared_width=0, forward_only=Fa
         if before_bwd is not None:
             before_bwd()                    # dy is first read below (the end-to-end arm waits for its upload)
         # the gate gradient comes out of the experts' backward, so combine_bwd reads no y_perm
-        B.mohge_combine_bwd(gcfg, T, inp["dy"], None, buf.prow_of, buf.gate_w, buf.counts,
-                            buf.aligned, buf.dy_perm, None)
+        if dy_fused:    # no dy_perm: the GEMMs gather the rows of dy
+            B.mohge_row_tokens(gcfg, T, buf.counts, buf.offsets, buf.aligned, buf.src_of, buf.tok_of_prow)
+        else:
+            B.mohge_combine_bwd(gcfg, T, inp["dy"], None, buf.prow_of, buf.gate_w, buf.counts,
+                                buf.aligned, buf.dy_perm, None)
         if mark:
             e2.record()
-        if gather:
+        if dy_fused:
+            B.mohge_expert_bwd_dy(gcfg, T, inp["dy"], buf.tok_of_prow, buf.x_perm, buf.au, buf.h, buf.counts,
+                                  buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13, buf.dw2,
+                                  0, buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate, buf.hs, buf.row_gate,
+                                  buf.ws)
+        elif gather:
             B.mohge_expert_bwd_gather(gcfg, T, buf.dy_perm, inp["x"], buf.tok_of_prow, buf.au, buf.h, buf.counts,
                                       buf.aligned, inp["w13"], inp["w2"], buf.dau, buf.dx_perm, buf.dw13,
                                       buf.dw2, 0, inp["dy"], buf.y_perm, buf.prow_of, buf.gate_w, buf.dgate,
@@ -395,6 +404,10 @@ def main():
     ap.add_argument("--gather", action="store_true",
                     help="time the route that never writes x_perm (mohge_dispatch_indices, "
                          "mohge_expert_fwd_gather, mohge_expert_bwd_gather); BF16 workloads only")
+    ap.add_argument("--dy-fused", action="store_true",
+                    help="time the backward that never writes dy_perm (mohge_row_tokens, "
+                         "mohge_expert_bwd_dy instead of mohge_combine_bwd, mohge_expert_bwd_dgate); "
+                         "BF16 workloads only")
     ap.add_argument("--graph", action="store_true",
                     help="capture one step in a CUDA graph and time its replays (launch-bound small "
                          "workloads); the GEMM share for the roofline object is then taken from a "
@@ -433,8 +446,11 @@ def main():
         shared = make_shared_weights(wl, args.shared_width, device=dev, seed=replica_seed(wl, rank))
     T = wl.T
     ev = lambda: torch.cuda.Event(enable_timing=True)
+    if args.dy_fused:
+        buf.hs = torch.empty_like(buf.h)
+        buf.row_gate = torch.empty(buf.h.shape[0], dtype=torch.float32, device=buf.h.device)
     step, gemm_marks = make_step(B, gcfg, T, inp, buf, shared, args.shared_width, args.forward_only,
-                                 args.gather)
+                                 args.gather, args.dy_fused)
 
     def barrier():
         if dist is not None:
@@ -597,7 +613,8 @@ def main():
     # ---- outside the timed region: every HBM-bound entry point on its own, then short runs of the
     # other benchmark workloads (default line only) ----
     hbm_steps, others = None, None
-    if not args.no_extras and world == 1 and not args.forward_only and not args.shared_width and not args.gather:
+    if not args.no_extras and world == 1 and not args.forward_only and not args.shared_width and not args.gather \
+            and not args.dy_fused:
         hbm_steps = hbm_step_rooflines(B, gcfg, wl, inp, buf, pk["hbm"])
         if args.workload == DEFAULT_WORKLOAD:
             others = [quick_workload_line(B, n, dev, pk) for n in
@@ -643,7 +660,8 @@ def main():
                    "count_ratio": count_ratio(counts),
                    "l2": "inputs larger than L2 (no flush)", "parallelism": "replicas only",
                    "launch": "CUDA graph replay" if args.graph else "stream launches",
-                   "x_perm": "never written (rows gathered by the GEMMs)" if args.gather else "materialised"},
+                   "x_perm": "never written (rows gathered by the GEMMs)" if args.gather else "materialised",
+                   "dy_perm": "never written (rows gathered by the GEMMs)" if args.dy_fused else "materialised"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "device_status": status,
         "host_enqueue_ms_per_step": host_enqueue_ms,
         "roofline": roofline, "roofline_hbm_steps": hbm_steps, "cpu_baseline": cpu_baseline,

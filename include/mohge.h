@@ -317,6 +317,37 @@ int32_t mohge_expert_bwd_gather(const mohge_config* cfg, int64_t T, const void* 
                                 float* dgate_w, void* ws, void* stream);
 
 /*
+ * The experts' backward without dy_perm (no paper counterpart; an implementation choice like the
+ * calls above, and like them slower than the materialised copy on B200: see the note above).
+ * Replaces mohge_combine_bwd + mohge_expert_bwd_dgate after a forward pass through the listed
+ * calls.  The two GEMMs that read dy_perm (the gradient of the hidden activation, Eq. 15
+ * differentiated with respect to the down projection's input, and the down projection's weight
+ * gradient) gather the rows of dy [T, d] themselves through tok_of_prow; the gate of Eq. 6
+ * enters after the contraction: dH[r, :] = row_gate[r] * (dy[tok(r), :] . W2) in the epilogue of
+ * the first, which also writes hs = row_gate * H, and dW2 = dy[tok(.), :]^T . hs in the second.
+ * The gate gradient is formed as in mohge_expert_bwd_dgate.  Products are rounded at other
+ * places than on the route through dy_perm (gate * dy is never rounded to the layer dtype,
+ * gate * H is), so results agree with that route to the layer dtype's tolerance, not bit for bit.
+ *   mohge_row_tokens      tok_of_prow [mohge_perm_rows + 128] from the outputs of mohge_dispatch
+ *                         (the same array mohge_dispatch_indices writes)
+ *   mohge_expert_bwd_dy   dy [T, d] dtype; hs: scratch with the layout of h_saved, written;
+ *                         row_gate [mohge_perm_rows] float32 scratch, written; y_perm, prow_of,
+ *                         gate_w, dgate_w as in mohge_expert_bwd_dgate; the rest as in
+ *                         mohge_expert_bwd.  BF16 tensor-core path only; T > 0.
+ */
+int32_t mohge_row_tokens(const mohge_config* cfg, int64_t T, const int32_t* counts,
+                         const int32_t* offsets, const int32_t* aligned_offsets,
+                         const int32_t* src_of, int32_t* tok_of_prow, void* stream);
+int32_t mohge_expert_bwd_dy(const mohge_config* cfg, int64_t T, const void* dy,
+                            const int32_t* tok_of_prow, const void* x_perm, const void* au_saved,
+                            const void* h_saved, const int32_t* counts,
+                            const int32_t* aligned_offsets, const void* const* w13,
+                            const void* const* w2, void* dau, void* dx_perm, float* const* dw13,
+                            float* const* dw2, int32_t accumulate, const void* y_perm,
+                            const int32_t* prow_of, const float* gate_w, float* dgate_w, void* hs,
+                            float* row_gate, void* ws, void* stream);
+
+/*
  * Backward of the permutation: dx[t, :] = sum_k dx_perm[prow_of[t,k], :] (+ dx_add[t, :]).
  *   dx [T, d] dtype;  dx_add [T, d] dtype, nullable (the shared experts' input gradient).
  */

@@ -60,6 +60,9 @@ _SIGS = {
     "mohge_expert_fwd_gather": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 11),
     "mohge_expert_bwd_gather": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 13
                                 + [C.c_int32] + [_P] * 7),
+    "mohge_row_tokens": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 6),
+    "mohge_expert_bwd_dy": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 13
+                            + [C.c_int32] + [_P] * 8),
     "mohge_dispatch_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64] + [_P] * 5),
     "mohge_shared_fwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 8),
     "mohge_shared_bwd": (C.c_int32, [C.POINTER(mohge_config), C.c_int64, C.c_int32] + [_P] * 10
@@ -325,6 +328,23 @@ def mohge_expert_bwd_gather(cfg, T, dy_perm, x, tok_of_prow, au_saved, h_saved, 
            "mohge_expert_bwd_gather")
 
 
+def mohge_row_tokens(cfg, T, counts, offsets, aligned_offsets, src_of, tok_of_prow):
+    _check(lib().mohge_row_tokens(C.byref(cfg.c()), T, _ptr(counts), _ptr(offsets), _ptr(aligned_offsets),
+                                  _ptr(src_of), _ptr(tok_of_prow), _stream()), "mohge_row_tokens")
+
+
+def mohge_expert_bwd_dy(cfg, T, dy, tok_of_prow, x_perm, au_saved, h_saved, counts, aligned_offsets, w13, w2,
+                        dau, dx_perm, dw13, dw2, accumulate, y_perm, prow_of, gate_w, dgate_w, hs, row_gate,
+                        ws):
+    a13, a2, d13, d2 = _ptr_array(w13), _ptr_array(w2), _ptr_array(dw13), _ptr_array(dw2)
+    _check(lib().mohge_expert_bwd_dy(C.byref(cfg.c()), T, _ptr(dy), _ptr(tok_of_prow), _ptr(x_perm),
+                                     _ptr(au_saved), _ptr(h_saved), _ptr(counts), _ptr(aligned_offsets),
+                                     C.cast(a13, _P), C.cast(a2, _P), _ptr(dau), _ptr(dx_perm),
+                                     C.cast(d13, _P), C.cast(d2, _P), int(accumulate), _ptr(y_perm),
+                                     _ptr(prow_of), _ptr(gate_w), _ptr(dgate_w), _ptr(hs), _ptr(row_gate),
+                                     _ptr(ws), _stream()), "mohge_expert_bwd_dy")
+
+
 def mohge_dispatch_bwd(cfg, T, dx_perm, prow_of, dx, dx_add=None):
     _check(lib().mohge_dispatch_bwd(C.byref(cfg.c()), T, _ptr(dx_perm), _ptr(prow_of),
                                     _ptr(dx_add), _ptr(dx), _stream()), "mohge_dispatch_bwd")
@@ -423,12 +443,21 @@ def layer_forward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, logit_bias
 
 
 def layer_backward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, dy, aux=True, accumulate=False,
-                   shared=None, fused_dgate=True, gather=False):
+                   shared=None, fused_dgate=True, gather=False, dy_fused=False):
     """combine_bwd -> expert_bwd (-> shared_bwd) -> dispatch_bwd -> route_bwd; results stay in `b`.
     fused_dgate: the gate gradient comes out of the experts' backward (mohge_expert_bwd_dgate) and
-    combine_bwd does not read y_perm; otherwise combine_bwd computes it from y_perm."""
+    combine_bwd does not read y_perm; otherwise combine_bwd computes it from y_perm.
+    dy_fused: no combine_bwd and no dy_perm at all (mohge_expert_bwd_dy gathers the rows of dy)."""
     T = b.T
-    if gather:      # after a forward with gather=True: x_perm was never written
+    if dy_fused:    # after a forward through x_perm
+        if getattr(b, "hs", None) is None:
+            b.hs = torch.empty_like(b.h)
+            b.row_gate = torch.empty(b.h.shape[0], dtype=torch.float32, device=b.h.device)
+        mohge_row_tokens(cfg, T, b.counts, b.offsets, b.aligned, b.src_of, b.tok_of_prow)
+        mohge_expert_bwd_dy(cfg, T, dy, b.tok_of_prow, b.x_perm, b.au, b.h, b.counts, b.aligned, w13, w2,
+                            b.dau, b.dx_perm, b.dw13, b.dw2, accumulate, b.y_perm, b.prow_of, b.gate_w,
+                            b.dgate, b.hs, b.row_gate, b.ws)
+    elif gather:    # after a forward with gather=True: x_perm was never written
         mohge_combine_bwd(cfg, T, dy, None, b.prow_of, b.gate_w, b.counts, b.aligned, b.dy_perm, None)
         mohge_expert_bwd_gather(cfg, T, b.dy_perm, x, b.tok_of_prow, b.au, b.h, b.counts, b.aligned, w13,
                                 w2, b.dau, b.dx_perm, b.dw13, b.dw2, accumulate, dy, b.y_perm, b.prow_of,

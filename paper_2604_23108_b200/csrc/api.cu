@@ -480,9 +480,10 @@ static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy
                                const void* x_perm, const void* au_saved, const void* h_saved,
                                const int32_t* counts, const int32_t* aligned_offsets, void* dau,
                                void* dx_perm, int32_t accumulate, const Ws& w, cudaStream_t st,
-                               const DgateArgs* dg = nullptr, const int32_t* gather = nullptr) {
+                               const DgateArgs* dg = nullptr, const int32_t* gather = nullptr,
+                               const DyFuse* dyf = nullptr) {
   int32_t rc;
-  if (gather && !(D.bf16 && !force_simt())) {
+  if ((gather || dyf) && !(D.bf16 && !force_simt())) {
     set_error("the row-gathering entry points need the BF16 tensor-core path");
     return MOHGE_ERR_UNSUPPORTED;
   }
@@ -501,14 +502,16 @@ static int32_t expert_bwd_impl(const Dims& D, const GroupPtrs& P, const void* dy
     for (int r = 0; r < 4; ++r) {
       const void* A = nullptr; const void* B = nullptr; void* C = nullptr; void* C2 = nullptr;
       switch (roles[r]) {
+        // dyf: dy_perm is dy [T, d] itself (rows gathered by the kernels), and WGRAD_DOWN reads
+        // the gate * H that DGRAD_DOWN has just written instead of H
         case ROLE_DGRAD_DOWN: A = dy_perm; B = au_saved; C = dau; break;
-        case ROLE_WGRAD_DOWN: A = dy_perm; B = h_saved; break;
+        case ROLE_WGRAD_DOWN: A = dy_perm; B = dyf ? dyf->hs : h_saved; break;
         case ROLE_DGRAD_13: A = dau; C = dx_perm; break;
         default: A = dau; B = x_perm; break;
       }
       rc = launch_tc_grouped(D, roles[r], P, A, B, C, C2, counts, aligned_offsets, accumulate,
                              w.tile_count + 64 * r, w.tiles + w.tiles_cap * r, w.tiles_cap, w.status,
-                             st, true, dg ? w.dgp : nullptr, w.dgate_slots, gather);
+                             st, true, dg ? w.dgp : nullptr, w.dgate_slots, gather, dyf);
       if (rc) return rc;
       if (dg && roles[r] == ROLE_DGRAD_DOWN) {
         int bn[MOHGE_MAX_GROUPS];
@@ -611,6 +614,44 @@ int32_t mohge_expert_bwd_gather(const mohge_config* cfg, int64_t T, const void* 
   const DgateArgs dg = {dy, y_perm, prow_of, gate_w, dgate_w};
   return expert_bwd_impl(D, P, dy_perm, x, au_saved, h_saved, counts, aligned_offsets, dau, dx_perm,
                          accumulate, carve(D, ws), (cudaStream_t)stream, &dg, tok_of_prow);
+}
+
+int32_t mohge_row_tokens(const mohge_config* cfg, int64_t T, const int32_t* counts,
+                         const int32_t* offsets, const int32_t* aligned_offsets,
+                         const int32_t* src_of, int32_t* tok_of_prow, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(counts); REQ_PTR(offsets); REQ_PTR(aligned_offsets); REQ_PTR(src_of); REQ_PTR(tok_of_prow);
+  return launch_token_of_row(D, counts, offsets, aligned_offsets, src_of, tok_of_prow, (cudaStream_t)stream);
+}
+
+int32_t mohge_expert_bwd_dy(const mohge_config* cfg, int64_t T, const void* dy,
+                            const int32_t* tok_of_prow, const void* x_perm, const void* au_saved,
+                            const void* h_saved, const int32_t* counts,
+                            const int32_t* aligned_offsets, const void* const* w13,
+                            const void* const* w2, void* dau, void* dx_perm, float* const* dw13,
+                            float* const* dw2, int32_t accumulate, const void* y_perm,
+                            const int32_t* prow_of, const float* gate_w, float* dgate_w, void* hs,
+                            float* row_gate, void* ws, void* stream) {
+  Dims D;
+  int32_t rc = make_dims(cfg, T, &D);
+  if (rc) return rc;
+  REQ_PTR(dy); REQ_PTR(tok_of_prow); REQ_PTR(x_perm); REQ_PTR(au_saved); REQ_PTR(h_saved); REQ_PTR(counts);
+  REQ_PTR(aligned_offsets); REQ_PTR(dau); REQ_PTR(dx_perm); REQ_PTR(ws);
+  REQ_PTR(y_perm); REQ_PTR(prow_of); REQ_PTR(gate_w); REQ_PTR(dgate_w); REQ_PTR(hs); REQ_PTR(row_gate);
+  MOHGE_CHECK_ARG(w13 && w2 && dw13 && dw2, "w13, w2, dw13, dw2 must be host arrays of n_groups device pointers");
+  MOHGE_CHECK_ARG(T > 0, "the row-gathering entry points need T > 0");
+  GroupPtrs P;
+  rc = group_ptrs(D, w13, w2, dw13, dw2, &P);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  rc = launch_row_gate(D, prow_of, gate_w, row_gate, st);
+  if (rc) return rc;
+  const DgateArgs dg = {dy, y_perm, prow_of, gate_w, dgate_w};
+  const DyFuse dyf = {tok_of_prow, row_gate, hs};
+  return expert_bwd_impl(D, P, dy, x_perm, au_saved, h_saved, counts, aligned_offsets, dau, dx_perm,
+                         accumulate, carve(D, ws), st, &dg, nullptr, &dyf);
 }
 
 int32_t mohge_dispatch_bwd(const mohge_config* cfg, int64_t T, const void* dx_perm,

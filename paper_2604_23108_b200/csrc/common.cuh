@@ -188,6 +188,14 @@ int32_t launch_combine(const Dims& D, const void* y_perm, const int32_t* prow_of
 int32_t launch_combine_bwd(const Dims& D, int mode, const void* dy, const void* y_perm,
                            const int32_t* prow_of, const float* gate_w, const int32_t* counts,
                            const int32_t* aligned, void* dy_perm, float* dgate_w, cudaStream_t st);
+// tok_of_prow[r] = token whose row sits at physical row r, T for padding rows and the 128 rows
+// past the last segment
+int32_t launch_token_of_row(const Dims& D, const int32_t* counts, const int32_t* offsets,
+                            const int32_t* aligned, const int32_t* src_of, int32_t* tok_of_prow,
+                            cudaStream_t st);
+// row_gate[prow_of[t, k]] = gate_w[t, k], 0 at every other physical row (padding)
+int32_t launch_row_gate(const Dims& D, const int32_t* prow_of, const float* gate_w, float* row_gate,
+                        cudaStream_t st);
 int32_t launch_dgate_reduce(const Dims& D, const int* bn, const float* part, int slots,
                             const int32_t* prow_of, const float* gate_w, const int32_t* aligned,
                             const void* dy, const void* y_perm, float* dgate_w, cudaStream_t st);
@@ -215,12 +223,19 @@ int32_t launch_simt_plain(int M, int N, int K, const void* A, int a_f32, int64_t
 // gemm_tc.cu (tcgen05 path, BF16)
 // gather != nullptr (FWD1, WGRAD_13 only): the x_perm operand (A of FWD1, B of WGRAD_13) is x
 // itself, [T, d], and row r of the permuted numbering is row gather[r] of it (>= T: zeros)
+// The experts' backward without dy_perm: DGRAD_DOWN and WGRAD_DOWN gather the rows of dy [T, d]
+// (A operand) through tok_of_prow; DGRAD_DOWN scales by row_gate and writes hs = gate * H.
+struct DyFuse {
+  const int32_t* tok_of_prow;    // [mohge_perm_rows + 128]
+  const float* row_gate;         // [mohge_perm_rows]: gate of the pair at a physical row, 0 for padding
+  void* hs;                      // layout of h_saved
+};
 int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const void* A,
                           const void* B, void* C, void* C2, const int32_t* counts,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
                           int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt = false,
                           float* dgate_part = nullptr, int dgate_slots = 0,
-                          const int32_t* gather = nullptr);
+                          const int32_t* gather = nullptr, const struct DyFuse* dyf = nullptr);
 // UMMA N of a group in ROLE_DGRAD_DOWN (128 or 256): which 128-column slots of dgate_part are written
 int tc_dgrad_down_bn(const Dims& D, int g);
 TilePlan tc_tile_plan(const Dims& D, int role);

@@ -447,6 +447,16 @@ int block_for(int row_vecs) {
 
 }  // namespace
 
+int32_t launch_token_of_row(const Dims& D, const int32_t* counts, const int32_t* offsets,
+                            const int32_t* aligned, const int32_t* src_of, int32_t* tok_of_prow,
+                            cudaStream_t st) {
+  const int n_rows = (int)D.Rcap + kGatherSlack;
+  launch_dep(token_of_row_kernel, dim3((n_rows + 255) / 256 < 1184 ? (n_rows + 255) / 256 : 1184), dim3(256), st,
+             n_rows, (int)D.T, D.Ke, D.Ne, counts, offsets, aligned, src_of, tok_of_prow);
+  MOHGE_LAUNCH_CHECK("token_of_row_kernel");
+  return MOHGE_OK;
+}
+
 // x != nullptr: rows of x are copied into x_perm; tok_of_prow != nullptr: the row map for the
 // gathering GEMMs is written instead (kGatherSlack rows past mohge_perm_rows included).
 int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx, int32_t* counts,
@@ -467,11 +477,8 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
     MOHGE_LAUNCH_CHECK("dispatch_scatter_kernel");
   }
   if (tok_of_prow != nullptr) {
-    const int n_rows = (int)D.Rcap + kGatherSlack;
-    launch_dep(token_of_row_kernel, dim3((n_rows + 255) / 256 < 1184 ? (n_rows + 255) / 256 : 1184), dim3(256), st,
-               n_rows, T, D.Ke, D.Ne, (const int32_t*)counts, (const int32_t*)offsets, (const int32_t*)aligned,
-               (const int32_t*)src_of, tok_of_prow);
-    MOHGE_LAUNCH_CHECK("token_of_row_kernel");
+    const int32_t rc = launch_token_of_row(D, counts, offsets, aligned, src_of, tok_of_prow, st);
+    if (rc) return rc;
   }
   if (chunks == 0 || x == nullptr) return MOHGE_OK;
   const int row_vecs = D.d * (D.bf16 ? 2 : 4) / 16;
@@ -480,6 +487,34 @@ int32_t launch_dispatch(const Dims& D, const void* x, const int32_t* expert_idx,
   launch_dep(permute_rows_kernel, dim3(blocks + pad_blocks), dim3(block_for(row_vecs)), st,
       (const Vec16*)x, prow_of, T, D.Ke, row_vecs, (int)D.Rcap, (Vec16*)x_perm, blocks, counts, aligned);
   MOHGE_LAUNCH_CHECK("permute_rows_kernel");
+  return MOHGE_OK;
+}
+
+namespace {
+__global__ void __launch_bounds__(256)
+row_gate_kernel(int n_rows, int n_slots, const int32_t* __restrict__ prow_of,
+                const float* __restrict__ gate_w, float* __restrict__ row_gate, int phase) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (phase == 0) {
+    if (i < n_rows) row_gate[i] = 0.0f;
+  } else if (i < n_slots) {
+    const int r = prow_of[i];
+    if ((unsigned)r < (unsigned)n_rows) row_gate[r] = gate_w[i];
+  }
+}
+}  // namespace
+
+int32_t launch_row_gate(const Dims& D, const int32_t* prow_of, const float* gate_w, float* row_gate,
+                        cudaStream_t st) {
+  const int n_rows = (int)D.Rcap, n_slots = (int)(D.T * D.Ke);
+  if (n_rows > 0) {
+    row_gate_kernel<<<(n_rows + 255) / 256, 256, 0, st>>>(n_rows, n_slots, prow_of, gate_w, row_gate, 0);
+    MOHGE_LAUNCH_CHECK("row_gate_kernel");
+  }
+  if (n_slots > 0) {
+    row_gate_kernel<<<(n_slots + 255) / 256, 256, 0, st>>>(n_rows, n_slots, prow_of, gate_w, row_gate, 1);
+    MOHGE_LAUNCH_CHECK("row_gate_kernel");
+  }
   return MOHGE_OK;
 }
 

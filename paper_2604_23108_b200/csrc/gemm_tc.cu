@@ -138,6 +138,13 @@ struct TcParams {
   const int32_t* gather;
   const void* gather_src;
   int gather_rows;
+  // Gathering form of the two roles that read dy_perm (DGRAD_DOWN and WGRAD_DOWN: A operand):
+  // gather_src = dy [T, d] itself, unscaled.  DGRAD_DOWN then multiplies the accumulator row r by
+  // row_gate[r] (the gate of the routed pair at physical row r, 0 for padding rows) and also
+  // writes hs = row_gate * H (the layout of h_saved), the B operand WGRAD_DOWN needs instead of H.
+  const float* row_gate;
+  __nv_bfloat16* hs;
+  int hs_pitch;                  // elements per row of hs
   GroupShape gs;
   GroupPtrs gp;
   int BN[MOHGE_MAX_GROUPS];      // UMMA N per group (FWD1: gate half + up half)
@@ -670,6 +677,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
     //             for a tile and live in registers
     //   WGRAD_13  B tile = blocks of 64 k-rows x 128 B; the rows are the contraction index, so a
     //             lane's 16 row indices change with every k-block and are fetched one ahead
+    //   DGRAD_DOWN, WGRAD_DOWN (the backward without dy_perm): the rows of dy through the same
+    //             map, as FWD1 does for its A tile and as WGRAD_13 does for its B tile, here for
+    //             the A tile (two 64-column blocks per CTA) with B brought by TMA
     // Each lane's copies of a stage end in cp.async.mbarrier.arrive on the stage's gather
     // barrier; the relay warp waits for that barrier, makes the rows visible to the async proxy
     // and arrives on the pair leader's full barrier.  Row indices >= T (padding rows) and columns
@@ -695,15 +705,20 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
       const int nb = q.bn / CG;
       const int pieces = (WIDE && q.wide) ? 2 : 1;
       const int am0 = q.m0 + BM * (int)cta_rank;
+      // which operand is gathered: A with rows = tile rows (K-major: FWD1 gathers x, DGRAD_DOWN dy),
+      // B with rows = contraction index (WGRAD_13 gathers x), A with rows = contraction index
+      // (WGRAD_DOWN gathers dy)
+      constexpr bool kGatherAK = ROLE == ROLE_FWD1 || ROLE == ROLE_DGRAD_DOWN;
+      constexpr bool kGatherAMN = ROLE == ROLE_WGRAD_DOWN;
       // bytes TMA brings per stage: the operand that is not gathered
-      const uint32_t tx = ROLE == ROLE_FWD1 ? (uint32_t)pieces * nb * BK * 2 : (uint32_t)kABytes;
-      constexpr int kRowsF = 32 / kGatherWarps;         // FWD1: row slots of this warp's lanes
-      // WGRAD_13: a stage has nblk 64-column blocks of 16 row slots (j) each; the warps share the
-      // blocks (or, with fewer blocks than warps, the slots of a block)
-      const int nblk = pieces * (nb / 64);
-      int rows[kRowsF > 16 ? kRowsF : 16];             // FWD1: row of slot j of this warp; WGRAD_13: row of slot j
+      const uint32_t tx = (kGatherAK || kGatherAMN) ? (uint32_t)pieces * nb * BK * 2 : (uint32_t)kABytes;
+      constexpr int kRowsF = 32 / kGatherWarps;         // A, K-major: row slots of this warp's lanes
+      // contraction-index gathers: a stage has nblk 64-column blocks of 16 row slots (j) each; the
+      // warps share the blocks (or, with fewer blocks than warps, the slots of a block)
+      const int nblk = kGatherAMN ? 2 : pieces * (nb / 64);
+      int rows[kRowsF > 16 ? kRowsF : 16];             // row of slot j (of this warp, K-major A)
       int rows_next[16];
-      if (ROLE == ROLE_FWD1) {
+      if (kGatherAK) {
 #pragma unroll
         for (int j = 0; j < kRowsF; ++j) rows[j] = p.gather[am0 + r_lo + 4 * (gw * kRowsF + j)];
       } else {
@@ -711,7 +726,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         for (int j = 0; j < 16; ++j) rows[j] = p.gather[q.r0 + r_lo + 4 * j];
       }
       for (int kb = 0; kb < q.num_kb; ++kb) {
-        if (ROLE == ROLE_WGRAD_13) {
+        if (!kGatherAK) {
 #pragma unroll
           for (int j = 0; j < 16; ++j)
             rows_next[j] = kb + 1 < q.num_kb ? p.gather[q.r0 + (kb + 1) * BK + r_lo + 4 * j] : 0;
@@ -737,6 +752,20 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
                 tma_3d<CG>(sB + half * 128, mB, fb, k0, h0, 2 * q.i + 1, polB);
               }
             }
+          } else if (ROLE == ROLE_DGRAD_DOWN) {
+            for (int pc = 0; pc < pieces; ++pc) {
+              const uint32_t sB = sA + kABytes + pc * G::kBBytes;
+              const int bn0 = q.n0 + pc * q.bn + nb * (int)cta_rank;
+              if (p.b_blk[q.g]) tma_4d<CG>(sB, mB, fb, 0, k0, bn0 >> 6, q.i, polB);
+              else for (int j = 0; j < nb / 64; ++j) tma_3d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, k0, q.i, polB);
+            }
+          } else if (ROLE == ROLE_WGRAD_DOWN) {
+            for (int pc = 0; pc < pieces; ++pc) {
+              const uint32_t sB = sA + kABytes + pc * G::kBBytes;
+              const int bn0 = q.n0 + pc * q.bn + nb * (int)cta_rank;
+              if (p.b_blk[q.g]) tma_3d<CG>(sB, mB, fb, 0, q.r0 + k0, bn0 >> 6, polB);
+              else for (int j = 0; j < nb / 64; ++j) tma_2d<CG>(sB + j * 8192, mB, fb, bn0 + 64 * j, q.r0 + k0, polB);
+            }
           } else {
             if (p.a_blk[q.g]) {
               tma_3d<CG>(sA, mA, fb, 0, q.r0 + k0, am0 >> 6, polA);
@@ -746,7 +775,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
             }
           }
         }
-        if (ROLE == ROLE_FWD1) {
+        if (kGatherAK) {
           const int col = k0 + 8 * c16;                  // first of this lane's 8 columns
           const uint32_t col_ok = col < p.gs.d ? 16u : 0u;
           const size_t col_off = col < p.gs.d ? 2 * (size_t)col : 0;
@@ -763,9 +792,12 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
           const int share = nblk >= kGatherWarps ? 1 : kGatherWarps / nblk;     // warps per block
           const int j_lo = (gw / nblk) * (16 / share) * (share > 1 ? 1 : 0), j_n = 16 / share;
           for (int blk = share > 1 ? gw % nblk : gw; blk < nblk; blk += share > 1 ? nblk : kGatherWarps) {
-            const int pc = blk / (nb / 64), jb = blk % (nb / 64);
-            const uint32_t sB = sA + kABytes + pc * G::kBBytes;
-            const int col = q.n0 + pc * q.bn + nb * (int)cta_rank + 64 * jb + 8 * c16;
+            // B blocks of the piece's column slice, or (A gathered) the two 64-column blocks of
+            // this CTA's 128 tile rows
+            const int pc = kGatherAMN ? 0 : blk / (nb / 64), jb = kGatherAMN ? blk : blk % (nb / 64);
+            const uint32_t sB = kGatherAMN ? sA : sA + kABytes + pc * G::kBBytes;
+            const int col = kGatherAMN ? am0 + 64 * jb + 8 * c16
+                                       : q.n0 + pc * q.bn + nb * (int)cta_rank + 64 * jb + 8 * c16;
             const uint32_t col_ok = col < p.gs.d ? 16u : 0u;
             const size_t col_off = col < p.gs.d ? 2 * (size_t)col : 0;
 #pragma unroll
@@ -1210,6 +1242,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
         // per 64-column chunk: A and U arrive by TMA in one of two buffer pairs, dA and dU are
         // written over them in place and leave by TMA; the next chunk's loads fly meanwhile
         float2 dg2 = make_float2(0.0f, 0.0f);          // sum over this tile's columns of dH * h
+        // gathering form: the accumulator is dy W2 without the gate; the gate of the row comes in here
+        float2 gate2 = make_float2(1.0f, 1.0f);
+        if (GATHER && nch_in > 0) { const float gr = p.row_gate[row0 + lane]; gate2 = make_float2(gr, gr); }
         for (int ci = 0; ci < nch_in; ++ci, ++n_chunk) {
           const int c = ci * 64;
           const uint32_t set = n_chunk & 1u;
@@ -1241,6 +1276,7 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               if (ci + 1 == nch_in) release_acc();
             }
             uint32_t oa[4][4], ou[4][4];
+            uint32_t oh[GATHER ? 4 : 1][4];           // gathering form: gate * H
 #pragma unroll
             for (int j4 = 0; j4 < 4; ++j4) {
               const uint32_t wa[4] = {va[j4].x, va[j4].y, va[j4].z, va[j4].w};
@@ -1249,8 +1285,9 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
               for (int e2 = 0; e2 < 4; ++e2) {
                 const float2 a2 = make_float2(bf_lo(wa[e2]), bf_hi(wa[e2]));
                 const float2 u2 = make_float2(bf_lo(wu[e2]), bf_hi(wu[e2]));
-                const float2 dh2 = make_float2(__uint_as_float(r[hh][j4 * 8 + 2 * e2]),
-                                               __uint_as_float(r[hh][j4 * 8 + 2 * e2 + 1]));
+                float2 dh2 = make_float2(__uint_as_float(r[hh][j4 * 8 + 2 * e2]),
+                                         __uint_as_float(r[hh][j4 * 8 + 2 * e2 + 1]));
+                if (GATHER) dh2 = __fmul2_rn(dh2, gate2);
                 const float2 one = make_float2(1.0f, 1.0f);
                 const float2 s2 = sigmoid2_fast(a2);
                 const float2 oms = __ffma2_rn(s2, make_float2(-1.0f, -1.0f), one);      // 1 - s
@@ -1261,12 +1298,25 @@ tc_grouped_kernel(const __grid_constant__ TcParams p) {
                 dg2 = __ffma2_rn(du2, u2, dg2);                                         // dh * h
                 oa[j4][e2] = pack2(da2.x, da2.y);
                 ou[j4][e2] = pack2(du2.x, du2.y);
+                if (GATHER) {
+                  const float2 hg2 = __fmul2_rn(__fmul2_rn(__fmul2_rn(a2, s2), u2), gate2);   // gate * silu(a) * u
+                  oh[j4][e2] = pack2(hg2.x, hg2.y);
+                }
               }
             }
 #pragma unroll
             for (int j4 = 0; j4 < 4; ++j4) {
               st_shared_v4(stg_addr(bA, lane, hh * 4 + j4), oa[j4][0], oa[j4][1], oa[j4][2], oa[j4][3]);
               st_shared_v4(stg_addr(bU, lane, hh * 4 + j4), ou[j4][0], ou[j4][1], ou[j4][2], ou[j4][3]);
+            }
+            if (GATHER) {
+              // gate * H of this thread's row, straight from registers (eight columns per store)
+              __nv_bfloat16* ph = p.hs + (size_t)(row0 + lane) * p.hs_pitch;
+#pragma unroll
+              for (int j4 = 0; j4 < 4; ++j4) {
+                const int col = q.n0 + c + hh * 32 + j4 * 8;
+                if (col < q.W) *reinterpret_cast<uint4*>(ph + col) = make_uint4(oh[j4][0], oh[j4][1], oh[j4][2], oh[j4][3]);
+              }
             }
           }
           fence_async_smem();
@@ -1953,7 +2003,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
                           const void* B, void* C, void* C2, const int32_t* /*counts*/,
                           const int32_t* aligned, int accumulate, int32_t* tile_count, Tile* tiles,
                           int64_t tiles_cap, int32_t* status, cudaStream_t st, bool list_prebuilt,
-                          float* dgate_part, int dgate_slots, const int32_t* gather) {
+                          float* dgate_part, int dgate_slots, const int32_t* gather, const DyFuse* dyf) {
   DeviceInfo di;
   int32_t rcd = current_device(&di);
   if (rcd) return rcd;
@@ -1971,8 +2021,15 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   p.dgate_part = role == ROLE_DGRAD_DOWN ? dgate_part : nullptr;
   p.dgate_slots = dgate_slots;
   p.gather = (role == ROLE_FWD1 || role == ROLE_WGRAD_13) ? gather : nullptr;
+  const bool dy_gather = dyf != nullptr && (role == ROLE_DGRAD_DOWN || role == ROLE_WGRAD_DOWN);
+  if (dy_gather) p.gather = dyf->tok_of_prow;
   p.gather_src = nullptr;
   p.gather_rows = (int)D.T;
+  if (dy_gather && role == ROLE_DGRAD_DOWN) {
+    p.row_gate = dyf->row_gate;
+    p.hs = (__nv_bfloat16*)dyf->hs;
+    p.hs_pitch = D.Wmax;
+  }
 
   const uint64_t d = D.d, rows = D.Rcap, pitchAU = 2ull * D.Wmax * 2, pitchH = (uint64_t)D.Wmax * 2;
   const int CG = cta_group_size(D);
@@ -1995,7 +2052,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
     key.w[0][g] = P.w13[g]; key.w[1][g] = P.w2[g]; key.w[2][g] = P.dw13[g]; key.w[3][g] = P.dw2[g];
   }
   const bool cached = map_cache_find(key, &p);
-  if (p.gather) p.gather_src = role == ROLE_FWD1 ? A : B;
+  if (p.gather) p.gather_src = (role == ROLE_FWD1 || dy_gather) ? A : B;
   for (int g = 0; g < D.Ng && rc == MOHGE_OK && !cached; ++g) {
     const uint64_t W = D.W[g], N = D.N;
     uint64_t dims[3], str[2];
@@ -2034,8 +2091,10 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
       } break;
       case ROLE_DGRAD_DOWN: {
         p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
-        dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
-        rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        if (!dy_gather) {    // else A = dy [T, d], gathered row by row by the producer warp
+          dims[0] = d; dims[1] = rows; str[0] = d * 2; box[0] = BK; box[1] = BM;
+          rc = encode_map(&p.mapA[g], A, 2, dims, str, box);
+        }
         if (rc) break;
         rc = encode_mn_map(&p.mapB[g], P.w2[g], W, d, W * 2, N, d * W * 2, p.BN[g] / CG / 64, &p.b_blk[g]);
         if (rc) break;
@@ -2058,7 +2117,7 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
       } break;
       case ROLE_WGRAD_DOWN: {
         p.BN[g] = bn_plan[g] = pick_bn(D.W[g], cand_n, ncand);
-        rc = encode_mn_map(&p.mapA[g], A, d, rows, d * 2, 0, 0, 2, &p.a_blk[g]);
+        if (!dy_gather) rc = encode_mn_map(&p.mapA[g], A, d, rows, d * 2, 0, 0, 2, &p.a_blk[g]);
         if (rc) break;
         rc = encode_mn_map(&p.mapB[g], B, W, rows, pitchH, 0, 0, p.BN[g] / CG / 64, &p.b_blk[g]);
         if (rc) break;
@@ -2085,6 +2144,16 @@ int32_t launch_tc_grouped(const Dims& D, int role, const GroupPtrs& P, const voi
   if (!list_prebuilt) {
     rc = launch_build_tiles_plan(plan, aligned, tile_count, tiles, tiles_cap, status, st);
     if (rc) return rc;
+  }
+  if (p.gather && role == ROLE_DGRAD_DOWN) {     // row-gathering forms of the roles that read dy_perm
+    if (CG == 2 && wide) return launch_role<ROLE_DGRAD_DOWN, 2, 1, 1>(p, di, st);
+    if (CG == 2) return launch_role<ROLE_DGRAD_DOWN, 2, 0, 1>(p, di, st);
+    return launch_role<ROLE_DGRAD_DOWN, 1, 0, 1>(p, di, st);
+  }
+  if (p.gather && role == ROLE_WGRAD_DOWN) {
+    if (CG == 2 && wide) return launch_role<ROLE_WGRAD_DOWN, 2, 1, 1>(p, di, st);
+    if (CG == 2) return launch_role<ROLE_WGRAD_DOWN, 2, 0, 1>(p, di, st);
+    return launch_role<ROLE_WGRAD_DOWN, 1, 0, 1>(p, di, st);
   }
   if (p.gather) {          // row-gathering form of the two roles that read x_perm
     if (role == ROLE_FWD1) {
