@@ -9,6 +9,8 @@
 //               a full 128-byte row piece; the SwiGLU backward also reads A and U through TMA)
 //   warp 6      only in the row-gathering form (GATHER = 1, see "gathering form" below): forwards
 //               the completion of the producer warp's asynchronous row copies to the MMA issuer
+//   warps 6..9  only in the router-logits GEMM whose epilogue also selects (Eq. 2-6): a second
+//               epilogue warp for every quarter of the accumulator rows (route_epilogue.cuh)
 // One persistent CTA per SM (a CTA pair per two SMs for the expert roles; single CTAs when the
 // batch brings 128 rows per expert or fewer) walks the device-built, cost-sorted tile list with a
 // fixed stride, in alternating directions when tile costs differ.  The kernel is launched as a
@@ -25,6 +27,10 @@
 //   DGRAD_13    dXp = [dA | dU] . W13 (B read MN-major)
 //   WGRAD_DOWN  dW2  = dYp^T . H      (A and B read MN-major, contraction over the expert's rows)
 //   WGRAD_13    dW13 = [dA | dU]^T . Xp
+// plus three single-problem GEMMs of the router (logits, with the two-level selection in the
+// epilogue; router weight gradient; router part of dx).  In the gathering form the rows of an
+// operand that the default route reads from a permuted copy (Xp of FWD1 and WGRAD_13, dYp of
+// DGRAD_DOWN and WGRAD_DOWN) are fetched from the unpermuted tensor through a row map.
 // Expert segments start at multiples of 128 physical rows with zero padding rows, so a 128-row
 // tile never straddles two experts and padding contributes exact zeros to the weight gradients.
 // Hidden widths that are not multiples of the tile are handled by TMA's out-of-bounds zero fill
