@@ -498,7 +498,10 @@ __device__ __forceinline__ void load_row32(const __nv_bfloat16* p, float (&v)[32
 // one burst it delays that tile's operand loads (both share the SM's path to L2) by about as
 // long as the burst lasts.  The store-heavy roles therefore spread their chunks over
 // kPacePct % of the next tile's MMA time (512 clocks per 64-deep k-block at full rate).
-constexpr int kPacePct = 75;
+#ifndef MOHGE_PACE_PCT
+#define MOHGE_PACE_PCT 75
+#endif
+constexpr int kPacePct = MOHGE_PACE_PCT;      // 0 = no pacing (for measurements)
 __device__ __forceinline__ void pace(long long t0, int i, int n, int next_num_kb) {
   const long long target = t0 + (long long)next_num_kb * (512 * kPacePct / 100) * i / n;
   while (clock64() < target) __nanosleep(64);
