@@ -35,7 +35,7 @@ from paper_2604_23108_b200.inputs import WORKLOADS, Workload, make_device_inputs
 # figure is the capture of "cfg5_slice" (one eighth of the experts, the same tokens per expert,
 # widths and tile forms) times eight: every expert's tiles are independent problems, so the traffic
 # grows with the number of experts.  None: no capture of the current kernels.
-NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 8 * 8.809e9, "cfg5_slice": 8.809e9}
+NCU_DRAM_TRAFFIC_PER_STEP = {"cfg5_bf16_large": 8 * 8.825e9, "cfg5_slice": 8.825e9}
 NCU_DRAM_TRAFFIC_SOURCE = {
     "cfg5_bf16_large": "ncu counters of the six launches at cfg5_slice (one eighth of the experts, same tokens per "
                        "expert, widths and tile forms) times 8; not measured in this run",
