@@ -413,6 +413,8 @@ def main():
                          "workloads); the GEMM share for the roofline object is then taken from a "
                          "short eager loop before the timed region")
     args = ap.parse_args()
+    if args.gather and args.dy_fused:
+        ap.error("--gather and --dy-fused are separate routes: the backward without dy_perm reads x_perm")
     if args.forward_only:          # the end-to-end and CPU arms describe the fwd+bwd step only
         args.no_e2e = args.no_cpu_baseline = True
     wl = WORKLOADS[args.workload]

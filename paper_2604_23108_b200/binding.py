@@ -449,6 +449,7 @@ def layer_backward(cfg: Config, b: LayerBuffers, x, w_router, w13, w2, dy, aux=T
     combine_bwd does not read y_perm; otherwise combine_bwd computes it from y_perm.
     dy_fused: no combine_bwd and no dy_perm at all (mohge_expert_bwd_dy gathers the rows of dy)."""
     T = b.T
+    assert not (gather and dy_fused), "the backward without dy_perm reads x_perm: not with gather=True"
     if dy_fused:    # after a forward through x_perm
         if getattr(b, "hs", None) is None:
             b.hs = torch.empty_like(b.h)
